@@ -1,0 +1,149 @@
+/*
+ * soar.h - C ABI of the SOAR NVFP4 weight quantizer for NVIDIA B200 (sm_100a).
+ *
+ * The library turns a bf16 weight matrix into the NVFP4 triple of the SOAR paper
+ * (Sec. 3.1): 4-bit E2M1 codes, one FP8 E4M3 scale per 16 consecutive elements of
+ * a row, one FP32 scale per tensor; the scales and codes are chosen by Closed-form
+ * Joint Scale Optimization (Sec. 3.2, Eq. 4-6) and Decoupled Scale Search
+ * (Sec. 3.3, Eq. 7-8) run as the loop of Algorithm 1.
+ *
+ * Conventions that hold for every call
+ *   - "device" pointers are CUDA global memory owned by the caller; "host" pointers
+ *     are ordinary memory.  The library never allocates or frees device memory and
+ *     never synchronizes: work is enqueued on `stream` in order, so results are
+ *     readable once the caller has synchronized that stream.
+ *   - The int return value is a host-side status (SOAR_OK or a negative SOAR_ERR_*)
+ *     for argument and launch errors; nothing is enqueued when it is an argument error.
+ *     Conditions that depend on the data (non-finite input, all-zero tensor, magnitude
+ *     outside the supported range) are reported in soar_result.status on the device.
+ *   - Calls that share a workspace or output buffers must be ordered on one stream.
+ */
+#ifndef SOAR_H_
+#define SOAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SOAR_OK 0
+#define SOAR_ERR_INVALID_ARG (-1)      /* null pointer, bad struct size, bad count          */
+#define SOAR_ERR_UNSUPPORTED (-2)      /* cols % 16, ld < cols, alignment, block != 16, ... */
+#define SOAR_ERR_WORKSPACE (-3)        /* workspace missing or too small                    */
+#define SOAR_ERR_CUDA (-4)             /* a CUDA runtime call or kernel launch failed       */
+
+/* soar_result.status bits (device side, data dependent) */
+#define SOAR_STATUS_ZERO_TENSOR 1      /* every element is zero: alpha = 1, scales = 0      */
+#define SOAR_STATUS_NONFINITE 2        /* NaN or Inf in the input: outputs unspecified      */
+#define SOAR_STATUS_RANGE 4            /* max |W| outside [2^-100, 2^100]: outputs unspecified */
+
+/* scale_layout bits */
+#define SOAR_SCALES_LINEAR 1           /* row-major [rows][cols/16] bytes                   */
+#define SOAR_SCALES_SWIZZLED 2         /* 128x4 tiles as Blackwell block-scaled MMA reads   */
+
+/* presets for soar_default_cfg */
+#define SOAR_PRESET_PAPER 0            /* T=15, stop 1e-3, 2 E4M3 neighbours, 101 beta (Sec. 4.1, App. B.3) */
+#define SOAR_PRESET_SINGLE_PASS 1      /* T=1, no early stop, 2 neighbours, beta = {1}       */
+#define SOAR_PRESET_RTN 2              /* T=0: the max-based rule of Eq. 1-3 only            */
+
+#define SOAR_MAX_ITERS 64
+#define SOAR_MAX_BETA 512
+#define SOAR_MAX_DQ 16
+
+/* Search settings (host memory).  Names follow Algorithm 1 and App. B.3. */
+typedef struct soar_cfg {
+  uint32_t struct_size;   /* sizeof(soar_cfg), checked                                      */
+  int32_t block;          /* elements per E4M3 scale; 16 only (Sec. 3.1)                    */
+  int32_t max_iters;      /* T of Algorithm 1, 0..SOAR_MAX_ITERS; 0 = Eq. 1-3 only           */
+  float early_stop_rel;   /* stop after an iteration whose relative error gain is below this
+                             (Sec. 4.1: 1e-3); <= 0 disables                                */
+  int32_t n_dq;           /* E4M3 dequantization-scale candidates per block, 1..SOAR_MAX_DQ
+                             (App. B.3: 2, the codes bracketing the Eq. 6 solution; 1 = the
+                             nearest code; n >= 2: n/2 codes at or below, n/2 above)        */
+  int32_t n_beta;         /* multipliers of the quantization scale, 1..SOAR_MAX_BETA
+                             (App. B.3: 101, i.e. 0.50 .. 1.50); centred on 1.00            */
+  int32_t beta_step_pct;  /* multiplier step in hundredths (App. B.3: 1)                     */
+  int32_t scale_layout;   /* SOAR_SCALES_* bits: which scale outputs to write               */
+  int32_t flags;          /* reserved, must be 0                                            */
+} soar_cfg;
+
+/* Per-call report (device memory, written by the last kernel of soar_quantize). */
+typedef struct soar_result {
+  int32_t status;                           /* SOAR_STATUS_* bits                            */
+  int32_t iters_run;                        /* iterations of Algorithm 1 executed            */
+  float alpha;                              /* the FP32 global scale (same as *out_global)   */
+  float amax;                               /* max |W|                                       */
+  double sse;                               /* sum (W - What)^2 of the returned state (Eq. 4) */
+  double sse_init;                          /* same for the max-based start (Eq. 1-3)        */
+  double sumsq;                             /* sum W^2                                       */
+  int64_t zero_blocks;                      /* blocks whose 16 elements are all zero         */
+  int64_t wide_candidates;                  /* candidate evaluations that took the binary64
+                                               accumulation path (scale far below block max) */
+  double trace_alpha[SOAR_MAX_ITERS + 1];   /* alpha^(0), then alpha of each executed iteration */
+  double trace_sse[SOAR_MAX_ITERS + 1];     /* error of the start, then after each iteration */
+} soar_result;
+
+/* Fill *cfg (host) with a preset.  Returns SOAR_ERR_INVALID_ARG for a null pointer or
+ * unknown preset. */
+int soar_default_cfg(soar_cfg* cfg, int preset);
+
+/* Bytes of device scratch soar_quantize needs for this shape and cfg (0 on bad arguments).
+ * It is a small fixed part for the tensor-wide sums of Eq. 5 plus, when cfg->scale_layout
+ * lacks SOAR_SCALES_LINEAR, rows*cols/16 bytes for the row-major scales the loop works on. */
+size_t soar_workspace_bytes(int64_t rows, int64_t cols, const soar_cfg* cfg);
+
+/* Bytes of the swizzled scale buffer: scales padded to multiples of 128 rows and 4 columns. */
+size_t soar_swizzled_scale_bytes(int64_t rows, int64_t cols);
+
+/*
+ * Quantize one matrix with Algorithm 1 (max-based start of Eq. 1; per iteration the
+ * global scale of Eq. 5, the block scales of Eq. 6 and the search of Eq. 8 over
+ * cfg->n_beta x cfg->n_dq candidate pairs; early stop per Sec. 4.1).
+ *
+ *   W_bf16             device, read only: rows x cols bf16, row r at W + r*ld elements;
+ *                      blocks are 16 consecutive columns.  Base 16-byte aligned, ld % 8 == 0,
+ *                      ld >= cols, cols % 16 == 0, rows*cols/16 < 2^31.
+ *   cfg                host.
+ *   out_fp4_packed     device, rows*cols/2 bytes, 16-byte aligned.  Byte k of row r holds
+ *                      columns 2k (low nibble) and 2k+1 (high nibble); a nibble is
+ *                      sign<<3 | E2M1 magnitude code (0,.5,1,1.5,2,3,4,6 -> 0..7); the sign
+ *                      bit is the input's sign bit, also on zeros.
+ *   out_e4m3_scales    device, rows*cols/16 bytes row-major, or NULL when cfg->scale_layout
+ *                      lacks SOAR_SCALES_LINEAR.  An all-zero block gets scale byte 0x00.
+ *   out_e4m3_scales_sw device, soar_swizzled_scale_bytes() bytes, or NULL when
+ *                      cfg->scale_layout lacks SOAR_SCALES_SWIZZLED.  Padding bytes are zero.
+ *   out_global_fp32    device, one float: alpha, so that What = code value * alpha * scale (Eq. 3).
+ *   workspace          device scratch of at least soar_workspace_bytes(), 256-byte aligned;
+ *                      contents before the call are ignored, after it unspecified.
+ *   out_result         device, one soar_result, or NULL.
+ *   stream             a cudaStream_t passed as void* (NULL = the default stream).
+ */
+int soar_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld,
+                  const soar_cfg* cfg, void* out_fp4_packed, void* out_e4m3_scales,
+                  void* out_e4m3_scales_sw, float* out_global_fp32, void* workspace,
+                  size_t workspace_bytes, soar_result* out_result, void* stream);
+
+/*
+ * Reconstruction error of a stored NVFP4 triple against W (Eq. 3 and Eq. 4):
+ * *out_sse = sum (W - code value * alpha * scale)^2 and *out_sumsq = sum W^2, both
+ * accumulated in binary64.  All pointers device; scale_layout is exactly one SOAR_SCALES_*
+ * bit and names the layout of e4m3_scales.  W, rows, cols, ld as in soar_quantize.
+ */
+int soar_dequant_error(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld,
+                       const void* fp4_packed, const void* e4m3_scales, int scale_layout,
+                       const float* global_fp32, double* out_sse, double* out_sumsq,
+                       void* stream);
+
+/* Number of kernels soar_quantize enqueues for this cfg (host-side bookkeeping for callers
+ * that count launches); 0 on bad arguments. */
+int soar_quantize_launches(const soar_cfg* cfg);
+
+/* Text for a host-side return value. */
+const char* soar_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SOAR_H_ */

@@ -1,0 +1,192 @@
+"""Thin Python binding of the C ABI in include/soar.h.
+
+Argument marshalling only: every step of the quantizer runs in the CUDA kernels of
+libsoar.so.  torch is used for device memory and streams.  There is no CPU path; importing
+works without a GPU (so that symbols can be inspected), but every compute call requires
+CUDA tensors, and a missing library raises instead of falling back to anything.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libsoar.so")
+
+SOAR_OK = 0
+STATUS_ZERO_TENSOR, STATUS_NONFINITE, STATUS_RANGE = 1, 2, 4
+SCALES_LINEAR, SCALES_SWIZZLED = 1, 2
+PRESET_PAPER, PRESET_SINGLE_PASS, PRESET_RTN = 0, 1, 2
+MAX_ITERS = 64
+
+EXPORTS = (
+    "soar_default_cfg", "soar_workspace_bytes", "soar_swizzled_scale_bytes", "soar_quantize",
+    "soar_dequant_error", "soar_quantize_launches", "soar_status_string",
+)
+
+
+class SoarCfg(C.Structure):
+    """Mirror of ``soar_cfg``."""
+
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("block", C.c_int32), ("max_iters", C.c_int32),
+        ("early_stop_rel", C.c_float), ("n_dq", C.c_int32), ("n_beta", C.c_int32),
+        ("beta_step_pct", C.c_int32), ("scale_layout", C.c_int32), ("flags", C.c_int32),
+    ]
+
+
+class SoarResult(C.Structure):
+    """Mirror of ``soar_result``."""
+
+    _fields_ = [
+        ("status", C.c_int32), ("iters_run", C.c_int32), ("alpha", C.c_float), ("amax", C.c_float),
+        ("sse", C.c_double), ("sse_init", C.c_double), ("sumsq", C.c_double),
+        ("zero_blocks", C.c_int64), ("wide_candidates", C.c_int64),
+        ("trace_alpha", C.c_double * (MAX_ITERS + 1)), ("trace_sse", C.c_double * (MAX_ITERS + 1)),
+    ]
+
+
+class SoarError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libsoar.so (built in-tree by ``paper_2605_12245_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise SoarError(f"{LIB_PATH} is missing: run `python -m paper_2605_12245_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        vp, i64 = C.c_void_p, C.c_int64
+        L.soar_default_cfg.restype = C.c_int
+        L.soar_default_cfg.argtypes = [C.POINTER(SoarCfg), C.c_int]
+        L.soar_workspace_bytes.restype = C.c_size_t
+        L.soar_workspace_bytes.argtypes = [i64, i64, C.POINTER(SoarCfg)]
+        L.soar_swizzled_scale_bytes.restype = C.c_size_t
+        L.soar_swizzled_scale_bytes.argtypes = [i64, i64]
+        L.soar_quantize.restype = C.c_int
+        L.soar_quantize.argtypes = [vp, i64, i64, i64, C.POINTER(SoarCfg), vp, vp, vp, vp, vp,
+                                    C.c_size_t, vp, vp]
+        L.soar_dequant_error.restype = C.c_int
+        L.soar_dequant_error.argtypes = [vp, i64, i64, i64, vp, vp, C.c_int, vp, vp, vp, vp]
+        L.soar_quantize_launches.restype = C.c_int
+        L.soar_quantize_launches.argtypes = [C.POINTER(SoarCfg)]
+        L.soar_status_string.restype = C.c_char_p
+        L.soar_status_string.argtypes = [C.c_int]
+        _lib = L
+    return _lib
+
+
+def _check(rc: int, what: str):
+    if rc != SOAR_OK:
+        raise SoarError(f"{what}: {lib().soar_status_string(rc).decode()} ({rc})")
+
+
+def soar_default_cfg(preset: int = PRESET_PAPER, **overrides) -> SoarCfg:
+    cfg = SoarCfg()
+    _check(lib().soar_default_cfg(C.byref(cfg), preset), "soar_default_cfg")
+    for k, v in overrides.items():
+        if not hasattr(cfg, k):
+            raise AttributeError(k)
+        setattr(cfg, k, v)
+    return cfg
+
+
+def soar_workspace_bytes(rows: int, cols: int, cfg: SoarCfg) -> int:
+    return int(lib().soar_workspace_bytes(rows, cols, C.byref(cfg)))
+
+
+def soar_swizzled_scale_bytes(rows: int, cols: int) -> int:
+    return int(lib().soar_swizzled_scale_bytes(rows, cols))
+
+
+def soar_quantize_launches(cfg: SoarCfg) -> int:
+    return int(lib().soar_quantize_launches(C.byref(cfg)))
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _require_cuda(*tensors):
+    for t in tensors:
+        if t is not None and not t.is_cuda:
+            raise SoarError("device pointers required: tensor is not on a CUDA device")
+
+
+@dataclass
+class QuantBuffers:
+    """Device buffers of one quantized matrix; allocate once, reuse across calls."""
+
+    packed: torch.Tensor            # uint8 [rows, cols/2]
+    scales: torch.Tensor | None     # uint8 [rows, cols/16] (linear layout)
+    scales_sw: torch.Tensor | None  # uint8 [soar_swizzled_scale_bytes]
+    alpha: torch.Tensor             # float32 [1]
+    result: torch.Tensor            # uint8 [sizeof(soar_result)]
+    workspace: torch.Tensor         # uint8
+
+    def read_result(self) -> SoarResult:
+        """Synchronizing copy of the device report to the host."""
+        raw = self.result.cpu().numpy().tobytes()
+        return SoarResult.from_buffer_copy(raw)
+
+
+def alloc_buffers(rows: int, cols: int, cfg: SoarCfg, device="cuda") -> QuantBuffers:
+    u8 = dict(dtype=torch.uint8, device=device)
+    lin = torch.empty((rows, cols // 16), **u8) if cfg.scale_layout & SCALES_LINEAR else None
+    sw = (torch.empty(soar_swizzled_scale_bytes(rows, cols), **u8)
+          if cfg.scale_layout & SCALES_SWIZZLED else None)
+    ws_bytes = soar_workspace_bytes(rows, cols, cfg)
+    if ws_bytes == 0:
+        raise SoarError("soar_workspace_bytes rejected the shape or cfg")
+    return QuantBuffers(
+        packed=torch.empty((rows, cols // 2), **u8), scales=lin, scales_sw=sw,
+        alpha=torch.empty(1, dtype=torch.float32, device=device),
+        result=torch.empty(C.sizeof(SoarResult), **u8),
+        workspace=torch.empty(ws_bytes, **u8),
+    )
+
+
+def soar_quantize(W: torch.Tensor, cfg: SoarCfg, out: QuantBuffers | None = None, stream=None,
+                  ld: int | None = None) -> QuantBuffers:
+    """Enqueue ``soar_quantize`` for a bf16 CUDA matrix (2-D, unit column stride)."""
+    _require_cuda(W)
+    if W.dtype != torch.bfloat16 or W.dim() != 2 or W.stride(1) != 1:
+        raise SoarError("W must be a 2-D bf16 tensor with unit column stride")
+    rows, cols = W.shape
+    ld = W.stride(0) if ld is None else ld
+    if out is None:
+        out = alloc_buffers(rows, cols, cfg, W.device)
+    _require_cuda(out.packed, out.scales, out.scales_sw, out.alpha, out.result, out.workspace)
+    rc = lib().soar_quantize(
+        _ptr(W), rows, cols, ld, C.byref(cfg), _ptr(out.packed), _ptr(out.scales),
+        _ptr(out.scales_sw), _ptr(out.alpha), _ptr(out.workspace), out.workspace.numel(),
+        _ptr(out.result), _stream_ptr(stream))
+    _check(rc, "soar_quantize")
+    return out
+
+
+def soar_dequant_error(W: torch.Tensor, packed: torch.Tensor, scales: torch.Tensor,
+                       alpha: torch.Tensor, scale_layout: int = SCALES_LINEAR, stream=None,
+                       out: torch.Tensor | None = None) -> torch.Tensor:
+    """Enqueue ``soar_dequant_error``; returns a float64 CUDA tensor [sse, sumsq]."""
+    _require_cuda(W, packed, scales, alpha)
+    rows, cols = W.shape
+    if out is None:
+        out = torch.empty(2, dtype=torch.float64, device=W.device)
+    rc = lib().soar_dequant_error(
+        _ptr(W), rows, cols, W.stride(0), _ptr(packed), _ptr(scales), scale_layout, _ptr(alpha),
+        C.c_void_p(out.data_ptr()), C.c_void_p(out.data_ptr() + 8), _stream_ptr(stream))
+    _check(rc, "soar_dequant_error")
+    return out

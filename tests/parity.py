@@ -1,0 +1,98 @@
+"""Helpers shared by the GPU parity tests: run the CUDA library through its C ABI on bf16
+bit patterns, run the CPU oracle on the same bytes, and compare block by block.
+
+Comparison rule: E2M1 codes and E4M3 scale bytes must be bit-exact, except in blocks the
+oracle flags as ties (its best two distinct candidate outcomes within 1e-6 relative in some
+iteration); mismatching blocks are counted and must stay below 0.01 % of all blocks.  The
+global scale must agree within 1e-6 relative and the reconstruction error within 1e-5.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+from oracle import soar_ref as R
+from paper_2605_12245_b200 import api
+
+ALPHA_RTOL = 1e-6
+SSE_RTOL = 1e-5
+MAX_MISMATCH_FRACTION = 1e-4
+
+
+def to_device(w_bits: np.ndarray, ld: int | None = None) -> torch.Tensor:
+    """uint16 bit patterns -> bf16 CUDA tensor (optionally with a padded row stride)."""
+    rows, cols = w_bits.shape
+    t = torch.from_numpy(w_bits.view(np.int16)).cuda().view(torch.bfloat16)
+    if ld is None or ld == cols:
+        return t
+    buf = torch.full((rows, ld), float("nan"), dtype=torch.bfloat16, device="cuda")
+    buf[:, :cols] = t
+    return buf[:, :cols]
+
+
+def cfg_pair(**kw):
+    """Matching (library cfg, oracle cfg) from keyword overrides of the paper's preset."""
+    ref = R.RefCfg(**kw)
+    cfg = api.soar_default_cfg(api.PRESET_PAPER, max_iters=ref.max_iters,
+                               early_stop_rel=ref.early_stop_rel, n_dq=ref.n_dq,
+                               n_beta=ref.n_beta, beta_step_pct=ref.beta_step_pct)
+    return cfg, ref
+
+
+@dataclass
+class GpuOut:
+    packed: np.ndarray
+    scales: np.ndarray
+    alpha: float
+    result: api.SoarResult
+    buffers: api.QuantBuffers
+
+
+def run_gpu(w_bits: np.ndarray, cfg, ld: int | None = None) -> GpuOut:
+    W = to_device(w_bits, ld)
+    out = api.soar_quantize(W, cfg)
+    torch.cuda.synchronize()
+    res = out.read_result()
+    scales = out.scales.cpu().numpy() if out.scales is not None else None
+    return GpuOut(out.packed.cpu().numpy(), scales, float(out.alpha.cpu()[0]), res, out)
+
+
+@dataclass
+class Report:
+    blocks: int
+    mismatched: int
+    mismatched_outside_ties: int
+    tie_blocks: int
+    alpha_rel: float
+    sse_rel: float
+
+
+def compare(gpu: GpuOut, ref: R.RefResult) -> Report:
+    rows, nb = ref.scales.shape
+    code_diff = (gpu.packed != ref.packed).reshape(rows, nb, 8).any(axis=2)
+    scale_diff = gpu.scales != ref.scales
+    bad = code_diff | scale_diff
+    ties = ref.tie_flags.astype(bool)
+    alpha_rel = abs(gpu.alpha - ref.alpha) / abs(ref.alpha) if ref.alpha else abs(gpu.alpha - ref.alpha)
+    ref_sse = ref.trace_sse[-1]
+    sse_rel = abs(gpu.result.sse - ref_sse) / ref_sse if ref_sse else abs(gpu.result.sse)
+    return Report(rows * nb, int(bad.sum()), int((bad & ~ties).sum()), int(ties.sum()),
+                  float(alpha_rel), float(sse_rel))
+
+
+def assert_parity(gpu: GpuOut, ref: R.RefResult) -> Report:
+    rep = compare(gpu, ref)
+    assert gpu.result.status == ref.status
+    assert gpu.result.iters_run == ref.iters_run, (gpu.result.iters_run, ref.iters_run)
+    assert rep.alpha_rel <= ALPHA_RTOL, rep
+    assert rep.mismatched_outside_ties == 0, rep
+    assert rep.mismatched <= MAX_MISMATCH_FRACTION * rep.blocks, rep
+    assert rep.sse_rel <= SSE_RTOL, rep
+    n = ref.iters_run + 1
+    ta = np.array(gpu.result.trace_alpha[:n])
+    ts = np.array(gpu.result.trace_sse[:n])
+    assert np.allclose(ta, ref.trace_alpha, rtol=ALPHA_RTOL, atol=0), (ta, ref.trace_alpha)
+    assert np.allclose(ts, ref.trace_sse, rtol=SSE_RTOL, atol=0), (ts, ref.trace_sse)
+    return rep

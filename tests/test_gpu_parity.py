@@ -1,0 +1,181 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the
+same seeded bytes.  Shapes span several CTAs' worth of blocks, ragged tails and padded row
+strides; settings cover the paper's preset and the smaller candidate grids."""
+import ml_dtypes
+import numpy as np
+import pytest
+import torch
+
+from oracle import soar_ref as R
+from paper_2605_12245_b200 import api
+from paper_2605_12245_b200 import workloads as WL
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("rows,cols,ld,seed,kw", [
+    (1, 16, None, 0, {}),
+    (3, 48, 64, 1, {}),
+    (37, 1040, None, 2, dict(outlier_entry_frac=0.01, outlier_scale=50.0)),
+    (130, 2064, 2072, 3, dict(dist="laplace", outlier_cols_frac=0.01, outlier_scale=20.0)),
+    (257, 4096, None, 4, dict(dist="gauss_t2mix")),
+])
+@pytest.mark.parametrize("cfgkw", [
+    dict(),                                                   # the paper's preset
+    dict(max_iters=0),                                        # Eq. 1-3 only
+    dict(max_iters=1, early_stop_rel=0.0, n_dq=2, n_beta=1),  # single pass
+    dict(max_iters=3, early_stop_rel=0.0, n_dq=1, n_beta=1),  # CJSO with the nearest scale
+    dict(max_iters=2, early_stop_rel=0.0, n_dq=4, n_beta=6, beta_step_pct=3),
+])
+def test_parity_small(rows, cols, ld, seed, kw, cfgkw):
+    w = WL.small_case(rows, cols, seed, **kw)
+    cfg, ref_cfg = P.cfg_pair(**cfgkw)
+    gpu = P.run_gpu(w, cfg, ld)
+    ref = R.quantize(w, ref_cfg)
+    P.assert_parity(gpu, ref)
+    assert gpu.result.sumsq == pytest.approx(ref.sumsq, rel=1e-12)
+
+
+def test_parity_medium_paper_preset():
+    """512 x 2048 with outlier columns: 65 536 blocks, full 15 x 202 search."""
+    w = WL.small_case(512, 2048, 11, outlier_cols_frac=0.001, outlier_scale=20.0)
+    cfg, ref_cfg = P.cfg_pair()
+    rep = P.assert_parity(P.run_gpu(w, cfg), R.quantize(w, ref_cfg))
+    print("medium:", rep)
+
+
+def test_rounding_ties_e2m1_and_e4m3():
+    """Inputs built so that |W|/(alpha*scale) lands exactly on E2M1 midpoints and
+    bmax/(6 alpha) exactly on E4M3 midpoints: both sides must break the ties alike."""
+    e4 = np.arange(0x7F, dtype=np.uint8).view(ml_dtypes.float8_e4m3fn).astype(np.float64)
+    unit = 2.0 ** -10                       # alpha0 = amax/2688 = 2^-10 exactly
+    rows = []
+    mids = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 6.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 0.0, 5.5])
+    for c in range(0x28, 0x7E, 3):          # block scales with exact products in bf16
+        s = e4[c]
+        blk = mids * s * unit
+        blk[7] = 6.0 * s * unit             # block max pins the scale to code c
+        rows.append(blk)
+    for c in range(0x30, 0x7D):             # block max on the midpoint between codes c and c+1
+        mid = 0.5 * (e4[c] + e4[c + 1])
+        blk = np.zeros(16)
+        blk[0] = 6.0 * mid * unit
+        blk[1:8] = mids[:7] * e4[c] * unit
+        rows.append(blk)
+    top = np.zeros(16); top[0] = 2688.0 * unit
+    rows.append(top)
+    w = np.array(rows, np.float32)
+    w = np.concatenate([w, -w], axis=0)
+    bits = WL.f32_to_bf16_bits(w)
+    assert np.array_equal(WL.bf16_bits_to_f32(bits), w), "test values must be exact in bf16"
+    for cfgkw in (dict(max_iters=0), dict(max_iters=2, early_stop_rel=0.0)):
+        cfg, ref_cfg = P.cfg_pair(**cfgkw)
+        P.assert_parity(P.run_gpu(bits, cfg), R.quantize(bits, ref_cfg))
+
+
+def test_degenerate_blocks_and_tensors():
+    w = WL.small_case(8, 256, 20)
+    w[1, 16:32] = 0
+    w[1, 20] = 0x8000                                        # negative zero inside a zero block
+    w[2, 32:48] = WL.f32_to_bf16_bits(np.full(16, 1e-12, np.float32))
+    cfg, ref_cfg = P.cfg_pair(max_iters=3)
+    gpu = P.run_gpu(w, cfg)
+    P.assert_parity(gpu, R.quantize(w, ref_cfg))
+    assert gpu.result.zero_blocks == 1
+    z = np.zeros((4, 64), np.uint16); z[0, 5] = 0x8000
+    gz, rz = P.run_gpu(z, cfg), R.quantize(z, ref_cfg)
+    assert gz.result.status == api.STATUS_ZERO_TENSOR == rz.status
+    assert gz.alpha == 1.0 and np.array_equal(gz.packed, rz.packed) and not gz.scales.any()
+    bad = w.copy(); bad[3, 7] = 0x7FC0
+    assert P.run_gpu(bad, cfg).result.status & api.STATUS_NONFINITE
+    bad[3, 7] = 0xFF80
+    assert P.run_gpu(bad, cfg).result.status & api.STATUS_NONFINITE
+    tiny = WL.f32_to_bf16_bits(np.full((2, 32), 1e-35, np.float32))
+    assert P.run_gpu(tiny, cfg).result.status & api.STATUS_RANGE
+
+
+def test_wide_candidates_take_the_exact_path():
+    """One element 200x above the rest of its block: candidates with a scale fit to the
+    small elements saturate the large one far beyond 32 and must still be scored exactly."""
+    rng = np.random.default_rng(5)
+    w = (rng.standard_normal((16, 256)) * 0.01).astype(np.float32)
+    w[:, ::16] *= 300.0
+    bits = WL.f32_to_bf16_bits(w)
+    cfg, ref_cfg = P.cfg_pair(max_iters=2, early_stop_rel=0.0, n_dq=2, n_beta=101, beta_step_pct=1)
+    gpu = P.run_gpu(bits, cfg)
+    P.assert_parity(gpu, R.quantize(bits, ref_cfg))
+
+
+def test_argument_errors_are_reported_on_the_host():
+    w = P.to_device(WL.small_case(4, 64, 0))
+    cfg = api.soar_default_cfg()
+    with pytest.raises(api.SoarError):
+        api.soar_quantize(w[:, :40], cfg)                      # cols % 16 != 0
+    bad = api.soar_default_cfg(block=32)
+    with pytest.raises(api.SoarError):
+        api.soar_quantize(w, bad)
+    out = api.alloc_buffers(4, 64, cfg)
+    out.workspace = out.workspace[:16]
+    with pytest.raises(api.SoarError):
+        api.soar_quantize(w, cfg, out)
+    with pytest.raises(api.SoarError):
+        api.soar_quantize(w.cpu(), cfg)
+
+
+def swizzle_reference(lin: np.ndarray) -> np.ndarray:
+    """128x4-tiled scale layout written with array reshapes (independent of the kernel's
+    index formula): pad to (128k, 4m); a tile is stored as [32 rows][4 row-groups][4 cols]."""
+    rows, nbc = lin.shape
+    rt, ct = -(-rows // 128), -(-nbc // 4)
+    pad = np.zeros((rt * 128, ct * 4), np.uint8)
+    pad[:rows, :nbc] = lin
+    t = pad.reshape(rt, 4, 32, ct, 4)          # [row tile][row group][row in group][col tile][col]
+    return t.transpose(0, 3, 2, 1, 4).reshape(-1)
+
+
+@pytest.mark.parametrize("rows,cols", [(128, 64), (130, 16 * 5), (300, 16 * 33)])
+def test_swizzled_scale_layout(rows, cols):
+    w = WL.small_case(rows, cols, 31)
+    both = api.soar_default_cfg(api.PRESET_SINGLE_PASS, scale_layout=api.SCALES_LINEAR | api.SCALES_SWIZZLED)
+    g = P.run_gpu(w, both)
+    sw = g.buffers.scales_sw.cpu().numpy()
+    assert sw.size == api.soar_swizzled_scale_bytes(rows, cols)
+    assert np.array_equal(sw, swizzle_reference(g.scales))
+    only = api.soar_default_cfg(api.PRESET_SINGLE_PASS, scale_layout=api.SCALES_SWIZZLED)
+    W = P.to_device(w)
+    o = api.soar_quantize(W, only)
+    torch.cuda.synchronize()
+    assert o.scales is None
+    assert np.array_equal(o.scales_sw.cpu().numpy(), sw)
+    assert np.array_equal(o.packed.cpu().numpy(), g.packed)
+    # the error kernel reads either layout
+    e_lin = api.soar_dequant_error(W, g.buffers.packed, g.buffers.scales, g.buffers.alpha).cpu().numpy()
+    e_sw = api.soar_dequant_error(W, o.packed, o.scales_sw, o.alpha, api.SCALES_SWIZZLED).cpu().numpy()
+    assert e_lin[0] == pytest.approx(e_sw[0], rel=1e-12)
+    assert e_lin[0] == pytest.approx(g.result.sse, rel=1e-9)
+
+
+def test_dequant_error_matches_oracle():
+    w = WL.small_case(96, 1024, 41, outlier_entry_frac=0.002, outlier_scale=50.0)
+    cfg, ref_cfg = P.cfg_pair(max_iters=2)
+    g = P.run_gpu(w, cfg, ld=1040)
+    W = P.to_device(w, 1040)
+    e = api.soar_dequant_error(W, g.buffers.packed, g.buffers.scales, g.buffers.alpha).cpu().numpy()
+    sse, ss = R.dequant_error(w, g.packed, g.scales, g.alpha)
+    assert e[0] == pytest.approx(sse, rel=1e-12)
+    assert e[1] == pytest.approx(ss, rel=1e-12)
+    assert g.result.sse == pytest.approx(sse, rel=1e-9)
+
+
+def test_two_calls_share_a_workspace_and_repeat_exactly():
+    w1, w2 = WL.small_case(64, 512, 50), WL.small_case(64, 512, 51)
+    cfg, _ = P.cfg_pair(max_iters=2)
+    out = api.alloc_buffers(64, 512, cfg)
+    a = api.soar_quantize(P.to_device(w1), cfg, out); torch.cuda.synchronize()
+    p1, s1, al1 = a.packed.cpu().numpy().copy(), a.scales.cpu().numpy().copy(), float(a.alpha.cpu()[0])
+    api.soar_quantize(P.to_device(w2), cfg, out)
+    api.soar_quantize(P.to_device(w1), cfg, out); torch.cuda.synchronize()
+    assert np.array_equal(out.packed.cpu().numpy(), p1)
+    assert np.array_equal(out.scales.cpu().numpy(), s1)
+    assert float(out.alpha.cpu()[0]) == al1
