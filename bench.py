@@ -1,0 +1,382 @@
+#!/usr/bin/env python
+"""Benchmark of the SOAR NVFP4 quantize pass on B200.
+
+One "step" quantizes every tensor of the workload once (the whole hot path: tensor
+maximum, max-based start, the CJSO + DSS iterations, alpha and the report), through the
+C-ABI library with all inputs already resident in HBM.  Prints ONE JSON line on stdout.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--workload config1|config2|config3|config4|config5] [--preset paper|single_pass]
+
+Multi-GPU runs are launched by torch.distributed.run, one rank per GPU; the tensors of a
+model are independent, so every rank quantizes its own copy of the workload with no
+collective on the data path (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2605_12245_b200 import workloads as WL  # noqa: E402
+
+SM_COUNT = 148
+FP32_LANES_PER_SM = 128
+# Instructions an element of one candidate needs at the least: scale multiply, rounding to
+# the E2M1 grid, and the two accumulations of Eq. 5/6's block sums.
+OPS_PER_ELEMENT_EVAL = 4
+OPS_PER_PAIR_SCORE = 3
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), sm_max_mhz=float(p.get("sm_max_mhz", 1965.0)), source="measured")
+    return dict(hbm_gbs=6650.0, sm_max_mhz=1965.0, source="fallback")
+
+
+def pick_workload(name: str):
+    if name == "config1":
+        return WL.config1()
+    if name == "config2":
+        return WL.config2()
+    if name == "config4":
+        return WL.config4()
+    if name == "config5":
+        return WL.config5()
+    raise SystemExit(f"unknown workload {name}")
+
+
+def preset_cfg(api, preset: str, **over):
+    base = api.PRESET_PAPER if preset == "paper" else api.PRESET_SINGLE_PASS
+    return api.soar_default_cfg(base, **over)
+
+
+def ref_cfg_of(R, cfg):
+    return R.RefCfg(max_iters=cfg.max_iters, early_stop_rel=cfg.early_stop_rel, n_dq=cfg.n_dq,
+                    n_beta=cfg.n_beta, beta_step_pct=cfg.beta_step_pct)
+
+
+# Algorithmic work per 16-element block (what the method itself demands)
+def iterate_ops_per_block(cfg) -> float:
+    return cfg.n_beta * (16 * OPS_PER_ELEMENT_EVAL + cfg.n_dq * OPS_PER_PAIR_SCORE)
+
+
+KERNEL_BYTES_PER_ELEM = {          # algorithmic HBM bytes per weight element and launch
+    "amax_kernel": 2.0,                                  # read W
+    "init_kernel": 2.0 + 0.5 + 1.0 / 16,                 # read W, write codes + scale byte
+    "iterate_kernel": 2.0 + 2 * (0.5 + 1.0 / 16),        # read W, codes, scale; write codes, scale
+    "dequant_error_kernel": 2.0 + 0.5 + 1.0 / 16,
+}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        # samples under load: the upper half of the observed clocks (idle samples sit far below)
+        load = sorted(sm)[len(sm) // 2:] if sm else []
+        return dict(sm_mhz=statistics.median(load) if load else None,
+                    sm_max_mhz=max(mx) if mx else None, samples=len(sm), reasons=sorted(reasons))
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, on a bounded sample of the same workload and preset."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import soar_ref as R
+    from paper_2605_12245_b200 import api
+    wl = pick_workload(args.workload)
+    cfg = preset_cfg(api, args.preset)
+    rcfg = ref_cfg_of(R, cfg)
+    spec = wl.tensors[0]
+    rows = min(spec.rows, max(1, args.ref_rows))
+    rows = max(1, rows // WL._chunk_rows(spec.cols)) * WL._chunk_rows(spec.cols)
+    w = WL.generate(wl, 0, 0, rows)
+    for _ in range(args.warmup):
+        R.quantize(w[: max(1, rows // 8)], rcfg)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        R.quantize(w, rcfg)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = 2.0 * w.size / dt / 1e9
+    sample = f"{rows} rows x {spec.cols} cols of tensor '{spec.name}' of {wl.name} per step"
+    line = dict(
+        impl="reference", metric="soar_quantize_bf16_input_throughput", value=value, unit="GB/s",
+        n_gpus=args.gpus, steps=args.steps, warmup=args.warmup, ms_per_step=dt * 1e3,
+        higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32", data="synthetic",
+        config=dict(workload=wl.name, preset=args.preset, max_iters=cfg.max_iters, n_beta=cfg.n_beta,
+                    n_dq=cfg.n_dq, early_stop_rel=cfg.early_stop_rel, sample=sample),
+        cpu_baseline=dict(value=value, unit="GB/s", cores=R.num_threads(), kind="oracle", sample=sample),
+        e2e=dict(value=value, unit="GB/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+        elements_per_s=w.size / dt, gpu_launches=0,
+    )
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2605_12245_b200 import api
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    api.lib()
+    peaks = load_peaks()
+    wl = pick_workload(args.workload)
+    cfg = preset_cfg(api, args.preset)
+
+    # ---- inputs: generated on the host (seeded), resident in HBM before timing
+    host_w, dev_w, outs = [], [], []
+    for i, spec in enumerate(wl.tensors):
+        bits = WL.generate(wl, i)
+        h = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+        host_w.append(h)
+        dev_w.append(h.cuda())
+        outs.append(api.alloc_buffers(spec.rows, spec.cols, cfg))
+    elements = wl.elements
+    stream = torch.cuda.current_stream()
+
+    def step(c=cfg):
+        for W, o in zip(dev_w, outs):
+            api.soar_quantize(W, c, o, stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup, trace=True):
+        for _ in range(warmup):
+            fn()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if trace:
+            api.soar_trace_begin()
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        tr = api.soar_trace_end() if trace else {}
+        barrier()
+        ms = e0.elapsed_time(e1) / steps
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, tr
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms, trace = timed(step, args.steps, args.warmup)
+    clocks = sampler.stop()
+    results = [o.read_result() for o in outs]
+    iters = [r.iters_run for r in results]
+    value = world * 2.0 * elements / (ms * 1e-3) / 1e9
+    launches = sum(v[0] for v in trace.values())
+
+    # ---- roofline of the dominant kernel
+    dom = max(trace, key=lambda k: trace[k][1])
+    n_launch, tot_ms = trace[dom]
+    if dom == "iterate_kernel" and iterate_ops_per_block(cfg) > 16 * 180:
+        # candidate loop dominates: bound by plain FP32/INT issue
+        blocks_iters = sum((s.rows * s.cols // 16) * it for s, it in zip(wl.tensors, iters)) * args.steps
+        ops = blocks_iters * iterate_ops_per_block(cfg)
+        achieved = ops / (tot_ms * 1e-3) / 1e12
+        peak = SM_COUNT * FP32_LANES_PER_SM * peaks["sm_max_mhz"] * 1e6 / 1e12
+        roofline = dict(bound="alu", kernel=dom, achieved=achieved, peak=peak, unit="Tlane-op/s",
+                        frac=achieved / peak, traffic=None, launches=n_launch,
+                        active_launches=sum(iters) * args.steps, kernel_ms_per_step=tot_ms / args.steps,
+                        peak_source="148 SMs x 128 FP32 lanes x clocks.max.sm",
+                        hbm_gbs_for_context=blocks_iters * 16 * KERNEL_BYTES_PER_ELEM[dom] / (tot_ms * 1e-3) / 1e9)
+    else:
+        if dom == "iterate_kernel":
+            units = sum(s.rows * s.cols * it for s, it in zip(wl.tensors, iters)) * args.steps
+        else:
+            units = elements * args.steps
+        byts = units * KERNEL_BYTES_PER_ELEM.get(dom, 2.0)
+        achieved = byts / (tot_ms * 1e-3) / 1e9
+        roofline = dict(bound="hbm", kernel=dom, achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
+                        frac=achieved / peaks["hbm_gbs"], traffic=None, launches=n_launch,
+                        kernel_ms_per_step=tot_ms / args.steps, peak_source=peaks["source"],
+                        frac_of_nominal_8000=achieved / 8000.0)
+    kernels = {k: dict(launches=v[0], ms_per_step=v[1] / args.steps, share=v[1] / sum(x[1] for x in trace.values()))
+               for k, v in trace.items()}
+
+    # ---- the HBM-bound shape of the same path (T=1, beta={1}, 2 neighbours), for the bandwidth bar
+    extra = {}
+    if args.preset == "paper" and not args.no_single_pass:
+        sp = preset_cfg(api, "single_pass")
+        sp_ms, sp_tr = timed(lambda: step(sp), max(args.steps, 5), 3)
+        sp_bytes = elements * (KERNEL_BYTES_PER_ELEM["amax_kernel"] + KERNEL_BYTES_PER_ELEM["init_kernel"]
+                               + KERNEL_BYTES_PER_ELEM["iterate_kernel"])
+        gbs = sp_bytes / (sp_ms * 1e-3) / 1e9
+        extra["single_pass"] = dict(
+            ms_per_step=sp_ms, value=world * 2.0 * elements / (sp_ms * 1e-3) / 1e9, unit="GB/s",
+            algorithmic_bytes_per_step=sp_bytes, achieved_gbs=gbs, frac_of_measured_hbm=gbs / peaks["hbm_gbs"],
+            frac_of_nominal_8000=gbs / 8000.0,
+            kernels={k: dict(launches=v[0], ms_per_step=v[1] / max(args.steps, 5)) for k, v in sp_tr.items()})
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    import ctypes
+    ctypes_sizeof_result = ctypes.sizeof(api.SoarResult)
+    e2e = None
+    if not args.no_e2e:
+        big = max(wl.tensors, key=lambda s: s.rows * s.cols)
+        streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        stage = [(torch.empty((big.rows * big.cols,), dtype=torch.bfloat16, device="cuda"),
+                  api.alloc_buffers(big.rows, big.cols, cfg)) for _ in streams]
+        hosts = []
+        for h, spec in zip(host_w, wl.tensors):
+            hb = api.alloc_host_buffers(spec.rows, spec.cols, cfg)
+            hb.W.copy_(h)
+            hosts.append(hb)
+
+        def e2e_step():
+            for i, (hb, spec) in enumerate(zip(hosts, wl.tensors)):
+                s = streams[i % 2]
+                dW, big_out = stage[i % 2]
+                n = spec.rows * spec.cols
+                view = api.QuantBuffers(
+                    packed=big_out.packed.view(-1)[: n // 2].view(spec.rows, spec.cols // 2),
+                    scales=big_out.scales.view(-1)[: n // 16].view(spec.rows, spec.cols // 16),
+                    scales_sw=None, alpha=big_out.alpha, result=big_out.result, workspace=big_out.workspace)
+                api.soar_quantize_host(hb, cfg, dW[:n].view(spec.rows, spec.cols), view, s)
+
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            e2e_step()
+        torch.cuda.synchronize()
+        dt = (time.perf_counter() - t0) / args.steps
+        if world > 1:
+            t = torch.tensor([dt], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        # results must equal the resident-input run
+        assert hosts[0].read_result().iters_run == iters[0]
+        e2e = dict(value=world * 2.0 * elements / dt / 1e9, unit="GB/s", ms_per_step=dt * 1e3,
+                   h2d_bytes_per_step=2 * elements,
+                   d2h_bytes_per_step=elements // 2 + elements // 16 + len(wl.tensors) * (4 + ctypes_sizeof_result),
+                   api="soar_quantize_host, two streams, pinned host buffers")
+
+    # ---- the oracle on the host cores, bounded sample (rank 0, single GPU only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        from oracle import soar_ref as R
+        spec = wl.tensors[0]
+        rows = max(1, min(spec.rows, args.cpu_rows) // WL._chunk_rows(spec.cols)) * WL._chunk_rows(spec.cols)
+        w = host_w[0][:rows].view(torch.int16).numpy().view(np.uint16)
+        t0 = time.perf_counter()
+        ref = R.quantize(w, ref_cfg_of(R, cfg))
+        dt = time.perf_counter() - t0
+        cpu = dict(value=2.0 * w.size / dt / 1e9, unit="GB/s", cores=R.num_threads(), kind="oracle",
+                   sample=f"first {rows} rows x {spec.cols} cols of tensor '{spec.name}', {ref.iters_run} iterations, {dt:.1f} s",
+                   elements_per_s=w.size / dt)
+
+    if rank == 0:
+        line = dict(
+            metric="soar_quantize_bf16_input_throughput", value=value, unit="GB/s", n_gpus=world,
+            steps=args.steps, warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak",
+            vs_baseline=None, dtype="f32", data="synthetic",
+            config=dict(workload=wl.name, preset=args.preset, max_iters=cfg.max_iters, n_beta=cfg.n_beta,
+                        n_dq=cfg.n_dq, early_stop_rel=cfg.early_stop_rel, tensors=len(wl.tensors),
+                        elements=elements, iters_run=iters,
+                        l2="inputs (%.2f GB per step) exceed the 126 MB L2" % (2 * elements / 1e9),
+                        parallelism=f"replicated workload x{world}, no collective"),
+            elements_per_s=world * elements / (ms * 1e-3),
+            hbm_frac_end_to_end_of_measured=value / peaks["hbm_gbs"],
+            roofline=roofline, kernels=kernels, cpu_baseline=cpu, e2e=e2e, gpu_launches=launches,
+            clocks=clocks, **extra)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="config4")
+    ap.add_argument("--preset", default="paper", choices=["paper", "single_pass"])
+    ap.add_argument("--cpu-rows", type=int, default=256, help="rows of tensor 0 the CPU baseline quantizes")
+    ap.add_argument("--ref-rows", type=int, default=128, help="rows per step of the reference arm")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-single-pass", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -125,6 +125,32 @@ int soar_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld,
                   void* out_e4m3_scales_sw, float* out_global_fp32, void* workspace,
                   size_t workspace_bytes, soar_result* out_result, void* stream);
 
+/* Device staging buffers for soar_quantize_host (all device memory, caller-owned, same sizes
+ * and alignment as the matching soar_quantize arguments; W holds rows*ld bf16 elements). */
+typedef struct soar_staging {
+  void* W;
+  void* packed;
+  void* scales;        /* NULL when cfg lacks SOAR_SCALES_LINEAR   */
+  void* scales_sw;     /* NULL when cfg lacks SOAR_SCALES_SWIZZLED */
+  float* alpha;
+  soar_result* result; /* NULL when no report is wanted            */
+  void* workspace;
+  size_t workspace_bytes;
+} soar_staging;
+
+/*
+ * soar_quantize for a matrix that lives in host memory (Algorithm 1, same outputs): copies
+ * W host->device into dev->W, runs soar_quantize on the staging buffers, and copies the
+ * codes, scales, alpha and report back to the host pointers, all enqueued in order on
+ * `stream`.  Host buffers should be page-locked for the copies to be asynchronous; they are
+ * valid after the caller synchronizes the stream.  out_*_host pointers follow the rules of
+ * the matching soar_quantize outputs (NULL where the layout is not requested).
+ */
+int soar_quantize_host(const void* W_host, int64_t rows, int64_t cols, int64_t ld,
+                       const soar_cfg* cfg, void* out_fp4_packed_host, void* out_e4m3_scales_host,
+                       void* out_e4m3_scales_sw_host, float* out_global_host,
+                       soar_result* out_result_host, const soar_staging* dev, void* stream);
+
 /*
  * Reconstruction error of a stored NVFP4 triple against W (Eq. 3 and Eq. 4):
  * *out_sse = sum (W - code value * alpha * scale)^2 and *out_sumsq = sum W^2, both
@@ -139,6 +165,19 @@ int soar_dequant_error(const void* W_bf16, int64_t rows, int64_t cols, int64_t l
 /* Number of kernels soar_quantize enqueues for this cfg (host-side bookkeeping for callers
  * that count launches); 0 on bad arguments. */
 int soar_quantize_launches(const soar_cfg* cfg);
+
+/* Launch tracing for benchmarks (no counterpart in the paper).  Between soar_trace_begin()
+ * and soar_trace_end(), every kernel the library launches is bracketed by two CUDA events on
+ * its stream.  soar_trace_end() waits for those events and writes, per kernel name, the
+ * number of launches and the summed device time in milliseconds into out[0..capacity)
+ * (host); *count receives the number of distinct kernels seen.  Process-wide, not re-entrant. */
+typedef struct soar_trace_entry {
+  char kernel[32];
+  int64_t launches;
+  double total_ms;
+} soar_trace_entry;
+int soar_trace_begin(void);
+int soar_trace_end(soar_trace_entry* out, int capacity, int* count);
 
 /* Text for a host-side return value. */
 const char* soar_status_string(int status);

@@ -24,7 +24,8 @@ MAX_ITERS = 64
 
 EXPORTS = (
     "soar_default_cfg", "soar_workspace_bytes", "soar_swizzled_scale_bytes", "soar_quantize",
-    "soar_dequant_error", "soar_quantize_launches", "soar_status_string",
+    "soar_dequant_error", "soar_quantize_launches", "soar_status_string", "soar_quantize_host",
+    "soar_trace_begin", "soar_trace_end",
 )
 
 
@@ -47,6 +48,22 @@ class SoarResult(C.Structure):
         ("zero_blocks", C.c_int64), ("wide_candidates", C.c_int64),
         ("trace_alpha", C.c_double * (MAX_ITERS + 1)), ("trace_sse", C.c_double * (MAX_ITERS + 1)),
     ]
+
+
+class SoarStaging(C.Structure):
+    """Mirror of ``soar_staging``."""
+
+    _fields_ = [
+        ("W", C.c_void_p), ("packed", C.c_void_p), ("scales", C.c_void_p), ("scales_sw", C.c_void_p),
+        ("alpha", C.c_void_p), ("result", C.c_void_p), ("workspace", C.c_void_p),
+        ("workspace_bytes", C.c_size_t),
+    ]
+
+
+class SoarTraceEntry(C.Structure):
+    """Mirror of ``soar_trace_entry``."""
+
+    _fields_ = [("kernel", C.c_char * 32), ("launches", C.c_int64), ("total_ms", C.c_double)]
 
 
 class SoarError(RuntimeError):
@@ -77,6 +94,13 @@ def lib() -> C.CDLL:
         L.soar_dequant_error.argtypes = [vp, i64, i64, i64, vp, vp, C.c_int, vp, vp, vp, vp]
         L.soar_quantize_launches.restype = C.c_int
         L.soar_quantize_launches.argtypes = [C.POINTER(SoarCfg)]
+        L.soar_quantize_host.restype = C.c_int
+        L.soar_quantize_host.argtypes = [vp, i64, i64, i64, C.POINTER(SoarCfg), vp, vp, vp, vp, vp,
+                                         C.POINTER(SoarStaging), vp]
+        L.soar_trace_begin.restype = C.c_int
+        L.soar_trace_begin.argtypes = []
+        L.soar_trace_end.restype = C.c_int
+        L.soar_trace_end.argtypes = [C.POINTER(SoarTraceEntry), C.c_int, C.POINTER(C.c_int)]
         L.soar_status_string.restype = C.c_char_p
         L.soar_status_string.argtypes = [C.c_int]
         _lib = L
@@ -190,3 +214,61 @@ def soar_dequant_error(W: torch.Tensor, packed: torch.Tensor, scales: torch.Tens
         C.c_void_p(out.data_ptr()), C.c_void_p(out.data_ptr() + 8), _stream_ptr(stream))
     _check(rc, "soar_dequant_error")
     return out
+
+
+@dataclass
+class HostBuffers:
+    """Page-locked host buffers for one matrix, inputs and outputs of soar_quantize_host."""
+
+    W: torch.Tensor                  # bf16 [rows, cols], pinned
+    packed: torch.Tensor             # uint8 [rows, cols/2], pinned
+    scales: torch.Tensor | None
+    scales_sw: torch.Tensor | None
+    alpha: torch.Tensor              # float32 [1], pinned
+    result: torch.Tensor             # uint8 [sizeof(soar_result)], pinned
+
+    def read_result(self) -> SoarResult:
+        return SoarResult.from_buffer_copy(self.result.numpy().tobytes())
+
+
+def alloc_host_buffers(rows: int, cols: int, cfg: SoarCfg) -> HostBuffers:
+    pin = dict(pin_memory=True)
+    lin = torch.empty((rows, cols // 16), dtype=torch.uint8, **pin) if cfg.scale_layout & SCALES_LINEAR else None
+    sw = (torch.empty(soar_swizzled_scale_bytes(rows, cols), dtype=torch.uint8, **pin)
+          if cfg.scale_layout & SCALES_SWIZZLED else None)
+    return HostBuffers(
+        W=torch.empty((rows, cols), dtype=torch.bfloat16, **pin),
+        packed=torch.empty((rows, cols // 2), dtype=torch.uint8, **pin), scales=lin, scales_sw=sw,
+        alpha=torch.empty(1, dtype=torch.float32, **pin),
+        result=torch.empty(C.sizeof(SoarResult), dtype=torch.uint8, **pin))
+
+
+def soar_quantize_host(host: HostBuffers, cfg: SoarCfg, dev_W: torch.Tensor, dev: QuantBuffers,
+                       stream=None) -> None:
+    """Enqueue ``soar_quantize_host``: H2D copy of ``host.W``, the quantizer, D2H copies of
+    every output, in order on ``stream``.  ``dev_W``/``dev`` are the device staging buffers."""
+    _require_cuda(dev_W, dev.packed, dev.scales, dev.scales_sw, dev.alpha, dev.result, dev.workspace)
+    rows, cols = host.W.shape
+    if tuple(dev_W.shape) != (rows, cols) or dev_W.dtype != torch.bfloat16 or not dev_W.is_contiguous():
+        raise SoarError("dev_W must be a contiguous bf16 tensor of the host matrix's shape")
+    st = SoarStaging(dev_W.data_ptr(), dev.packed.data_ptr(),
+                     dev.scales.data_ptr() if dev.scales is not None else None,
+                     dev.scales_sw.data_ptr() if dev.scales_sw is not None else None,
+                     dev.alpha.data_ptr(), dev.result.data_ptr(), dev.workspace.data_ptr(),
+                     dev.workspace.numel())
+    rc = lib().soar_quantize_host(
+        _ptr(host.W), rows, cols, cols, C.byref(cfg), _ptr(host.packed), _ptr(host.scales),
+        _ptr(host.scales_sw), _ptr(host.alpha), _ptr(host.result), C.byref(st), _stream_ptr(stream))
+    _check(rc, "soar_quantize_host")
+
+
+def soar_trace_begin() -> None:
+    _check(lib().soar_trace_begin(), "soar_trace_begin")
+
+
+def soar_trace_end() -> dict:
+    """Stops tracing; returns {kernel name: (launches, total device ms)}."""
+    buf = (SoarTraceEntry * 16)()
+    n = C.c_int(0)
+    _check(lib().soar_trace_end(buf, 16, C.byref(n)), "soar_trace_end")
+    return {buf[i].kernel.decode(): (int(buf[i].launches), float(buf[i].total_ms)) for i in range(min(n.value, 16))}

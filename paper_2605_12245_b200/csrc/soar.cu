@@ -22,6 +22,9 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <mutex>
+#include <vector>
+
 #include "soar.h"
 
 namespace {
@@ -523,6 +526,42 @@ __global__ void __launch_bounds__(kThreads) dequant_error_kernel(Params p, const
 
 // ------------------------------------------------------------------ host side
 
+// Optional launch tracing for benchmarks: while enabled, every kernel this library launches
+// is bracketed by two CUDA events on the launching stream.
+enum KernelId { K_AMAX = 0, K_INIT, K_ITERATE, K_FINALIZE, K_SWIZZLE, K_DEQUANT_ERROR, K_COUNT };
+const char* const kKernelNames[K_COUNT] = {"amax_kernel",     "init_kernel",    "iterate_kernel",
+                                           "finalize_kernel", "swizzle_kernel", "dequant_error_kernel"};
+struct TraceRec {
+  int id;
+  cudaEvent_t e0, e1;
+};
+struct Tracer {
+  std::mutex mu;
+  bool on = false;
+  std::vector<TraceRec> recs;
+};
+Tracer g_trace;
+
+struct ScopedLaunch {
+  bool active = false;
+  TraceRec rec;
+  cudaStream_t st;
+  ScopedLaunch(int id, cudaStream_t stream) : st(stream) {
+    if (!g_trace.on) return;
+    rec.id = id;
+    if (cudaEventCreate(&rec.e0) != cudaSuccess) return;
+    if (cudaEventCreate(&rec.e1) != cudaSuccess) { cudaEventDestroy(rec.e0); return; }
+    cudaEventRecord(rec.e0, st);
+    active = true;
+  }
+  ~ScopedLaunch() {
+    if (!active) return;
+    cudaEventRecord(rec.e1, st);
+    std::lock_guard<std::mutex> lk(g_trace.mu);
+    g_trace.recs.push_back(rec);
+  }
+};
+
 int g_sm_count[64];
 
 int sm_count() {
@@ -656,17 +695,30 @@ int soar_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, co
   p.beta_step_pct = cfg->beta_step_pct;
 
   if (cudaMemsetAsync(workspace, 0, kWsFixedBytes, st) != cudaSuccess) return SOAR_ERR_CUDA;
-  amax_kernel<<<persistent_grid(amax_kernel, p.nblk, kThreads), kThreads, 0, st>>>(p);
-  init_kernel<<<persistent_grid(init_kernel, p.nblk, kThreads), kThreads, 0, st>>>(p);
+  {
+    ScopedLaunch sl(K_AMAX, st);
+    amax_kernel<<<persistent_grid(amax_kernel, p.nblk, kThreads), kThreads, 0, st>>>(p);
+  }
+  {
+    ScopedLaunch sl(K_INIT, st);
+    init_kernel<<<persistent_grid(init_kernel, p.nblk, kThreads), kThreads, 0, st>>>(p);
+  }
   const unsigned int g_it = persistent_grid(iterate_kernel, p.nblk, kThreads);
-  for (int t = 0; t < cfg->max_iters; ++t) iterate_kernel<<<g_it, kThreads, 0, st>>>(p, t);
-  finalize_kernel<<<1, 32, 0, st>>>(p, out_global_fp32, out_result);
+  for (int t = 0; t < cfg->max_iters; ++t) {
+    ScopedLaunch sl(K_ITERATE, st);
+    iterate_kernel<<<g_it, kThreads, 0, st>>>(p, t);
+  }
+  {
+    ScopedLaunch sl(K_FINALIZE, st);
+    finalize_kernel<<<1, 32, 0, st>>>(p, out_global_fp32, out_result);
+  }
   if (want_sw) {
     const unsigned int rt = static_cast<unsigned int>((rows + 127) / 128);
     const unsigned int ct = (p.nbc + 3) / 4;
     const size_t total = static_cast<size_t>(rt) * ct * 512;
     const size_t blocks = (total + 255) / 256;
     const unsigned int grid = static_cast<unsigned int>(blocks < 65535u * 16u ? blocks : 65535u * 16u);
+    ScopedLaunch sl(K_SWIZZLE, st);
     swizzle_kernel<<<grid, 256, 0, st>>>(p.scales, static_cast<uint8_t*>(out_e4m3_scales_sw),
                                          static_cast<unsigned int>(rows), p.nbc, rt, ct);
   }
@@ -693,10 +745,86 @@ int soar_dequant_error(const void* W_bf16, int64_t rows, int64_t cols, int64_t l
   p.nblk = static_cast<unsigned int>(rows * (cols / 16));
   if (cudaMemsetAsync(out_sse, 0, sizeof(double), st) != cudaSuccess) return SOAR_ERR_CUDA;
   if (cudaMemsetAsync(out_sumsq, 0, sizeof(double), st) != cudaSuccess) return SOAR_ERR_CUDA;
-  dequant_error_kernel<<<persistent_grid(dequant_error_kernel, p.nblk, kThreads), kThreads, 0, st>>>(
-      p, static_cast<const uint8_t*>(e4m3_scales), scale_layout == SOAR_SCALES_SWIZZLED ? 1 : 0,
-      (p.nbc + 3) / 4, global_fp32, out_sse, out_sumsq);
+  {
+    ScopedLaunch sl(K_DEQUANT_ERROR, st);
+    dequant_error_kernel<<<persistent_grid(dequant_error_kernel, p.nblk, kThreads), kThreads, 0, st>>>(
+        p, static_cast<const uint8_t*>(e4m3_scales), scale_layout == SOAR_SCALES_SWIZZLED ? 1 : 0,
+        (p.nbc + 3) / 4, global_fp32, out_sse, out_sumsq);
+  }
   return cudaGetLastError() == cudaSuccess ? SOAR_OK : SOAR_ERR_CUDA;
+}
+
+int soar_quantize_host(const void* W_host, int64_t rows, int64_t cols, int64_t ld, const soar_cfg* cfg,
+                       void* out_fp4_packed_host, void* out_e4m3_scales_host, void* out_e4m3_scales_sw_host,
+                       float* out_global_host, soar_result* out_result_host, const soar_staging* dev,
+                       void* stream) {
+  if (dev == nullptr || W_host == nullptr || dev->W == nullptr) return SOAR_ERR_INVALID_ARG;
+  int rc = check_cfg(cfg);
+  if (rc != SOAR_OK) return rc;
+  if (rows <= 0 || cols <= 0 || ld < cols) return SOAR_ERR_INVALID_ARG;
+  if (out_fp4_packed_host == nullptr || out_global_host == nullptr) return SOAR_ERR_INVALID_ARG;
+  const bool want_lin = (cfg->scale_layout & SOAR_SCALES_LINEAR) != 0;
+  const bool want_sw = (cfg->scale_layout & SOAR_SCALES_SWIZZLED) != 0;
+  if (want_lin && (out_e4m3_scales_host == nullptr || dev->scales == nullptr)) return SOAR_ERR_INVALID_ARG;
+  if (want_sw && (out_e4m3_scales_sw_host == nullptr || dev->scales_sw == nullptr)) return SOAR_ERR_INVALID_ARG;
+  if (dev->packed == nullptr || dev->alpha == nullptr) return SOAR_ERR_INVALID_ARG;
+  if (out_result_host != nullptr && dev->result == nullptr) return SOAR_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t in_bytes = static_cast<size_t>(rows) * static_cast<size_t>(ld) * 2;
+  if (cudaMemcpyAsync(dev->W, W_host, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SOAR_ERR_CUDA;
+  rc = soar_quantize(dev->W, rows, cols, ld, cfg, dev->packed, dev->scales, dev->scales_sw, dev->alpha,
+                     dev->workspace, dev->workspace_bytes, out_result_host ? dev->result : nullptr, stream);
+  if (rc != SOAR_OK) return rc;
+  const size_t n = static_cast<size_t>(rows) * static_cast<size_t>(cols);
+  bool ok = cudaMemcpyAsync(out_fp4_packed_host, dev->packed, n / 2, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (want_lin)
+    ok = ok && cudaMemcpyAsync(out_e4m3_scales_host, dev->scales, n / 16, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (want_sw)
+    ok = ok && cudaMemcpyAsync(out_e4m3_scales_sw_host, dev->scales_sw, soar_swizzled_scale_bytes(rows, cols),
+                               cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(out_global_host, dev->alpha, sizeof(float), cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (out_result_host != nullptr)
+    ok = ok && cudaMemcpyAsync(out_result_host, dev->result, sizeof(soar_result), cudaMemcpyDeviceToHost, st) ==
+                   cudaSuccess;
+  return ok ? SOAR_OK : SOAR_ERR_CUDA;
+}
+
+int soar_trace_begin(void) {
+  std::lock_guard<std::mutex> lk(g_trace.mu);
+  for (TraceRec& r : g_trace.recs) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
+  g_trace.recs.clear();
+  g_trace.on = true;
+  return SOAR_OK;
+}
+
+int soar_trace_end(soar_trace_entry* out, int capacity, int* count) {
+  std::lock_guard<std::mutex> lk(g_trace.mu);
+  g_trace.on = false;
+  double total[K_COUNT] = {0};
+  int64_t launches[K_COUNT] = {0};
+  bool ok = true;
+  for (TraceRec& r : g_trace.recs) {
+    float ms = 0.0f;
+    if (cudaEventSynchronize(r.e1) != cudaSuccess || cudaEventElapsedTime(&ms, r.e0, r.e1) != cudaSuccess) ok = false;
+    total[r.id] += ms;
+    launches[r.id] += 1;
+    cudaEventDestroy(r.e0);
+    cudaEventDestroy(r.e1);
+  }
+  g_trace.recs.clear();
+  int n = 0;
+  for (int k = 0; k < K_COUNT; ++k) {
+    if (launches[k] == 0) continue;
+    if (out != nullptr && n < capacity) {
+      memset(&out[n], 0, sizeof(out[n]));
+      strncpy(out[n].kernel, kKernelNames[k], sizeof(out[n].kernel) - 1);
+      out[n].launches = launches[k];
+      out[n].total_ms = total[k];
+    }
+    ++n;
+  }
+  if (count != nullptr) *count = n;
+  return ok ? SOAR_OK : SOAR_ERR_CUDA;
 }
 
 const char* soar_status_string(int status) {
