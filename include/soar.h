@@ -33,6 +33,7 @@ extern "C" {
 #define SOAR_ERR_UNSUPPORTED (-2)      /* cols % 16, ld < cols, alignment, block != 16, ... */
 #define SOAR_ERR_WORKSPACE (-3)        /* workspace missing or too small                    */
 #define SOAR_ERR_CUDA (-4)             /* a CUDA runtime call or kernel launch failed       */
+#define SOAR_ERR_TOO_LARGE (-5)        /* matrix exceeds the built-in scratch of soar_quantize_static */
 
 /* soar_result.status bits (device side, data dependent) */
 #define SOAR_STATUS_ZERO_TENSOR 1      /* every element is zero: alpha = 1, scales = 0      */
@@ -161,6 +162,34 @@ int soar_dequant_error(const void* W_bf16, int64_t rows, int64_t cols, int64_t l
                        const void* fp4_packed, const void* e4m3_scales, int scale_layout,
                        const float* global_fp32, double* out_sse, double* out_sumsq,
                        void* stream);
+
+/*
+ * soar_quantize without a workspace argument, for callers that must not allocate device
+ * memory and have none to spare: code running inside another framework's memory pool, a
+ * plugin or callback that is handed only its input and output buffers, a process whose
+ * device memory is fully pre-assigned.  (The paper has no counterpart; this is a convenience
+ * of the library.)  The scratch soar_quantize would take from `workspace` lives in a fixed
+ * array inside the library image instead, so every GPU that loads the library holds
+ * SOAR_STATIC_SCRATCH_BYTES of device memory until the process exits.  The call itself
+ * makes no cudaMalloc/cudaFree and calls no allocating routine.
+ *
+ *   - Limit: rows*cols <= SOAR_STATIC_MAX_ELEMENTS, else SOAR_ERR_TOO_LARGE is returned and
+ *     nothing is enqueued.  All other arguments, outputs and return codes are those of
+ *     soar_quantize.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current) before it enqueues anything; make that first call outside any stream capture.
+ *   - There is one array per device, shared by every call and every stream.  The call
+ *     clears the part that must start at zero, so leftovers of earlier calls do no harm,
+ *     but two calls that overlap on the GPU (different streams, no ordering) race on it
+ *     and give unspecified results: order them, or use soar_quantize with separate
+ *     workspaces.
+ */
+#define SOAR_STATIC_MAX_ELEMENTS (1ll << 24)                 /* e.g. one 4096 x 4096 matrix */
+#define SOAR_STATIC_SCRATCH_BYTES (2048 + (1 << 20))
+int soar_quantize_static(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld,
+                         const soar_cfg* cfg, void* out_fp4_packed, void* out_e4m3_scales,
+                         void* out_e4m3_scales_sw, float* out_global_fp32,
+                         soar_result* out_result, void* stream);
 
 /* Number of kernels soar_quantize enqueues for this cfg (host-side bookkeeping for callers
  * that count launches); 0 on bad arguments. */

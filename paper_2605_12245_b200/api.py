@@ -25,7 +25,7 @@ MAX_ITERS = 64
 EXPORTS = (
     "soar_default_cfg", "soar_workspace_bytes", "soar_swizzled_scale_bytes", "soar_quantize",
     "soar_dequant_error", "soar_quantize_launches", "soar_status_string", "soar_quantize_host",
-    "soar_trace_begin", "soar_trace_end",
+    "soar_trace_begin", "soar_trace_end", "soar_quantize_static",
 )
 
 
@@ -97,6 +97,8 @@ def lib() -> C.CDLL:
         L.soar_quantize_host.restype = C.c_int
         L.soar_quantize_host.argtypes = [vp, i64, i64, i64, C.POINTER(SoarCfg), vp, vp, vp, vp, vp,
                                          C.POINTER(SoarStaging), vp]
+        L.soar_quantize_static.restype = C.c_int
+        L.soar_quantize_static.argtypes = [vp, i64, i64, i64, C.POINTER(SoarCfg), vp, vp, vp, vp, vp, vp]
         L.soar_trace_begin.restype = C.c_int
         L.soar_trace_begin.argtypes = []
         L.soar_trace_end.restype = C.c_int
@@ -198,6 +200,24 @@ def soar_quantize(W: torch.Tensor, cfg: SoarCfg, out: QuantBuffers | None = None
         _ptr(out.scales_sw), _ptr(out.alpha), _ptr(out.workspace), out.workspace.numel(),
         _ptr(out.result), _stream_ptr(stream))
     _check(rc, "soar_quantize")
+    return out
+
+
+STATIC_MAX_ELEMENTS = 1 << 24
+
+
+def soar_quantize_static(W: torch.Tensor, cfg: SoarCfg, out: QuantBuffers, stream=None) -> QuantBuffers:
+    """Enqueue ``soar_quantize_static``: the quantizer for callers that cannot allocate device
+    memory.  ``out`` supplies the output tensors only; its ``workspace`` is not passed on (the
+    library uses its built-in scratch), and matrices above ``STATIC_MAX_ELEMENTS`` are refused."""
+    _require_cuda(W, out.packed, out.scales, out.scales_sw, out.alpha, out.result)
+    if W.dtype != torch.bfloat16 or W.dim() != 2 or W.stride(1) != 1:
+        raise SoarError("W must be a 2-D bf16 tensor with unit column stride")
+    rows, cols = W.shape
+    rc = lib().soar_quantize_static(
+        _ptr(W), rows, cols, W.stride(0), C.byref(cfg), _ptr(out.packed), _ptr(out.scales),
+        _ptr(out.scales_sw), _ptr(out.alpha), _ptr(out.result), _stream_ptr(stream))
+    _check(rc, "soar_quantize_static")
     return out
 
 

@@ -725,6 +725,44 @@ int soar_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, co
   return cudaGetLastError() == cudaSuccess ? SOAR_OK : SOAR_ERR_CUDA;
 }
 
+// Built-in scratch of soar_quantize_static.  In host code the symbol below is only a handle:
+// the device address comes from cudaGetSymbolAddress, looked up once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[SOAR_STATIC_SCRATCH_BYTES];
+
+namespace {
+std::mutex g_static_mu;
+void* g_static_ptr[64];
+
+// Device address of g_static_scratch on the current device (nullptr on failure).
+void* static_scratch_ptr() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lk(g_static_mu);
+  if (g_static_ptr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) return nullptr;
+    g_static_ptr[dev] = ptr;
+  }
+  return g_static_ptr[dev];
+}
+}  // namespace
+
+int soar_quantize_static(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, const soar_cfg* cfg,
+                         void* out_fp4_packed, void* out_e4m3_scales, void* out_e4m3_scales_sw,
+                         float* out_global_fp32, soar_result* out_result, void* stream) {
+  int rc = check_cfg(cfg);
+  if (rc != SOAR_OK) return rc;
+  rc = check_shape(W_bf16, rows, cols, ld);
+  if (rc != SOAR_OK) return rc;
+  if (rows * cols > SOAR_STATIC_MAX_ELEMENTS) return SOAR_ERR_TOO_LARGE;
+  if (soar_workspace_bytes(rows, cols, cfg) > static_cast<size_t>(SOAR_STATIC_SCRATCH_BYTES))
+    return SOAR_ERR_TOO_LARGE;
+  void* scratch = static_scratch_ptr();
+  if (scratch == nullptr) return SOAR_ERR_CUDA;
+  return soar_quantize(W_bf16, rows, cols, ld, cfg, out_fp4_packed, out_e4m3_scales, out_e4m3_scales_sw,
+                       out_global_fp32, scratch, SOAR_STATIC_SCRATCH_BYTES, out_result, stream);
+}
+
 int soar_dequant_error(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, const void* fp4_packed,
                        const void* e4m3_scales, int scale_layout, const float* global_fp32,
                        double* out_sse, double* out_sumsq, void* stream) {
@@ -834,6 +872,7 @@ const char* soar_status_string(int status) {
     case SOAR_ERR_UNSUPPORTED: return "unsupported shape, alignment or block size";
     case SOAR_ERR_WORKSPACE: return "workspace missing or too small";
     case SOAR_ERR_CUDA: return "CUDA runtime or launch error";
+    case SOAR_ERR_TOO_LARGE: return "matrix exceeds the built-in scratch of soar_quantize_static";
     default: return "unknown status";
   }
 }
