@@ -39,6 +39,7 @@ extern "C" {
 #define SOAR_STATUS_ZERO_TENSOR 1      /* every element is zero: alpha = 1, scales = 0      */
 #define SOAR_STATUS_NONFINITE 2        /* NaN or Inf in the input: outputs unspecified      */
 #define SOAR_STATUS_RANGE 4            /* max |W| outside [2^-100, 2^100]: outputs unspecified */
+#define SOAR_STATUS_INTERNAL 8         /* a bounded wait inside a kernel gave up: outputs unspecified */
 
 /* scale_layout bits */
 #define SOAR_SCALES_LINEAR 1           /* row-major [rows][cols/16] bytes                   */
@@ -91,8 +92,9 @@ typedef struct soar_result {
 int soar_default_cfg(soar_cfg* cfg, int preset);
 
 /* Bytes of device scratch soar_quantize needs for this shape and cfg (0 on bad arguments).
- * It is a small fixed part for the tensor-wide sums of Eq. 5 plus, when cfg->scale_layout
- * lacks SOAR_SCALES_LINEAR, rows*cols/16 bytes for the row-major scales the loop works on. */
+ * It is a small fixed part for the tensor-wide sums of Eq. 5; 8 bytes per block of state
+ * carried between iterations when cfg->max_iters > 0; and, when cfg->scale_layout lacks
+ * SOAR_SCALES_LINEAR, rows*cols/16 bytes for the row-major scales the loop works on. */
 size_t soar_workspace_bytes(int64_t rows, int64_t cols, const soar_cfg* cfg);
 
 /* Bytes of the swizzled scale buffer: scales padded to multiples of 128 rows and 4 columns. */
@@ -185,7 +187,7 @@ int soar_dequant_error(const void* W_bf16, int64_t rows, int64_t cols, int64_t l
  *     workspaces.
  */
 #define SOAR_STATIC_MAX_ELEMENTS (1ll << 24)                 /* e.g. one 4096 x 4096 matrix */
-#define SOAR_STATIC_SCRATCH_BYTES (2048 + (1 << 20))
+#define SOAR_STATIC_SCRATCH_BYTES (2048 + 9 * (1 << 20))    /* 8 B of state + 1 scale byte per block */
 int soar_quantize_static(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld,
                          const soar_cfg* cfg, void* out_fp4_packed, void* out_e4m3_scales,
                          void* out_e4m3_scales_sw, float* out_global_fp32,

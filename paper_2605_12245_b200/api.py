@@ -17,7 +17,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libsoar.so")
 
 SOAR_OK = 0
-STATUS_ZERO_TENSOR, STATUS_NONFINITE, STATUS_RANGE = 1, 2, 4
+STATUS_ZERO_TENSOR, STATUS_NONFINITE, STATUS_RANGE, STATUS_INTERNAL = 1, 2, 4, 8
 SCALES_LINEAR, SCALES_SWIZZLED = 1, 2
 PRESET_PAPER, PRESET_SINGLE_PASS, PRESET_RTN = 0, 1, 2
 MAX_ITERS = 64

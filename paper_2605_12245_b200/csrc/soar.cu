@@ -1,23 +1,31 @@
 // SOAR NVFP4 weight quantizer for NVIDIA B200 (sm_100a): kernels and the C ABI of soar.h.
 //
 // What runs on the device, in launch order (Algorithm 1 of the SOAR paper):
-//   amax_kernel      tensor-wide max |W| and a non-finite check            (Eq. 1)
-//   init_kernel      max-based scales, first codes, first tensor sums      (Eq. 1-2, Alg. 1 "Initialization")
+//   amax_kernel      tensor-wide max |W|, sum W^2 and a non-finite check        (Eq. 1)
+//   init_kernel      max-based scales, first codes, first tensor sums          (Eq. 1-2, Alg. 1 "Initialization")
 //   iterate_kernel   T times: global scale (Eq. 5) from the previous kernel's sums, block
 //                    scale (Eq. 6), candidate search (Eq. 8, App. B.3), winners stored,
 //                    next sums accumulated
 //   finalize_kernel  early-stop bookkeeping (Sec. 4.1), alpha and the report
 //   swizzle_kernel   optional 128x4-tiled copy of the block scales
 //
-// State between iterations is the output itself: the packed E2M1 codes and the E4M3 scale
-// bytes.  The codes that iteration t+1 starts from are the codes of iteration t's winning
-// candidate (same alpha, same quantization scale), so the high-precision quantization
-// scale of Sec. 3.3 never has to be stored.
+// Data movement.  The three passes over W are persistent kernels: each CTA walks tiles of
+// 256 blocks (8 KB of bf16) that one thread fetches with bulk asynchronous copies
+// (cp.async.bulk, completion on an mbarrier) into a four-stage shared-memory ring, so the
+// copies of the next tiles are in flight while the 256 threads work on the current one
+// from registers.  One thread owns one 16-element block.
+//
+// State between iterations is 8 bytes per block in the workspace: the winner's
+// A = sum |W| m (binary32, exact), 4B = sum (2m)^2 and its E4M3 scale code.  That is all
+// Eq. 6 needs; the transient quantization scale of Sec. 3.3 is never stored.
 //
 // Arithmetic.  Whatever feeds a rounding decision is a fixed chain of IEEE binary32
-// round-to-nearest operations (explicit __f*_rn intrinsics, never contracted); tensor sums
-// and candidate comparisons are binary64.  Per-candidate block sums A = sum |W| m and
-// B = sum m^2 are accumulated in binary32 only where that is exact (see eval_candidate).
+// round-to-nearest operations (explicit __f*_rn intrinsics, never contracted); the E2M1
+// rounding itself is the sm_100a conversion cvt.rn.satfinite.e2m1x2.f32 (nearest, ties to
+// even, saturating, sign kept on zero).  Block sums A and B are integer dot products over
+// 16-bit fixed-point magnitudes and the codes' byte values (dp2a / dp4a), exact whenever
+// the block maximum times the reciprocal scale is at most 32; otherwise a binary64 path is
+// taken.  Tensor sums and candidate comparisons are binary64.
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <string.h>
@@ -29,29 +37,35 @@
 
 namespace {
 
-constexpr int kThreads = 128;
+constexpr int kThreads = 256;                  // threads per CTA = blocks per tile
+constexpr int kStages = 4;                     // depth of the shared-memory ring
+constexpr int kTileBytes = kThreads * 32;      // 16 bf16 per block
 constexpr size_t kWsFixedBytes = 2048;
+constexpr unsigned int kWaitLimit = 1u << 22;  // mbarrier polls before a wait gives up
 
 struct Ws {
   unsigned int amax_bits;            // max over the tensor of the bf16 magnitude bit pattern
-  unsigned int pad0;
+  unsigned int error;                // non-zero when a bounded wait gave up
   unsigned long long zero_blocks;
   unsigned long long wide;
-  double sumsq;
-  double num[SOAR_MAX_ITERS + 1];    // stage s: sum A_i * dd_i      (numerator of Eq. 5)
-  double den[SOAR_MAX_ITERS + 1];    // stage s: sum B_i * dd_i^2    (denominator of Eq. 5)
-  double sse[SOAR_MAX_ITERS + 1];    // stage s: sum of block errors (Eq. 4)
+  double sumsq;                      // sum W^2
+  double num[SOAR_MAX_ITERS + 1];    // stage s: sum A_i * dd_i        (numerator of Eq. 5)
+  double den[SOAR_MAX_ITERS + 1];    // stage s: sum B_i * dd_i^2      (denominator of Eq. 5)
+  double gsum[SOAR_MAX_ITERS + 1];   // stage s: sum of block errors minus sum W^2 (Eq. 4)
 };
 static_assert(sizeof(Ws) <= kWsFixedBytes, "workspace header too large");
 
 struct Params {
   const uint16_t* W;
   uint8_t* packed;
-  uint8_t* scales;     // row-major state, either the caller's buffer or workspace
+  uint8_t* scales;     // row-major scale bytes, either the caller's buffer or workspace
+  uint2* state;        // per block {A as binary32 bits, 4B | scale code << 16}; null when T == 0
   Ws* ws;
   long long ld;
   unsigned int nblk;   // rows * cols/16
   unsigned int nbc;    // cols/16
+  unsigned int ntiles;
+  int contiguous;      // ld == cols: a tile is one contiguous run of bytes
   int max_iters;
   float early_stop_rel;
   int n_dq;
@@ -79,19 +93,11 @@ __device__ __forceinline__ int e4m3_encode(float v) {
   return r & 0xFF;
 }
 
-// Eq. 2 on a magnitude x >= 0: nearest point of {0,.5,1,1.5,2,3,4,6}, ties to the even code,
-// saturating at 6.  Adding 2^(e+22), e = exponent of max(min(x,6),1), makes the binary32
-// adder round to the grid step of that binade (1/2 below 2, 1 below 4, 2 above).
-__device__ __forceinline__ float e2m1_round(float x) {
-  float xc = fminf(x, 6.0f);
-  float t = fmaxf(xc, 1.0f);
-  float M = __uint_as_float((__float_as_uint(t) & 0x7F800000u) + 0x0B000000u);
-  return __fsub_rn(__fadd_rn(xc, M), M);
-}
-
-// Eight grid magnitudes -> eight 4-bit codes (element 0 in the low nibble) with the sm_100a
-// E2M1 conversion; the inputs are grid points, so the conversion is exact.
-__device__ __forceinline__ unsigned int pack_e2m1x8(const float* m) {
+// Eq. 2 for eight signed values at once: nearest point of {0,.5,1,1.5,2,3,4,6} with the
+// input's sign, ties to the even code, saturating at 6.  Returns eight 4-bit codes
+// (sign << 3 | magnitude code), element 0 in the low nibble.
+__device__ __forceinline__ unsigned int e2m1x8(float x0, float x1, float x2, float x3, float x4, float x5,
+                                               float x6, float x7) {
   unsigned int out;
   asm("{\n"
       ".reg .b8 b0, b1, b2, b3;\n"
@@ -102,7 +108,15 @@ __device__ __forceinline__ unsigned int pack_e2m1x8(const float* m) {
       "mov.b32 %0, {b0, b1, b2, b3};\n"
       "}"
       : "=r"(out)
-      : "f"(m[0]), "f"(m[1]), "f"(m[2]), "f"(m[3]), "f"(m[4]), "f"(m[5]), "f"(m[6]), "f"(m[7]));
+      : "f"(x0), "f"(x1), "f"(x2), "f"(x3), "f"(x4), "f"(x5), "f"(x6), "f"(x7));
+  return out;
+}
+
+// Four magnitude codes (the low four nibbles of `codes`, sign bits already cleared) to four
+// bytes holding 2m: a byte permute over the table 0,1,2,3,4,6,8,12.
+__device__ __forceinline__ unsigned int twice_magnitude_x4(unsigned int codes) {
+  unsigned int out;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(0x03020100u), "r"(0x0C080604u), "r"(codes));
   return out;
 }
 
@@ -112,61 +126,234 @@ __device__ __forceinline__ float e2m1_code_value(unsigned int code3) {
   return 0.5f * static_cast<float>(static_cast<unsigned int>(lut >> (8 * code3)) & 0xFFu);
 }
 
+// Non-negative integer below 2^31 to binary64 without a conversion instruction.
+__device__ __forceinline__ double uint_to_double(unsigned int v) {
+  return __hiloint2double(0x43300000, static_cast<int>(v)) - 4503599627370496.0;
+}
+
+// ------------------------------------------------------------------ shared-memory tile ring
+
+__device__ __forceinline__ unsigned int smem_u32(const void* p) {
+  return static_cast<unsigned int>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned int bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+
+// One bulk copy global -> shared; src and dst 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned int bytes,
+                                          unsigned long long* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
+// Waits for the phase with the given parity; gives up after kWaitLimit polls.
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned int parity) {
+  const unsigned int addr = smem_u32(bar);
+  for (unsigned int i = 0; i < kWaitLimit; ++i) {
+    unsigned int ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(addr), "r"(parity)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+
+struct __align__(128) Ring {
+  unsigned char tile[kStages][kTileBytes];
+  unsigned long long full[kStages];
+  int fail;
+};
+
+// Thread 0: start the copies of tile `tile` into stage `s` (one copy when rows are
+// contiguous, else one per row segment) and arm the stage's barrier with the byte count.
+__device__ __forceinline__ void ring_issue(Ring& ring, const Params& p, unsigned int tile, int s) {
+  const unsigned int b0 = tile * kThreads;
+  unsigned int nb = min(static_cast<unsigned int>(kThreads), p.nblk - b0);
+  mbar_expect_tx(&ring.full[s], nb * 32u);
+  unsigned char* dst = ring.tile[s];
+  if (p.contiguous) {
+    bulk_load(dst, p.W + static_cast<size_t>(b0) * 16, nb * 32u, &ring.full[s]);
+    return;
+  }
+  unsigned int row = b0 / p.nbc, cb = b0 - row * p.nbc;
+  while (nb > 0) {
+    const unsigned int seg = min(nb, p.nbc - cb);
+    bulk_load(dst, p.W + static_cast<long long>(row) * p.ld + static_cast<long long>(cb) * 16, seg * 32u,
+              &ring.full[s]);
+    dst += seg * 32u;
+    nb -= seg;
+    ++row;
+    cb = 0;
+  }
+}
+
+// Order in which a CTA visits its tiles: n-th tile of this CTA, forward or from the end.
+// Consecutive passes alternate direction so that a pass starts on what the previous pass
+// left in L2.
+__device__ __forceinline__ unsigned int tile_of(const Params& p, unsigned int n, int reverse) {
+  const unsigned int t = blockIdx.x + n * gridDim.x;
+  return reverse ? p.ntiles - 1 - t : t;
+}
+__device__ __forceinline__ unsigned int tiles_of_cta(const Params& p) {
+  return blockIdx.x < p.ntiles ? (p.ntiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+}
+
+__device__ __forceinline__ void ring_start(Ring& ring, const Params& p, int reverse) {
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) mbar_init(&ring.full[s], 1);
+    ring.fail = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned int n = tiles_of_cta(p);
+    for (unsigned int i = 0; i < static_cast<unsigned int>(kStages) && i < n; ++i)
+      ring_issue(ring, p, tile_of(p, i, reverse), static_cast<int>(i));
+  }
+}
+
+// Fetches this thread's 32 bytes of the CTA's n-th tile into v0, v1; then (thread 0) refills
+// the stage with the tile kStages ahead.  Returns false, for every thread of the CTA alike,
+// when a wait gave up; the caller must then leave its tile loop.
+__device__ __forceinline__ bool ring_next(Ring& ring, const Params& p, unsigned int n, unsigned int ntile_cta,
+                                          int reverse, uint4& v0, uint4& v1) {
+  const int s = static_cast<int>(n % kStages);
+  const bool ok = mbar_wait(&ring.full[s], (n / kStages) & 1u);
+  if (!ok) ring.fail = 1;
+  if (ok) {
+    const uint4* src = reinterpret_cast<const uint4*>(ring.tile[s] + threadIdx.x * 32);
+    v0 = src[0];
+    v1 = src[1];
+  }
+  __syncthreads();
+  if (*static_cast<volatile int*>(&ring.fail)) return false;
+  if (threadIdx.x == 0 && n + kStages < ntile_cta) ring_issue(ring, p, tile_of(p, n + kStages, reverse), s);
+  return true;
+}
+
+// After a failed wait: record it, then give copies still in flight a bounded chance to land
+// before the CTA's shared memory is released.
+__device__ __forceinline__ void ring_abort(Ring& ring, const Params& p, unsigned int n, unsigned int ntile_cta) {
+  if (threadIdx.x != 0) return;
+  atomicOr(&p.ws->error, 1u);
+  for (unsigned int m = n; m < ntile_cta && m < n + kStages; ++m)
+    (void)mbar_wait(&ring.full[m % kStages], (m / kStages) & 1u);
+}
+
 // ------------------------------------------------------------------ block helpers
 
 struct Block {
-  float a[16];          // magnitudes |W_j|
-  unsigned int sign0;   // sign bits already at nibble bit 3 of packed word 0 / 1
-  unsigned int sign1;
-  float bmax;
+  float w[16];   // the block's elements, signed
+  float bmax;    // max |w_j|
 };
 
-__device__ __forceinline__ void load_block(const uint16_t* p, Block& blk) {
-  const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(p));
-  const uint4 v1 = __ldg(reinterpret_cast<const uint4*>(p) + 1);
-  const unsigned int w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-  unsigned int mx = 0, s0 = 0, s1 = 0;
+__device__ __forceinline__ void unpack_block(const uint4& v0, const uint4& v1, Block& blk) {
+  const unsigned int u[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+  float mx = 0.0f;
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    blk.a[2 * i] = __uint_as_float((w[i] << 16) & 0x7FFF0000u);
-    blk.a[2 * i + 1] = __uint_as_float(w[i] & 0x7FFF0000u);
-    mx = __vmaxu2(mx, w[i] & 0x7FFF7FFFu);
-    unsigned int sg = (((w[i] >> 15) & 1u) << 3) | ((w[i] >> 31) << 7);
-    if (i < 4) s0 |= sg << (8 * i);
-    else s1 |= sg << (8 * (i - 4));
+    blk.w[2 * i] = __uint_as_float(u[i] << 16);
+    blk.w[2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
+    mx = fmaxf(mx, fmaxf(fabsf(blk.w[2 * i]), fabsf(blk.w[2 * i + 1])));
   }
-  blk.sign0 = s0;
-  blk.sign1 = s1;
-  blk.bmax = bits_to_mag(max(mx & 0xFFFFu, mx >> 16));
+  blk.bmax = mx;
 }
 
-// One candidate: re-round the block under reciprocal scale r (Eq. 2) and return
-// A = sum |W_j| m_j, B = sum m_j^2.  Binary32 accumulation is exact when bmax*r <= 32:
-// an element with m_j > 0 then lies within 2^7 of the block maximum, every term is a
-// multiple of 2^(Emin-8) and every partial sum stays below 2^24 such units.  Otherwise the
-// caller switches to eval_candidate_wide.
-__device__ __forceinline__ void eval_candidate(const float (&a)[16], float r, float& A, float& B) {
-  float sa = 0.0f, sb = 0.0f;
+// Codes of the block under reciprocal scale r (Eq. 2): x_j = fl(w_j * r), rounded to E2M1.
+__device__ __forceinline__ void round_block(const Block& blk, float r, unsigned int& c0, unsigned int& c1) {
+  const float* w = blk.w;
+  c0 = e2m1x8(__fmul_rn(w[0], r), __fmul_rn(w[1], r), __fmul_rn(w[2], r), __fmul_rn(w[3], r), __fmul_rn(w[4], r),
+              __fmul_rn(w[5], r), __fmul_rn(w[6], r), __fmul_rn(w[7], r));
+  c1 = e2m1x8(__fmul_rn(w[8], r), __fmul_rn(w[9], r), __fmul_rn(w[10], r), __fmul_rn(w[11], r),
+              __fmul_rn(w[12], r), __fmul_rn(w[13], r), __fmul_rn(w[14], r), __fmul_rn(w[15], r));
+}
+
+// 16-bit fixed-point magnitudes of a block: a_j = fix_j * 2^(e - 15) with 2^e <= bmax < 2^(e+1),
+// exact for every element within 2^8 of the block maximum (smaller ones are rounded, and
+// only ever multiplied by a zero code when bmax * r <= 32).  Two values per word.
+struct Fixed {
+  unsigned int pair[8];
+  double unit;   // 2^(e - 16): A = unit * sum fix_j * (2 m_j)
+  bool ok;       // false for block maxima below 2^-110, which take the binary64 path
+};
+
+__device__ __forceinline__ void make_fixed(const Block& blk, Fixed& fx) {
+  const unsigned int eb = __float_as_uint(blk.bmax) >> 23;   // biased exponent of bmax
+  fx.ok = eb >= 17u;
+  const unsigned int ebc = max(eb, 17u);
+  const float S = __uint_as_float((269u - ebc) << 23);       // 2^(15 - e)
+  fx.unit = __hiloint2double(static_cast<int>((ebc + 880u) << 20), 0);
 #pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    float m = e2m1_round(__fmul_rn(a[j], r));
-    sa = __fmaf_rn(a[j], m, sa);
-    sb = __fmaf_rn(m, m, sb);
+  for (int i = 0; i < 8; ++i) {
+    const unsigned int lo = __float_as_uint(__fmaf_rn(fabsf(blk.w[2 * i]), S, 8388608.0f));
+    const unsigned int hi = __float_as_uint(__fmaf_rn(fabsf(blk.w[2 * i + 1]), S, 8388608.0f));
+    fx.pair[i] = (lo & 0xFFFFu) | (hi << 16);
   }
-  A = sa;
-  B = sb;
 }
 
-__device__ __noinline__ void eval_candidate_wide(const float (&a)[16], float r, double& A, float& B) {
+// Integer sums of a code vector: afix = sum fix_j * (2 m_j), b4 = sum (2 m_j)^2.
+__device__ __forceinline__ void code_sums(const Fixed& fx, unsigned int c0, unsigned int c1, unsigned int& afix,
+                                          unsigned int& b4) {
+  const unsigned int m0 = c0 & 0x77777777u, m1 = c1 & 0x77777777u;
+  const unsigned int t0 = twice_magnitude_x4(m0), t1 = twice_magnitude_x4(m0 >> 16);
+  const unsigned int t2 = twice_magnitude_x4(m1), t3 = twice_magnitude_x4(m1 >> 16);
+  unsigned int b = __dp4a(t0, t0, 0u);
+  b = __dp4a(t1, t1, b);
+  b = __dp4a(t2, t2, b);
+  b4 = __dp4a(t3, t3, b);
+  unsigned int a = __dp2a_lo(fx.pair[0], t0, 0u);
+  a = __dp2a_hi(fx.pair[1], t0, a);
+  a = __dp2a_lo(fx.pair[2], t1, a);
+  a = __dp2a_hi(fx.pair[3], t1, a);
+  a = __dp2a_lo(fx.pair[4], t2, a);
+  a = __dp2a_hi(fx.pair[5], t2, a);
+  a = __dp2a_lo(fx.pair[6], t3, a);
+  afix = __dp2a_hi(fx.pair[7], t3, a);
+}
+
+// The same sums for a code vector whose scale lies far below the block maximum: binary64
+// accumulation in element order.
+__device__ __forceinline__ void code_sums_wide(const float (&w)[16], unsigned int c0, unsigned int c1, double& A,
+                                               double& B) {
   double sa = 0.0;
   float sb = 0.0f;
+#pragma unroll
   for (int j = 0; j < 16; ++j) {
-    float m = e2m1_round(__fmul_rn(a[j], r));
-    sa = fma(static_cast<double>(a[j]), static_cast<double>(m), sa);
+    const unsigned int code = ((j < 8 ? c0 : c1) >> (4 * (j & 7))) & 7u;
+    const float m = e2m1_code_value(code);
+    sa = fma(static_cast<double>(fabsf(w[j])), static_cast<double>(m), sa);
     sb = __fmaf_rn(m, m, sb);
   }
   A = sa;
-  B = sb;
+  B = static_cast<double>(sb);
+}
+
+// A = sum |w_j| m_j and B = sum m_j^2 of a code vector made with reciprocal scale r.
+__device__ __forceinline__ void block_sums(const Block& blk, const Fixed& fx, float r, unsigned int c0,
+                                           unsigned int c1, double& A, double& B, unsigned int& wide) {
+  if (fx.ok && __fmul_rn(blk.bmax, r) <= 32.0f) {
+    unsigned int afix, b4;
+    code_sums(fx, c0, c1, afix, b4);
+    A = uint_to_double(afix) * fx.unit;
+    B = uint_to_double(b4) * 0.25;
+  } else {
+    code_sums_wide(blk.w, c0, c1, A, B);
+    ++wide;
+  }
 }
 
 __device__ __forceinline__ float recip_scale(float alpha, float dq) {
@@ -179,7 +366,7 @@ __device__ __forceinline__ double warp_sum(double v) {
   return v;
 }
 
-// Block-wide sums of up to four doubles, then one atomicAdd each from thread 0.
+// CTA-wide sums of N doubles, then one atomicAdd each from thread 0.
 template <int N>
 __device__ __forceinline__ void cta_accumulate(double (&v)[N], double* const (&dst)[N]) {
   __shared__ double red[N][kThreads / 32];
@@ -200,12 +387,6 @@ __device__ __forceinline__ void cta_accumulate(double (&v)[N], double* const (&d
   }
 }
 
-__device__ __forceinline__ const uint16_t* block_ptr(const Params& p, unsigned int b) {
-  const unsigned int row = b / p.nbc;
-  const unsigned int cb = b - row * p.nbc;
-  return p.W + static_cast<long long>(row) * p.ld + static_cast<long long>(cb) * 16;
-}
-
 // Data-dependent status from the tensor maximum (bf16 magnitude bits).
 __device__ __forceinline__ int status_from_amax(unsigned int amax_bits) {
   if (amax_bits >= 0x7F80u) return SOAR_STATUS_NONFINITE;
@@ -224,52 +405,75 @@ __device__ __forceinline__ bool stops_after(double prev, double cur, float eps) 
 
 // ------------------------------------------------------------------ kernels
 
-__global__ void __launch_bounds__(kThreads) amax_kernel(Params p) {
+// bf16 magnitude bits (15 bits) -> the binary64 with the same value; zero and bf16
+// subnormals (below 1.2e-38) map to zero.
+__device__ __forceinline__ double bf16_mag_to_double(unsigned int h15) {
+  const unsigned int hi = (h15 & 0x7F80u) ? (h15 << 13) + 0x38000000u : 0u;
+  return __hiloint2double(static_cast<int>(hi), 0);
+}
+
+// Eq. 1's tensor maximum, plus sum W^2 (binary64) for the error report.
+__global__ void __launch_bounds__(kThreads) amax_kernel(Params p, int reverse) {
+  __shared__ Ring ring;
+  ring_start(ring, p, reverse);
+  const unsigned int ntc = tiles_of_cta(p);
   unsigned int mx = 0;
-  for (unsigned int b = blockIdx.x * kThreads + threadIdx.x; b < p.nblk; b += gridDim.x * kThreads) {
-    const uint4* q = reinterpret_cast<const uint4*>(block_ptr(p, b));
-    const uint4 v0 = __ldg(q), v1 = __ldg(q + 1);
-    unsigned int m = __vmaxu2(v0.x & 0x7FFF7FFFu, v0.y & 0x7FFF7FFFu);
-    m = __vmaxu2(m, v0.z & 0x7FFF7FFFu);
-    m = __vmaxu2(m, v0.w & 0x7FFF7FFFu);
-    m = __vmaxu2(m, v1.x & 0x7FFF7FFFu);
-    m = __vmaxu2(m, v1.y & 0x7FFF7FFFu);
-    m = __vmaxu2(m, v1.z & 0x7FFF7FFFu);
-    m = __vmaxu2(m, v1.w & 0x7FFF7FFFu);
-    mx = __vmaxu2(mx, m);
+  double sq[2] = {0.0, 0.0};
+  unsigned int n = 0;
+  for (; n < ntc; ++n) {
+    uint4 v0, v1;
+    if (!ring_next(ring, p, n, ntc, reverse, v0, v1)) break;
+    const unsigned int b = tile_of(p, n, reverse) * kThreads + threadIdx.x;
+    if (b >= p.nblk) continue;
+    const unsigned int u[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const unsigned int m = u[i] & 0x7FFF7FFFu;
+      mx = __vmaxu2(mx, m);
+      const double lo = bf16_mag_to_double(m & 0xFFFFu), hi = bf16_mag_to_double(m >> 16);
+      sq[0] = fma(lo, lo, sq[0]);
+      sq[1] = fma(hi, hi, sq[1]);
+    }
   }
+  if (n < ntc) ring_abort(ring, p, n, ntc);
   mx = max(mx & 0xFFFFu, mx >> 16);
   mx = __reduce_max_sync(0xFFFFFFFFu, mx);
-  __shared__ unsigned int red[kThreads / 32];
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    unsigned int m = 0;
-    for (int w = 0; w < kThreads / 32; ++w) m = max(m, red[w]);
-    atomicMax(&p.ws->amax_bits, m);
-  }
+  if ((threadIdx.x & 31) == 0 && mx) atomicMax(&p.ws->amax_bits, mx);
+  double acc[1] = {sq[0] + sq[1]};
+  double* const dst[1] = {&p.ws->sumsq};
+  cta_accumulate<1>(acc, dst);
 }
 
 // Algorithm 1 "Initialization" (Eq. 1): alpha0 = amax/(6*448), dd0 = E4M3(bmax/(6 alpha0)),
-// dq0 = dd0; first codes (Eq. 2); stage-0 sums for Eq. 5 and the starting error.
-__global__ void __launch_bounds__(kThreads) init_kernel(Params p) {
+// dq0 = dd0; first codes (Eq. 2); stage-0 sums for Eq. 5 and the starting error.  Codes and
+// scales are written here only when no iteration follows (final != 0).
+__global__ void __launch_bounds__(kThreads) init_kernel(Params p, int reverse, int final) {
+  __shared__ Ring ring;
   const unsigned int amax_bits = p.ws->amax_bits;
   const int st = status_from_amax(amax_bits);
   if (st & (SOAR_STATUS_NONFINITE | SOAR_STATUS_RANGE)) return;
+  ring_start(ring, p, reverse);
+  const unsigned int ntc = tiles_of_cta(p);
   const float alpha = (st & SOAR_STATUS_ZERO_TENSOR) ? 1.0f : __fdiv_rn(bits_to_mag(amax_bits), 2688.0f);
   const float six_alpha = __fmul_rn(alpha, 6.0f);
   const double alpha_d = static_cast<double>(alpha);
-  double acc[4] = {0.0, 0.0, 0.0, 0.0};   // num, den, sse, sumsq
-  unsigned int zeros = 0;
-  for (unsigned int b = blockIdx.x * kThreads + threadIdx.x; b < p.nblk; b += gridDim.x * kThreads) {
+  double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum
+  unsigned int zeros = 0, wide = 0;
+  unsigned int n = 0;
+  for (; n < ntc; ++n) {
+    uint4 v0, v1;
+    if (!ring_next(ring, p, n, ntc, reverse, v0, v1)) break;
+    const unsigned int b = tile_of(p, n, reverse) * kThreads + threadIdx.x;
+    if (b >= p.nblk) continue;
     Block blk;
-    load_block(block_ptr(p, b), blk);
-    uint2 out;
+    unpack_block(v0, v1, blk);
+    uint2 codes;
     if (blk.bmax == 0.0f) {
-      out.x = blk.sign0;
-      out.y = blk.sign1;
-      reinterpret_cast<uint2*>(p.packed)[b] = out;
+      // all-zero block: codes carry the sign bits only, scale byte 0, left out of all sums
+      round_block(blk, 1.0f, codes.x, codes.y);
+      reinterpret_cast<uint2*>(p.packed)[b] = codes;
       p.scales[b] = 0;
+      if (p.state != nullptr) p.state[b] = make_uint2(0u, 0u);
       ++zeros;
       continue;
     }
@@ -277,37 +481,44 @@ __global__ void __launch_bounds__(kThreads) init_kernel(Params p) {
     c = max(c, 1);
     const float v = e4m3_value(c);
     const float r = recip_scale(alpha, v);
-    float m[16];
-    float Bf = 0.0f;
-    double A = 0.0, S = 0.0;
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      m[j] = e2m1_round(__fmul_rn(blk.a[j], r));
-      const double aj = static_cast<double>(blk.a[j]);
-      A = fma(aj, static_cast<double>(m[j]), A);
-      S = fma(aj, aj, S);
-      Bf = __fmaf_rn(m[j], m[j], Bf);
+    round_block(blk, r, codes.x, codes.y);
+    Fixed fx;
+    make_fixed(blk, fx);
+    double A, B;
+    block_sums(blk, fx, r, codes.x, codes.y, A, B, wide);
+    if (final) {
+      reinterpret_cast<uint2*>(p.packed)[b] = codes;
+      p.scales[b] = static_cast<uint8_t>(c);
     }
-    out.x = pack_e2m1x8(m) | blk.sign0;
-    out.y = pack_e2m1x8(m + 8) | blk.sign1;
-    reinterpret_cast<uint2*>(p.packed)[b] = out;
-    p.scales[b] = static_cast<uint8_t>(c);
-    const double B = static_cast<double>(Bf), vd = static_cast<double>(v);
+    if (p.state != nullptr)
+      p.state[b] = make_uint2(__float_as_uint(static_cast<float>(A)),
+                              static_cast<unsigned int>(B * 4.0) | (static_cast<unsigned int>(c) << 16));
+    const double vd = static_cast<double>(v);
     const double sd = alpha_d * vd;
-    acc[0] += A * vd;
-    acc[1] += B * vd * vd;
-    acc[2] += S + sd * fma(sd, B, -2.0 * A);
-    acc[3] += S;
+    acc[0] = fma(A, vd, acc[0]);
+    acc[1] = fma(B * vd, vd, acc[1]);
+    acc[2] += sd * fma(sd, B, -2.0 * A);
   }
-  double* const dst[4] = {&p.ws->num[0], &p.ws->den[0], &p.ws->sse[0], &p.ws->sumsq};
-  cta_accumulate<4>(acc, dst);
+  if (n < ntc) ring_abort(ring, p, n, ntc);
+  double* const dst[3] = {&p.ws->num[0], &p.ws->den[0], &p.ws->gsum[0]};
+  cta_accumulate<3>(acc, dst);
   zeros = __reduce_add_sync(0xFFFFFFFFu, zeros);
   if ((threadIdx.x & 31) == 0 && zeros) atomicAdd(&p.ws->zero_blocks, static_cast<unsigned long long>(zeros));
+  wide = __reduce_add_sync(0xFFFFFFFFu, wide);
+  if ((threadIdx.x & 31) == 0 && wide) atomicAdd(&p.ws->wide, static_cast<unsigned long long>(wide));
+}
+
+// Error of stage s (Eq. 4) from the tensor sums.
+__device__ __forceinline__ double stage_sse(const Ws* ws, int s) {
+  return fmax(ws->sumsq + ws->gsum[s], 0.0);
 }
 
 // One iteration t of Algorithm 1 for every block: Eq. 5 (from stage-t sums), Eq. 6,
 // App. B.3 candidate sets, Eq. 8 search, winner stored, stage-(t+1) sums accumulated.
-__global__ void __launch_bounds__(kThreads) iterate_kernel(Params p, int t) {
+// Codes and scale bytes are written when `emit` is set (the state after this iteration may
+// be the one returned).
+__global__ void __launch_bounds__(kThreads) iterate_kernel(Params p, int t, int reverse, int emit) {
+  __shared__ Ring ring;
   __shared__ float s_beta[SOAR_MAX_BETA];
   __shared__ float s_alpha;
   __shared__ int s_run;
@@ -315,12 +526,12 @@ __global__ void __launch_bounds__(kThreads) iterate_kernel(Params p, int t) {
   if (threadIdx.x == 0) {
     int run = 1;
     const unsigned int amax_bits = ws->amax_bits;
-    if (status_from_amax(amax_bits) != 0) run = 0;
+    if (status_from_amax(amax_bits) != 0 || ws->error != 0) run = 0;
     float alpha = __fdiv_rn(bits_to_mag(amax_bits), 2688.0f);
     if (run) {
-      double prev = ws->sse[0];
+      double prev = stage_sse(ws, 0);
       for (int i = 0; i < t; ++i) {           // did an earlier iteration trigger the stop?
-        const double cur = ws->sse[i + 1];
+        const double cur = stage_sse(ws, i + 1);
         if (stops_after(prev, cur, p.early_stop_rel)) { run = 0; break; }
         prev = cur;
       }
@@ -334,34 +545,28 @@ __global__ void __launch_bounds__(kThreads) iterate_kernel(Params p, int t) {
     s_beta[k] = static_cast<float>((100.0 + static_cast<double>((k - p.n_beta / 2) * p.beta_step_pct)) / 100.0);
   __syncthreads();
   if (!s_run) return;
+  ring_start(ring, p, reverse);
+  const unsigned int ntc = tiles_of_cta(p);
   const float alpha = s_alpha;
   const double alpha_d = static_cast<double>(alpha);
   const int n_dq = p.n_dq, n_beta = p.n_beta;
 
-  double acc[3] = {0.0, 0.0, 0.0};   // num, den, sse of stage t+1
+  double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum of stage t+1
   unsigned int wide = 0;
-  for (unsigned int b = blockIdx.x * kThreads + threadIdx.x; b < p.nblk; b += gridDim.x * kThreads) {
-    const int d_cur = p.scales[b];
+  unsigned int n = 0;
+  for (; n < ntc; ++n) {
+    uint4 v0, v1;
+    if (!ring_next(ring, p, n, ntc, reverse, v0, v1)) break;
+    const unsigned int b = tile_of(p, n, reverse) * kThreads + threadIdx.x;
+    if (b >= p.nblk) continue;
+    const uint2 st = p.state[b];
+    const int d_cur = static_cast<int>(st.y >> 16);
     if (d_cur == 0) continue;                       // all-zero block: nothing to optimise
     Block blk;
-    load_block(block_ptr(p, b), blk);
-    const uint2 cur = reinterpret_cast<const uint2*>(p.packed)[b];
-    // Sums of the current codes (the winner of the previous stage), exact in binary64.
-    double A0 = 0.0, S = 0.0;
-    float B0 = 0.0f;
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const unsigned int code = ((j < 8 ? cur.x : cur.y) >> (4 * (j & 7))) & 7u;
-      const float m = e2m1_code_value(code);
-      const double aj = static_cast<double>(blk.a[j]);
-      A0 = fma(aj, static_cast<double>(m), A0);
-      S = fma(aj, aj, S);
-      B0 = __fmaf_rn(m, m, B0);
-    }
-    // Eq. 6 with the new alpha; all codes zero keeps the stored scale.
-    const float center = (B0 > 0.0f)
-        ? __fdiv_rn(static_cast<float>(A0), __fmul_rn(alpha, B0))
-        : e4m3_value(d_cur);
+    unpack_block(v0, v1, blk);
+    // Eq. 6 with the new alpha from the previous winner's sums; all codes zero keeps the stored scale.
+    const float B0 = 0.25f * static_cast<float>(st.y & 0xFFFFu);
+    const float center = (B0 > 0.0f) ? __fdiv_rn(__uint_as_float(st.x), __fmul_rn(alpha, B0)) : e4m3_value(d_cur);
     // App. B.3: E4M3 codes around the analytic scale.
     int d_lo, d_hi;
     {
@@ -374,54 +579,56 @@ __global__ void __launch_bounds__(kThreads) iterate_kernel(Params p, int t) {
         d_hi = cf + n_dq / 2;
       }
     }
+    const int dc0 = max(1, min(0x7E, d_lo)), dc1 = max(1, min(0x7E, d_lo + 1));
+    const double sd0 = alpha_d * static_cast<double>(e4m3_value(dc0));
+    const double sd1 = alpha_d * static_cast<double>(e4m3_value(dc1));
+    Fixed fx;
+    make_fixed(blk, fx);
     // Eq. 8 over beta ascending, then scale code ascending; strict '<' keeps the first minimum.
     double best = __longlong_as_double(0x7FF0000000000000ll);
-    double bestA = 0.0;
-    float bestB = 0.0f;
-    int best_k = 0, best_d = max(1, min(0x7E, d_lo));
-    double prevA = -1.0;
-    float prevB = -1.0f;
+    double bestA = 0.0, bestB = 0.0;
+    int best_d = dc0;
+    unsigned int best0 = 0, best1 = 0, prev0 = 0, prev1 = 0;
     for (int k = 0; k < n_beta; ++k) {
       const float r = recip_scale(alpha, __fmul_rn(center, s_beta[k]));
-      double A;
-      float B;
-      if (__fmul_rn(blk.bmax, r) <= 32.0f) {
-        float Af;
-        eval_candidate(blk.a, r, Af, B);
-        A = static_cast<double>(Af);
+      unsigned int c0, c1;
+      round_block(blk, r, c0, c1);
+      if (k > 0 && c0 == prev0 && c1 == prev1) continue;   // same codes as the previous beta: same errors
+      prev0 = c0;
+      prev1 = c1;
+      double A, B;
+      block_sums(blk, fx, r, c0, c1, A, B, wide);
+      const double A2 = -2.0 * A;
+      if (n_dq <= 2) {
+        const double g0 = sd0 * fma(sd0, B, A2);            // block error minus sum W^2
+        if (g0 < best) { best = g0; bestA = A; bestB = B; best_d = dc0; best0 = c0; best1 = c1; }
+        if (n_dq == 2) {
+          const double g1 = sd1 * fma(sd1, B, A2);
+          if (g1 < best) { best = g1; bestA = A; bestB = B; best_d = dc1; best0 = c0; best1 = c1; }
+        }
       } else {
-        eval_candidate_wide(blk.a, r, A, B);
-        ++wide;
-      }
-      if (A == prevA && B == prevB) continue;     // same sums as the previous beta: same errors
-      prevA = A;
-      prevB = B;
-      const double Bd = static_cast<double>(B);
-      for (int d = d_lo; d <= d_hi; ++d) {
-        const int dc = max(1, min(0x7E, d));
-        const double sd = alpha_d * static_cast<double>(e4m3_value(dc));
-        const double g = sd * fma(sd, Bd, -2.0 * A);   // block error minus sum W^2
-        if (g < best) { best = g; bestA = A; bestB = B; best_k = k; best_d = dc; }
+        for (int d = d_lo; d <= d_hi; ++d) {
+          const int dc = max(1, min(0x7E, d));
+          const double sd = alpha_d * static_cast<double>(e4m3_value(dc));
+          const double g = sd * fma(sd, B, A2);
+          if (g < best) { best = g; bestA = A; bestB = B; best_d = dc; best0 = c0; best1 = c1; }
+        }
       }
     }
-    // Winner's codes (the assignment the next iteration, or the output, starts from).
-    {
-      const float r = recip_scale(alpha, __fmul_rn(center, s_beta[best_k]));
-      float m[16];
-#pragma unroll
-      for (int j = 0; j < 16; ++j) m[j] = e2m1_round(__fmul_rn(blk.a[j], r));
-      uint2 out;
-      out.x = pack_e2m1x8(m) | blk.sign0;
-      out.y = pack_e2m1x8(m + 8) | blk.sign1;
-      reinterpret_cast<uint2*>(p.packed)[b] = out;
+    // The winner: codes and scale out, sums kept for the next iteration's Eq. 6.
+    if (emit) {
+      reinterpret_cast<uint2*>(p.packed)[b] = make_uint2(best0, best1);
       p.scales[b] = static_cast<uint8_t>(best_d);
     }
+    p.state[b] = make_uint2(__float_as_uint(static_cast<float>(bestA)),
+                            static_cast<unsigned int>(bestB * 4.0) | (static_cast<unsigned int>(best_d) << 16));
     const double vd = static_cast<double>(e4m3_value(best_d));
-    acc[0] += bestA * vd;
-    acc[1] += static_cast<double>(bestB) * vd * vd;
-    acc[2] += S + best;
+    acc[0] = fma(bestA, vd, acc[0]);
+    acc[1] = fma(bestB * vd, vd, acc[1]);
+    acc[2] += best;
   }
-  double* const dst[3] = {&p.ws->num[t + 1], &p.ws->den[t + 1], &p.ws->sse[t + 1]};
+  if (n < ntc) ring_abort(ring, p, n, ntc);
+  double* const dst[3] = {&p.ws->num[t + 1], &p.ws->den[t + 1], &p.ws->gsum[t + 1]};
   cta_accumulate<3>(acc, dst);
   wide = __reduce_add_sync(0xFFFFFFFFu, wide);
   if ((threadIdx.x & 31) == 0 && wide) atomicAdd(&p.ws->wide, static_cast<unsigned long long>(wide));
@@ -437,12 +644,12 @@ __global__ void finalize_kernel(Params p, float* out_alpha, soar_result* res) {
   int iters = 0;
   double ta[SOAR_MAX_ITERS + 1], ts[SOAR_MAX_ITERS + 1];
   ta[0] = static_cast<double>(alpha);
-  ts[0] = ws->sse[0];
-  if (st == 0) {
-    double prev = ws->sse[0];
+  ts[0] = (st == 0) ? stage_sse(ws, 0) : 0.0;
+  if (st == 0 && ws->error == 0) {
+    double prev = ts[0];
     for (int i = 0; i < p.max_iters; ++i) {
       if (ws->den[i] > 0.0) alpha = static_cast<float>(ws->num[i] / ws->den[i]);
-      const double cur = ws->sse[i + 1];
+      const double cur = stage_sse(ws, i + 1);
       iters = i + 1;
       ta[iters] = static_cast<double>(alpha);
       ts[iters] = cur;
@@ -452,7 +659,7 @@ __global__ void finalize_kernel(Params p, float* out_alpha, soar_result* res) {
   }
   *out_alpha = alpha;
   if (res != nullptr) {
-    res->status = st;
+    res->status = st | (ws->error ? SOAR_STATUS_INTERNAL : 0);
     res->iters_run = iters;
     res->alpha = alpha;
     res->amax = bits_to_mag(amax_bits);
@@ -575,15 +782,19 @@ int sm_count() {
   return g_sm_count[dev];
 }
 
+// Grid of a persistent kernel: every SM filled to the kernel's occupancy, never more CTAs
+// than tiles.
 template <typename K>
 unsigned int persistent_grid(K kernel, unsigned int nblk, int threads) {
   int per_sm = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, 0) != cudaSuccess || per_sm <= 0)
-    per_sm = 4;
+    per_sm = 2;
   const unsigned long long cap = static_cast<unsigned long long>(sm_count()) * per_sm;
   const unsigned long long need = (static_cast<unsigned long long>(nblk) + threads - 1) / threads;
   return static_cast<unsigned int>(need < cap ? (need ? need : 1) : cap);
 }
+
+size_t round256(size_t n) { return (n + 255) / 256 * 256; }
 
 bool cfg_ok(const soar_cfg* cfg) {
   return cfg != nullptr && cfg->struct_size == sizeof(soar_cfg);
@@ -640,11 +851,10 @@ int soar_default_cfg(soar_cfg* cfg, int preset) {
 
 size_t soar_workspace_bytes(int64_t rows, int64_t cols, const soar_cfg* cfg) {
   if (check_cfg(cfg) != SOAR_OK || rows <= 0 || cols <= 0 || cols % 16 != 0) return 0;
+  const size_t nblk = static_cast<size_t>(rows) * static_cast<size_t>(cols / 16);
   size_t n = kWsFixedBytes;
-  if (!(cfg->scale_layout & SOAR_SCALES_LINEAR)) {
-    const size_t lin = static_cast<size_t>(rows) * static_cast<size_t>(cols / 16);
-    n += (lin + 255) / 256 * 256;
-  }
+  if (cfg->max_iters > 0) n += round256(nblk * sizeof(uint2));
+  if (!(cfg->scale_layout & SOAR_SCALES_LINEAR)) n += round256(nblk);
   return n;
 }
 
@@ -682,12 +892,21 @@ int soar_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, co
   Params p;
   p.W = static_cast<const uint16_t*>(W_bf16);
   p.packed = static_cast<uint8_t*>(out_fp4_packed);
-  p.scales = want_lin ? static_cast<uint8_t*>(out_e4m3_scales)
-                      : static_cast<uint8_t*>(workspace) + kWsFixedBytes;
   p.ws = static_cast<Ws*>(workspace);
   p.ld = ld;
   p.nbc = static_cast<unsigned int>(cols / 16);
   p.nblk = static_cast<unsigned int>(rows * (cols / 16));
+  p.ntiles = (p.nblk + kThreads - 1) / kThreads;
+  p.contiguous = (ld == cols) ? 1 : 0;
+  {
+    uint8_t* next = static_cast<uint8_t*>(workspace) + kWsFixedBytes;
+    p.state = nullptr;
+    if (cfg->max_iters > 0) {
+      p.state = reinterpret_cast<uint2*>(next);
+      next += round256(static_cast<size_t>(p.nblk) * sizeof(uint2));
+    }
+    p.scales = want_lin ? static_cast<uint8_t*>(out_e4m3_scales) : next;
+  }
   p.max_iters = cfg->max_iters;
   p.early_stop_rel = cfg->early_stop_rel;
   p.n_dq = cfg->n_dq;
@@ -695,18 +914,27 @@ int soar_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, co
   p.beta_step_pct = cfg->beta_step_pct;
 
   if (cudaMemsetAsync(workspace, 0, kWsFixedBytes, st) != cudaSuccess) return SOAR_ERR_CUDA;
+  // Passes alternate direction over the tiles: each starts where the previous one ended,
+  // on data still in L2.
+  int reverse = 0;
   {
     ScopedLaunch sl(K_AMAX, st);
-    amax_kernel<<<persistent_grid(amax_kernel, p.nblk, kThreads), kThreads, 0, st>>>(p);
+    amax_kernel<<<persistent_grid(amax_kernel, p.nblk, kThreads), kThreads, 0, st>>>(p, reverse);
   }
+  reverse ^= 1;
   {
     ScopedLaunch sl(K_INIT, st);
-    init_kernel<<<persistent_grid(init_kernel, p.nblk, kThreads), kThreads, 0, st>>>(p);
+    init_kernel<<<persistent_grid(init_kernel, p.nblk, kThreads), kThreads, 0, st>>>(p, reverse,
+                                                                                     cfg->max_iters == 0 ? 1 : 0);
   }
   const unsigned int g_it = persistent_grid(iterate_kernel, p.nblk, kThreads);
+  const bool may_stop = cfg->early_stop_rel > 0.0f;
   for (int t = 0; t < cfg->max_iters; ++t) {
+    reverse ^= 1;
+    // with the early stop on, any iteration may turn out to be the last one
+    const int emit = (may_stop || t == cfg->max_iters - 1) ? 1 : 0;
     ScopedLaunch sl(K_ITERATE, st);
-    iterate_kernel<<<g_it, kThreads, 0, st>>>(p, t);
+    iterate_kernel<<<g_it, kThreads, 0, st>>>(p, t, reverse, emit);
   }
   {
     ScopedLaunch sl(K_FINALIZE, st);
