@@ -75,12 +75,29 @@ def iterate_ops_per_block(cfg) -> float:
     return cfg.n_beta * (16 * OPS_PER_ELEMENT_EVAL + cfg.n_dq * OPS_PER_PAIR_SCORE)
 
 
-KERNEL_BYTES_PER_ELEM = {          # algorithmic HBM bytes per weight element and launch
-    "amax_kernel": 2.0,                                  # read W
-    "init_kernel": 2.0 + 0.5 + 1.0 / 16,                 # read W, write codes + scale byte
-    "iterate_kernel": 2.0 + 2 * (0.5 + 1.0 / 16),        # read W, codes, scale; write codes, scale
-    "dequant_error_kernel": 2.0 + 0.5 + 1.0 / 16,
-}
+OUT_BYTES = 0.5 + 1.0 / 16          # codes + scale byte per element
+STATE_BYTES = 0.5                   # 8 bytes of carried sums per 16-element block
+
+
+def kernel_bytes_per_elem(name: str, cfg, t: int = 0) -> float:
+    """Algorithmic HBM bytes per weight element of one launch (iteration ``t`` for iterate)."""
+    if name == "amax_kernel":
+        return 2.0                                                   # read W
+    if name == "init_kernel":                                        # read W; write state, or the outputs when T = 0
+        return 2.0 + (STATE_BYTES if cfg.max_iters > 0 else OUT_BYTES)
+    if name == "iterate_kernel":                                     # read W + state; write state unless last; outputs
+        last = t == cfg.max_iters - 1
+        emits = last or cfg.early_stop_rel > 0
+        return 2.0 + STATE_BYTES + (0.0 if last else STATE_BYTES) + (OUT_BYTES if emits else 0.0)
+    if name == "dequant_error_kernel":
+        return 2.0 + OUT_BYTES
+    return 0.0
+
+
+def call_bytes_per_elem(cfg, iters_run: int) -> float:
+    """Algorithmic HBM bytes per element of one soar_quantize call that ran ``iters_run`` iterations."""
+    return (kernel_bytes_per_elem("amax_kernel", cfg) + kernel_bytes_per_elem("init_kernel", cfg)
+            + sum(kernel_bytes_per_elem("iterate_kernel", cfg, t) for t in range(iters_run)))
 
 
 class ClockSampler:
@@ -250,13 +267,15 @@ def run_ours(args):
                         frac=achieved / peak, traffic=None, launches=n_launch,
                         active_launches=sum(iters) * args.steps, kernel_ms_per_step=tot_ms / args.steps,
                         peak_source="148 SMs x 128 FP32 lanes x clocks.max.sm",
-                        hbm_gbs_for_context=blocks_iters * 16 * KERNEL_BYTES_PER_ELEM[dom] / (tot_ms * 1e-3) / 1e9)
+                        hbm_gbs_for_context=sum(
+                            s.rows * s.cols * kernel_bytes_per_elem(dom, cfg, t)
+                            for s, it in zip(wl.tensors, iters) for t in range(it)) * args.steps / (tot_ms * 1e-3) / 1e9)
     else:
         if dom == "iterate_kernel":
-            units = sum(s.rows * s.cols * it for s, it in zip(wl.tensors, iters)) * args.steps
+            byts = sum(s.rows * s.cols * kernel_bytes_per_elem(dom, cfg, t)
+                       for s, it in zip(wl.tensors, iters) for t in range(it)) * args.steps
         else:
-            units = elements * args.steps
-        byts = units * KERNEL_BYTES_PER_ELEM.get(dom, 2.0)
+            byts = elements * args.steps * kernel_bytes_per_elem(dom, cfg)
         achieved = byts / (tot_ms * 1e-3) / 1e9
         roofline = dict(bound="hbm", kernel=dom, achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
                         frac=achieved / peaks["hbm_gbs"], traffic=None, launches=n_launch,
@@ -270,8 +289,7 @@ def run_ours(args):
     if args.preset == "paper" and not args.no_single_pass:
         sp = preset_cfg(api, "single_pass")
         sp_ms, sp_tr = timed(lambda: step(sp), max(args.steps, 5), 3)
-        sp_bytes = elements * (KERNEL_BYTES_PER_ELEM["amax_kernel"] + KERNEL_BYTES_PER_ELEM["init_kernel"]
-                               + KERNEL_BYTES_PER_ELEM["iterate_kernel"])
+        sp_bytes = elements * call_bytes_per_elem(sp, sp.max_iters)
         gbs = sp_bytes / (sp_ms * 1e-3) / 1e9
         extra["single_pass"] = dict(
             ms_per_step=sp_ms, value=world * 2.0 * elements / (sp_ms * 1e-3) / 1e9, unit="GB/s",

@@ -513,36 +513,71 @@ __device__ __forceinline__ double stage_sse(const Ws* ws, int s) {
   return fmax(ws->sumsq + ws->gsum[s], 0.0);
 }
 
+// Head of an iteration (one thread): has the loop already stopped (Sec. 4.1), and the global
+// scale of Eq. 5 from the sums of the stages so far.
+__device__ __forceinline__ void iteration_head(const Params& p, int t, float& alpha_out, int& run_out) {
+  const Ws* ws = p.ws;
+  int run = 1;
+  const unsigned int amax_bits = ws->amax_bits;
+  if (status_from_amax(amax_bits) != 0 || ws->error != 0) run = 0;
+  float alpha = __fdiv_rn(bits_to_mag(amax_bits), 2688.0f);
+  if (run) {
+    double prev = stage_sse(ws, 0);
+    for (int i = 0; i < t; ++i) {           // did an earlier iteration trigger the stop?
+      const double cur = stage_sse(ws, i + 1);
+      if (stops_after(prev, cur, p.early_stop_rel)) { run = 0; break; }
+      prev = cur;
+    }
+    for (int i = 0; i <= t; ++i)            // Eq. 5: alpha^(i+1) from stage-i sums
+      if (ws->den[i] > 0.0) alpha = static_cast<float>(ws->num[i] / ws->den[i]);
+  }
+  alpha_out = alpha;
+  run_out = run;
+}
+
+// Eq. 6 with the new alpha from the previous winner's sums (all codes zero keeps the stored
+// scale), and App. B.3's E4M3 codes around it: d_lo .. d_hi before clipping.
+__device__ __forceinline__ float block_center(const uint2 st, float alpha, int n_dq, int& d_lo, int& d_hi) {
+  const int d_cur = static_cast<int>(st.y >> 16);
+  const float B0 = 0.25f * static_cast<float>(st.y & 0xFFFFu);
+  const float center = (B0 > 0.0f) ? __fdiv_rn(__uint_as_float(st.x), __fmul_rn(alpha, B0)) : e4m3_value(d_cur);
+  const int cn = e4m3_encode(center);
+  if (n_dq <= 1) {
+    d_lo = d_hi = cn;
+  } else {
+    const int cf = (e4m3_value(cn) > center) ? cn - 1 : cn;   // largest code with value <= center
+    d_lo = cf - (n_dq / 2 - 1);
+    d_hi = cf + n_dq / 2;
+  }
+  return center;
+}
+
+__device__ __forceinline__ int clip_code(int d) { return max(1, min(0x7E, d)); }
+
 // One iteration t of Algorithm 1 for every block: Eq. 5 (from stage-t sums), Eq. 6,
 // App. B.3 candidate sets, Eq. 8 search, winner stored, stage-(t+1) sums accumulated.
 // Codes and scale bytes are written when `emit` is set (the state after this iteration may
-// be the one returned).
-__global__ void __launch_bounds__(kThreads) iterate_kernel(Params p, int t, int reverse, int emit) {
+// be the one returned); the per-block sums are kept when `keep` is set (another iteration
+// may follow).  kSingle is the shape with one quantization scale (beta = 1) and at most two
+// dequantization codes, whose passes are bound by HBM rather than by the candidate loop.
+template <bool kSingle>
+__global__ void __launch_bounds__(kThreads, kSingle ? 3 : 2)
+iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
   __shared__ Ring ring;
-  __shared__ float s_beta[SOAR_MAX_BETA];
+  __shared__ float s_beta[kSingle ? 1 : SOAR_MAX_BETA];
   __shared__ float s_alpha;
   __shared__ int s_run;
-  const Ws* ws = p.ws;
   if (threadIdx.x == 0) {
-    int run = 1;
-    const unsigned int amax_bits = ws->amax_bits;
-    if (status_from_amax(amax_bits) != 0 || ws->error != 0) run = 0;
-    float alpha = __fdiv_rn(bits_to_mag(amax_bits), 2688.0f);
-    if (run) {
-      double prev = stage_sse(ws, 0);
-      for (int i = 0; i < t; ++i) {           // did an earlier iteration trigger the stop?
-        const double cur = stage_sse(ws, i + 1);
-        if (stops_after(prev, cur, p.early_stop_rel)) { run = 0; break; }
-        prev = cur;
-      }
-      for (int i = 0; i <= t; ++i)            // Eq. 5: alpha^(i+1) from stage-i sums
-        if (ws->den[i] > 0.0) alpha = static_cast<float>(ws->num[i] / ws->den[i]);
-    }
-    s_alpha = alpha;
+    float a;
+    int run;
+    iteration_head(p, t, a, run);
+    s_alpha = a;
     s_run = run;
   }
-  for (int k = threadIdx.x; k < p.n_beta; k += kThreads)
-    s_beta[k] = static_cast<float>((100.0 + static_cast<double>((k - p.n_beta / 2) * p.beta_step_pct)) / 100.0);
+  if (!kSingle) {
+    for (int k = threadIdx.x; k < p.n_beta; k += kThreads)
+      s_beta[k] = static_cast<float>((100.0 + static_cast<double>((k - p.n_beta / 2) * p.beta_step_pct)) / 100.0);
+  }
   __syncthreads();
   if (!s_run) return;
   ring_start(ring, p, reverse);
@@ -560,58 +595,61 @@ __global__ void __launch_bounds__(kThreads) iterate_kernel(Params p, int t, int 
     const unsigned int b = tile_of(p, n, reverse) * kThreads + threadIdx.x;
     if (b >= p.nblk) continue;
     const uint2 st = p.state[b];
-    const int d_cur = static_cast<int>(st.y >> 16);
-    if (d_cur == 0) continue;                       // all-zero block: nothing to optimise
+    if ((st.y >> 16) == 0) continue;                // all-zero block: nothing to optimise
     Block blk;
     unpack_block(v0, v1, blk);
-    // Eq. 6 with the new alpha from the previous winner's sums; all codes zero keeps the stored scale.
-    const float B0 = 0.25f * static_cast<float>(st.y & 0xFFFFu);
-    const float center = (B0 > 0.0f) ? __fdiv_rn(__uint_as_float(st.x), __fmul_rn(alpha, B0)) : e4m3_value(d_cur);
-    // App. B.3: E4M3 codes around the analytic scale.
     int d_lo, d_hi;
-    {
-      const int cn = e4m3_encode(center);
-      if (n_dq <= 1) {
-        d_lo = d_hi = cn;
-      } else {
-        const int cf = (e4m3_value(cn) > center) ? cn - 1 : cn;   // largest code with value <= center
-        d_lo = cf - (n_dq / 2 - 1);
-        d_hi = cf + n_dq / 2;
-      }
-    }
-    const int dc0 = max(1, min(0x7E, d_lo)), dc1 = max(1, min(0x7E, d_lo + 1));
+    const float center = block_center(st, alpha, n_dq, d_lo, d_hi);
+    const int dc0 = clip_code(d_lo), dc1 = clip_code(d_lo + 1);
     const double sd0 = alpha_d * static_cast<double>(e4m3_value(dc0));
     const double sd1 = alpha_d * static_cast<double>(e4m3_value(dc1));
     Fixed fx;
     make_fixed(blk, fx);
-    // Eq. 8 over beta ascending, then scale code ascending; strict '<' keeps the first minimum.
-    double best = __longlong_as_double(0x7FF0000000000000ll);
-    double bestA = 0.0, bestB = 0.0;
+    double best, bestA, bestB;
     int best_d = dc0;
-    unsigned int best0 = 0, best1 = 0, prev0 = 0, prev1 = 0;
-    for (int k = 0; k < n_beta; ++k) {
-      const float r = recip_scale(alpha, __fmul_rn(center, s_beta[k]));
-      unsigned int c0, c1;
-      round_block(blk, r, c0, c1);
-      if (k > 0 && c0 == prev0 && c1 == prev1) continue;   // same codes as the previous beta: same errors
-      prev0 = c0;
-      prev1 = c1;
-      double A, B;
-      block_sums(blk, fx, r, c0, c1, A, B, wide);
-      const double A2 = -2.0 * A;
-      if (n_dq <= 2) {
-        const double g0 = sd0 * fma(sd0, B, A2);            // block error minus sum W^2
-        if (g0 < best) { best = g0; bestA = A; bestB = B; best_d = dc0; best0 = c0; best1 = c1; }
-        if (n_dq == 2) {
-          const double g1 = sd1 * fma(sd1, B, A2);
-          if (g1 < best) { best = g1; bestA = A; bestB = B; best_d = dc1; best0 = c0; best1 = c1; }
-        }
-      } else {
-        for (int d = d_lo; d <= d_hi; ++d) {
-          const int dc = max(1, min(0x7E, d));
-          const double sd = alpha_d * static_cast<double>(e4m3_value(dc));
-          const double g = sd * fma(sd, B, A2);
-          if (g < best) { best = g; bestA = A; bestB = B; best_d = dc; best0 = c0; best1 = c1; }
+    unsigned int best0, best1;
+    if (kSingle) {
+      // one quantization scale (beta = 1): the codes are fixed, only the E4M3 code is chosen
+      const float r = recip_scale(alpha, center);
+      round_block(blk, r, best0, best1);
+      block_sums(blk, fx, r, best0, best1, bestA, bestB, wide);
+      const double A2 = -2.0 * bestA;
+      best = sd0 * fma(sd0, bestB, A2);               // block error minus sum W^2
+      if (n_dq == 2) {
+        const double g1 = sd1 * fma(sd1, bestB, A2);
+        if (g1 < best) { best = g1; best_d = dc1; }
+      }
+    } else {
+      // Eq. 8 over beta ascending, then scale code ascending; strict '<' keeps the first minimum.
+      best = __longlong_as_double(0x7FF0000000000000ll);
+      bestA = 0.0;
+      bestB = 0.0;
+      best0 = best1 = 0;
+      unsigned int prev0 = 0, prev1 = 0;
+      for (int k = 0; k < n_beta; ++k) {
+        const float r = recip_scale(alpha, __fmul_rn(center, s_beta[k]));
+        unsigned int c0, c1;
+        round_block(blk, r, c0, c1);
+        if (k > 0 && c0 == prev0 && c1 == prev1) continue;   // same codes as the previous beta: same errors
+        prev0 = c0;
+        prev1 = c1;
+        double A, B;
+        block_sums(blk, fx, r, c0, c1, A, B, wide);
+        const double A2 = -2.0 * A;
+        if (n_dq <= 2) {
+          const double g0 = sd0 * fma(sd0, B, A2);
+          if (g0 < best) { best = g0; bestA = A; bestB = B; best_d = dc0; best0 = c0; best1 = c1; }
+          if (n_dq == 2) {
+            const double g1 = sd1 * fma(sd1, B, A2);
+            if (g1 < best) { best = g1; bestA = A; bestB = B; best_d = dc1; best0 = c0; best1 = c1; }
+          }
+        } else {
+          for (int d = d_lo; d <= d_hi; ++d) {
+            const int dc = clip_code(d);
+            const double sd = alpha_d * static_cast<double>(e4m3_value(dc));
+            const double g = sd * fma(sd, B, A2);
+            if (g < best) { best = g; bestA = A; bestB = B; best_d = dc; best0 = c0; best1 = c1; }
+          }
         }
       }
     }
@@ -620,8 +658,9 @@ __global__ void __launch_bounds__(kThreads) iterate_kernel(Params p, int t, int 
       reinterpret_cast<uint2*>(p.packed)[b] = make_uint2(best0, best1);
       p.scales[b] = static_cast<uint8_t>(best_d);
     }
-    p.state[b] = make_uint2(__float_as_uint(static_cast<float>(bestA)),
-                            static_cast<unsigned int>(bestB * 4.0) | (static_cast<unsigned int>(best_d) << 16));
+    if (keep)
+      p.state[b] = make_uint2(__float_as_uint(static_cast<float>(bestA)),
+                              static_cast<unsigned int>(bestB * 4.0) | (static_cast<unsigned int>(best_d) << 16));
     const double vd = static_cast<double>(e4m3_value(best_d));
     acc[0] = fma(bestA, vd, acc[0]);
     acc[1] = fma(bestB * vd, vd, acc[1]);
@@ -635,42 +674,56 @@ __global__ void __launch_bounds__(kThreads) iterate_kernel(Params p, int t, int 
 }
 
 // Replays the early-stop rule over the stage sums, writes alpha and the report.
-__global__ void finalize_kernel(Params p, float* out_alpha, soar_result* res) {
-  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+__global__ void __launch_bounds__(128) finalize_kernel(Params p, float* out_alpha, soar_result* res) {
+  __shared__ double s_num[SOAR_MAX_ITERS + 1], s_den[SOAR_MAX_ITERS + 1], s_sse[SOAR_MAX_ITERS + 1];
+  __shared__ double s_ta[SOAR_MAX_ITERS + 1];
+  __shared__ int s_iters;
   const Ws* ws = p.ws;
   const unsigned int amax_bits = ws->amax_bits;
   const int st = status_from_amax(amax_bits);
-  float alpha = (st & SOAR_STATUS_ZERO_TENSOR) ? 1.0f : __fdiv_rn(bits_to_mag(amax_bits), 2688.0f);
-  int iters = 0;
-  double ta[SOAR_MAX_ITERS + 1], ts[SOAR_MAX_ITERS + 1];
-  ta[0] = static_cast<double>(alpha);
-  ts[0] = (st == 0) ? stage_sse(ws, 0) : 0.0;
-  if (st == 0 && ws->error == 0) {
-    double prev = ts[0];
-    for (int i = 0; i < p.max_iters; ++i) {
-      if (ws->den[i] > 0.0) alpha = static_cast<float>(ws->num[i] / ws->den[i]);
-      const double cur = stage_sse(ws, i + 1);
-      iters = i + 1;
-      ta[iters] = static_cast<double>(alpha);
-      ts[iters] = cur;
-      if (stops_after(prev, cur, p.early_stop_rel)) break;
-      prev = cur;
+  for (int i = threadIdx.x; i <= SOAR_MAX_ITERS; i += blockDim.x) {
+    const bool used = i <= p.max_iters;
+    s_num[i] = used ? ws->num[i] : 0.0;
+    s_den[i] = used ? ws->den[i] : 0.0;
+    s_sse[i] = (used && st == 0) ? stage_sse(ws, i) : 0.0;
+    s_ta[i] = 0.0;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float alpha = (st & SOAR_STATUS_ZERO_TENSOR) ? 1.0f : __fdiv_rn(bits_to_mag(amax_bits), 2688.0f);
+    int iters = 0;
+    s_ta[0] = static_cast<double>(alpha);
+    if (st == 0 && ws->error == 0) {
+      double prev = s_sse[0];
+      for (int i = 0; i < p.max_iters; ++i) {
+        if (s_den[i] > 0.0) alpha = static_cast<float>(s_num[i] / s_den[i]);
+        const double cur = s_sse[i + 1];
+        iters = i + 1;
+        s_ta[iters] = static_cast<double>(alpha);
+        if (stops_after(prev, cur, p.early_stop_rel)) break;
+        prev = cur;
+      }
+    }
+    s_iters = iters;
+    *out_alpha = alpha;
+    if (res != nullptr) {
+      res->status = st | (ws->error ? SOAR_STATUS_INTERNAL : 0);
+      res->iters_run = iters;
+      res->alpha = alpha;
+      res->amax = bits_to_mag(amax_bits);
+      res->sse = s_sse[iters];
+      res->sse_init = s_sse[0];
+      res->sumsq = (st & SOAR_STATUS_ZERO_TENSOR) ? 0.0 : ws->sumsq;
+      res->zero_blocks = static_cast<int64_t>(ws->zero_blocks);
+      res->wide_candidates = static_cast<int64_t>(ws->wide);
     }
   }
-  *out_alpha = alpha;
+  __syncthreads();
   if (res != nullptr) {
-    res->status = st | (ws->error ? SOAR_STATUS_INTERNAL : 0);
-    res->iters_run = iters;
-    res->alpha = alpha;
-    res->amax = bits_to_mag(amax_bits);
-    res->sse = ts[iters];
-    res->sse_init = ts[0];
-    res->sumsq = ws->sumsq;
-    res->zero_blocks = static_cast<int64_t>(ws->zero_blocks);
-    res->wide_candidates = static_cast<int64_t>(ws->wide);
-    for (int i = 0; i <= SOAR_MAX_ITERS; ++i) {
-      res->trace_alpha[i] = (i <= iters) ? ta[i] : 0.0;
-      res->trace_sse[i] = (i <= iters) ? ts[i] : 0.0;
+    const int iters = s_iters;
+    for (int i = threadIdx.x; i <= SOAR_MAX_ITERS; i += blockDim.x) {
+      res->trace_alpha[i] = (i <= iters) ? s_ta[i] : 0.0;
+      res->trace_sse[i] = (i <= iters) ? s_sse[i] : 0.0;
     }
   }
 }
@@ -927,18 +980,22 @@ int soar_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, co
     init_kernel<<<persistent_grid(init_kernel, p.nblk, kThreads), kThreads, 0, st>>>(p, reverse,
                                                                                      cfg->max_iters == 0 ? 1 : 0);
   }
-  const unsigned int g_it = persistent_grid(iterate_kernel, p.nblk, kThreads);
+  const bool single = cfg->n_beta == 1 && cfg->n_dq <= 2;
+  const unsigned int g_it = single ? persistent_grid(iterate_kernel<true>, p.nblk, kThreads)
+                                   : persistent_grid(iterate_kernel<false>, p.nblk, kThreads);
   const bool may_stop = cfg->early_stop_rel > 0.0f;
   for (int t = 0; t < cfg->max_iters; ++t) {
     reverse ^= 1;
     // with the early stop on, any iteration may turn out to be the last one
-    const int emit = (may_stop || t == cfg->max_iters - 1) ? 1 : 0;
+    const int last = (t == cfg->max_iters - 1) ? 1 : 0;
+    const int emit = (may_stop || last) ? 1 : 0;
     ScopedLaunch sl(K_ITERATE, st);
-    iterate_kernel<<<g_it, kThreads, 0, st>>>(p, t, reverse, emit);
+    if (single) iterate_kernel<true><<<g_it, kThreads, 0, st>>>(p, t, reverse, emit, !last);
+    else iterate_kernel<false><<<g_it, kThreads, 0, st>>>(p, t, reverse, emit, !last);
   }
   {
     ScopedLaunch sl(K_FINALIZE, st);
-    finalize_kernel<<<1, 32, 0, st>>>(p, out_global_fp32, out_result);
+    finalize_kernel<<<1, 128, 0, st>>>(p, out_global_fp32, out_result);
   }
   if (want_sw) {
     const unsigned int rt = static_cast<unsigned int>((rows + 127) / 128);
