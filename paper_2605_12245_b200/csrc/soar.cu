@@ -178,12 +178,28 @@ struct __align__(128) Ring {
   int fail;
 };
 
+// The same ring with, per stage, the tile's 8-byte block states next to its weights.
+struct __align__(128) RingWithState {
+  unsigned char tile[kStages][kTileBytes];
+  unsigned char state[kStages][kThreads * 8];
+  unsigned long long full[kStages];
+  int fail;
+};
+
 // Thread 0: start the copies of tile `tile` into stage `s` (one copy when rows are
 // contiguous, else one per row segment) and arm the stage's barrier with the byte count.
-__device__ __forceinline__ void ring_issue(Ring& ring, const Params& p, unsigned int tile, int s) {
+template <typename R>
+__device__ __forceinline__ void ring_issue(R& ring, const Params& p, unsigned int tile, int s) {
   const unsigned int b0 = tile * kThreads;
   unsigned int nb = min(static_cast<unsigned int>(kThreads), p.nblk - b0);
-  mbar_expect_tx(&ring.full[s], nb * 32u);
+  if constexpr (sizeof(R) == sizeof(RingWithState)) {
+    // the state array is padded to 256 bytes, so rounding the copy up to 16 stays inside it
+    const unsigned int sbytes = (nb * 8u + 15u) & ~15u;
+    mbar_expect_tx(&ring.full[s], nb * 32u + sbytes);
+    bulk_load(ring.state[s], p.state + b0, sbytes, &ring.full[s]);
+  } else {
+    mbar_expect_tx(&ring.full[s], nb * 32u);
+  }
   unsigned char* dst = ring.tile[s];
   if (p.contiguous) {
     bulk_load(dst, p.W + static_cast<size_t>(b0) * 16, nb * 32u, &ring.full[s]);
@@ -212,7 +228,8 @@ __device__ __forceinline__ unsigned int tiles_of_cta(const Params& p) {
   return blockIdx.x < p.ntiles ? (p.ntiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
 }
 
-__device__ __forceinline__ void ring_start(Ring& ring, const Params& p, int reverse) {
+template <typename R>
+__device__ __forceinline__ void ring_start(R& ring, const Params& p, int reverse) {
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) mbar_init(&ring.full[s], 1);
     ring.fail = 0;
@@ -229,8 +246,9 @@ __device__ __forceinline__ void ring_start(Ring& ring, const Params& p, int reve
 // Fetches this thread's 32 bytes of the CTA's n-th tile into v0, v1; then (thread 0) refills
 // the stage with the tile kStages ahead.  Returns false, for every thread of the CTA alike,
 // when a wait gave up; the caller must then leave its tile loop.
-__device__ __forceinline__ bool ring_next(Ring& ring, const Params& p, unsigned int n, unsigned int ntile_cta,
-                                          int reverse, uint4& v0, uint4& v1) {
+template <typename R>
+__device__ __forceinline__ bool ring_next(R& ring, const Params& p, unsigned int n, unsigned int ntile_cta,
+                                          int reverse, uint4& v0, uint4& v1, uint2* st = nullptr) {
   const int s = static_cast<int>(n % kStages);
   const bool ok = mbar_wait(&ring.full[s], (n / kStages) & 1u);
   if (!ok) ring.fail = 1;
@@ -238,6 +256,8 @@ __device__ __forceinline__ bool ring_next(Ring& ring, const Params& p, unsigned 
     const uint4* src = reinterpret_cast<const uint4*>(ring.tile[s] + threadIdx.x * 32);
     v0 = src[0];
     v1 = src[1];
+    if constexpr (sizeof(R) == sizeof(RingWithState))
+      *st = reinterpret_cast<const uint2*>(ring.state[s])[threadIdx.x];
   }
   __syncthreads();
   if (*static_cast<volatile int*>(&ring.fail)) return false;
@@ -247,7 +267,8 @@ __device__ __forceinline__ bool ring_next(Ring& ring, const Params& p, unsigned 
 
 // After a failed wait: record it, then give copies still in flight a bounded chance to land
 // before the CTA's shared memory is released.
-__device__ __forceinline__ void ring_abort(Ring& ring, const Params& p, unsigned int n, unsigned int ntile_cta) {
+template <typename R>
+__device__ __forceinline__ void ring_abort(R& ring, const Params& p, unsigned int n, unsigned int ntile_cta) {
   if (threadIdx.x != 0) return;
   atomicOr(&p.ws->error, 1u);
   for (unsigned int m = n; m < ntile_cta && m < n + kStages; ++m)
@@ -405,11 +426,25 @@ __device__ __forceinline__ bool stops_after(double prev, double cur, float eps) 
 
 // ------------------------------------------------------------------ kernels
 
-// bf16 magnitude bits (15 bits) -> the binary64 with the same value; zero and bf16
-// subnormals (below 1.2e-38) map to zero.
-__device__ __forceinline__ double bf16_mag_to_double(unsigned int h15) {
-  const unsigned int hi = (h15 & 0x7F80u) ? (h15 << 13) + 0x38000000u : 0u;
-  return __hiloint2double(static_cast<int>(hi), 0);
+// Sum of squares of a block's sixteen bf16 values, binary64, scaled by 2^-256: a bf16
+// magnitude h (8 exponent bits e, 7 fraction bits) placed at bits 27..13 of a binary64 high
+// word and OR-ed with exponent 768 is the value times 2^-128, with no carry to handle.
+// Exact for normal bf16 values; kExact also maps zeros and bf16 subnormals (below 1.2e-38)
+// to zero, which the plain form would count as 2^-127 each.
+template <bool kExact>
+__device__ __forceinline__ void sumsq_block(const unsigned int (&u)[8], double& s0, double& s1) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    unsigned int lo = ((u[i] << 13) & 0x0FFFE000u) | 0x30000000u;
+    unsigned int hi = ((u[i] >> 3) & 0x0FFFE000u) | 0x30000000u;
+    if (kExact) {
+      if ((u[i] & 0x00007F80u) == 0) lo = 0;
+      if ((u[i] & 0x7F800000u) == 0) hi = 0;
+    }
+    const double dl = __hiloint2double(static_cast<int>(lo), 0), dh = __hiloint2double(static_cast<int>(hi), 0);
+    s0 = fma(dl, dl, s0);
+    s1 = fma(dh, dh, s1);
+  }
 }
 
 // Eq. 1's tensor maximum, plus sum W^2 (binary64) for the error report.
@@ -426,20 +461,23 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(Params p, int reverse) {
     const unsigned int b = tile_of(p, n, reverse) * kThreads + threadIdx.x;
     if (b >= p.nblk) continue;
     const unsigned int u[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+    unsigned int bmx = 0, bmn = 0x7FFF7FFFu;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const unsigned int m = u[i] & 0x7FFF7FFFu;
-      mx = __vmaxu2(mx, m);
-      const double lo = bf16_mag_to_double(m & 0xFFFFu), hi = bf16_mag_to_double(m >> 16);
-      sq[0] = fma(lo, lo, sq[0]);
-      sq[1] = fma(hi, hi, sq[1]);
+      bmx = __vmaxu2(bmx, m);
+      bmn = __vminu2(bmn, m);
     }
+    mx = __vmaxu2(mx, bmx);
+    // a magnitude below 0x0080 has a zero exponent field: zero or subnormal
+    if (min(bmn & 0xFFFFu, bmn >> 16) >= 0x80u) sumsq_block<false>(u, sq[0], sq[1]);
+    else sumsq_block<true>(u, sq[0], sq[1]);
   }
   if (n < ntc) ring_abort(ring, p, n, ntc);
   mx = max(mx & 0xFFFFu, mx >> 16);
   mx = __reduce_max_sync(0xFFFFFFFFu, mx);
   if ((threadIdx.x & 31) == 0 && mx) atomicMax(&p.ws->amax_bits, mx);
-  double acc[1] = {sq[0] + sq[1]};
+  double acc[1] = {(sq[0] + sq[1]) * 0x1p256};   // undo the 2^-128 scaling of the values
   double* const dst[1] = {&p.ws->sumsq};
   cta_accumulate<1>(acc, dst);
 }
@@ -563,7 +601,7 @@ __device__ __forceinline__ int clip_code(int d) { return max(1, min(0x7E, d)); }
 template <bool kSingle>
 __global__ void __launch_bounds__(kThreads, kSingle ? 3 : 2)
 iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
-  __shared__ Ring ring;
+  __shared__ RingWithState ring;
   __shared__ float s_beta[kSingle ? 1 : SOAR_MAX_BETA];
   __shared__ float s_alpha;
   __shared__ int s_run;
@@ -591,10 +629,10 @@ iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
   unsigned int n = 0;
   for (; n < ntc; ++n) {
     uint4 v0, v1;
-    if (!ring_next(ring, p, n, ntc, reverse, v0, v1)) break;
+    uint2 st;
+    if (!ring_next(ring, p, n, ntc, reverse, v0, v1, &st)) break;
     const unsigned int b = tile_of(p, n, reverse) * kThreads + threadIdx.x;
     if (b >= p.nblk) continue;
-    const uint2 st = p.state[b];
     if ((st.y >> 16) == 0) continue;                // all-zero block: nothing to optimise
     Block blk;
     unpack_block(v0, v1, blk);
