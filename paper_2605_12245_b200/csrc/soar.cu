@@ -9,11 +9,13 @@
 //   finalize_kernel  early-stop bookkeeping (Sec. 4.1), alpha and the report
 //   swizzle_kernel   optional 128x4-tiled copy of the block scales
 //
-// Data movement.  The three passes over W are persistent kernels: each CTA walks tiles of
-// 256 blocks (8 KB of bf16) that one thread fetches with bulk asynchronous copies
-// (cp.async.bulk, completion on an mbarrier) into a four-stage shared-memory ring, so the
-// copies of the next tiles are in flight while the 256 threads work on the current one
-// from registers.  One thread owns one 16-element block.
+// Data movement.  The three passes over W are persistent, warp-specialised kernels: each CTA
+// walks tiles of 256 blocks (8 KB of bf16).  One thread of a producer warp fetches them with
+// bulk asynchronous copies (cp.async.bulk, completion on a "full" mbarrier) into a
+// four-stage shared-memory ring; 256 consumer threads, one per 16-element block, pull their
+// 32 bytes into registers, hand the stage back through an "empty" mbarrier and work from
+// registers, so no CTA-wide barrier sits in the tile loop and the copies of the next tiles
+// are always in flight.
 //
 // State between iterations is 8 bytes per block in the workspace: the winner's
 // A = sum |W| m (binary32, exact), 4B = sum (2m)^2 and its E4M3 scale code.  That is all
@@ -37,9 +39,10 @@
 
 namespace {
 
-constexpr int kThreads = 256;                  // threads per CTA = blocks per tile
+constexpr int kTile = 256;                     // blocks per tile = consumer threads per CTA
+constexpr int kThreads = kTile + 32;           // plus one producer warp that issues the copies
 constexpr int kStages = 4;                     // depth of the shared-memory ring
-constexpr int kTileBytes = kThreads * 32;      // 16 bf16 per block
+constexpr int kTileBytes = kTile * 32;         // 16 bf16 per block
 constexpr size_t kWsFixedBytes = 2048;
 constexpr unsigned int kWaitLimit = 1u << 22;  // mbarrier polls before a wait gives up
 
@@ -146,6 +149,10 @@ __device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned
                : "memory");
 }
 
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
 // One bulk copy global -> shared; src and dst 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned int bytes,
                                           unsigned long long* bar) {
@@ -174,15 +181,17 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned int 
 
 struct __align__(128) Ring {
   unsigned char tile[kStages][kTileBytes];
-  unsigned long long full[kStages];
+  unsigned long long full[kStages];    // producer -> consumers: the stage's bytes have landed
+  unsigned long long empty[kStages];   // consumers -> producer: every consumer has read the stage
   int fail;
 };
 
 // The same ring with, per stage, the tile's 8-byte block states next to its weights.
 struct __align__(128) RingWithState {
   unsigned char tile[kStages][kTileBytes];
-  unsigned char state[kStages][kThreads * 8];
+  unsigned char state[kStages][kTile * 8];
   unsigned long long full[kStages];
+  unsigned long long empty[kStages];
   int fail;
 };
 
@@ -190,8 +199,8 @@ struct __align__(128) RingWithState {
 // contiguous, else one per row segment) and arm the stage's barrier with the byte count.
 template <typename R>
 __device__ __forceinline__ void ring_issue(R& ring, const Params& p, unsigned int tile, int s) {
-  const unsigned int b0 = tile * kThreads;
-  unsigned int nb = min(static_cast<unsigned int>(kThreads), p.nblk - b0);
+  const unsigned int b0 = tile * kTile;
+  unsigned int nb = min(static_cast<unsigned int>(kTile), p.nblk - b0);
   if constexpr (sizeof(R) == sizeof(RingWithState)) {
     // the state array is padded to 256 bytes, so rounding the copy up to 16 stays inside it
     const unsigned int sbytes = (nb * 8u + 15u) & ~15u;
@@ -228,51 +237,61 @@ __device__ __forceinline__ unsigned int tiles_of_cta(const Params& p) {
   return blockIdx.x < p.ntiles ? (p.ntiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
 }
 
+// All threads: barriers ready before anyone uses them.
 template <typename R>
-__device__ __forceinline__ void ring_start(R& ring, const Params& p, int reverse) {
+__device__ __forceinline__ void ring_init(R& ring) {
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) mbar_init(&ring.full[s], 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&ring.full[s], 1);
+      mbar_init(&ring.empty[s], kTile);
+    }
     ring.fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
-    const unsigned int n = tiles_of_cta(p);
-    for (unsigned int i = 0; i < static_cast<unsigned int>(kStages) && i < n; ++i)
-      ring_issue(ring, p, tile_of(p, i, reverse), static_cast<int>(i));
+}
+
+__device__ __forceinline__ bool is_producer_warp() { return threadIdx.x >= kTile; }
+
+// Producer (one thread): walks the CTA's tile sequence, refilling a stage as soon as every
+// consumer has handed it back.  A wait that gives up records the failure, lets copies still
+// in flight land (bounded) and ends the sequence; the consumers then give up on their own.
+template <typename R>
+__device__ __forceinline__ void ring_produce(R& ring, const Params& p, int reverse) {
+  const unsigned int ntc = tiles_of_cta(p);
+  unsigned int n = 0;
+  bool ok = true;
+  for (; n < ntc; ++n) {
+    const int s = static_cast<int>(n % kStages);
+    if (n >= static_cast<unsigned int>(kStages)) ok = mbar_wait(&ring.empty[s], (n / kStages - 1) & 1u);
+    if (!ok || *static_cast<volatile int*>(&ring.fail)) break;
+    ring_issue(ring, p, tile_of(p, n, reverse), s);
+  }
+  if (n < ntc) {
+    *static_cast<volatile int*>(&ring.fail) = 1;
+    atomicOr(&p.ws->error, 1u);
+    for (unsigned int m = (n > static_cast<unsigned int>(kStages) ? n - kStages : 0); m < n; ++m)
+      (void)mbar_wait(&ring.full[m % kStages], (m / kStages) & 1u);
   }
 }
 
-// Fetches this thread's 32 bytes of the CTA's n-th tile into v0, v1; then (thread 0) refills
-// the stage with the tile kStages ahead.  Returns false, for every thread of the CTA alike,
-// when a wait gave up; the caller must then leave its tile loop.
+// Consumer: this thread's 32 bytes (and block state) of the CTA's n-th tile, then the stage
+// is handed back.  Returns false when the wait gave up; the caller leaves its tile loop.
 template <typename R>
-__device__ __forceinline__ bool ring_next(R& ring, const Params& p, unsigned int n, unsigned int ntile_cta,
-                                          int reverse, uint4& v0, uint4& v1, uint2* st = nullptr) {
+__device__ __forceinline__ bool ring_consume(R& ring, const Params& p, unsigned int n, uint4& v0, uint4& v1,
+                                             uint2* st = nullptr) {
   const int s = static_cast<int>(n % kStages);
-  const bool ok = mbar_wait(&ring.full[s], (n / kStages) & 1u);
-  if (!ok) ring.fail = 1;
-  if (ok) {
-    const uint4* src = reinterpret_cast<const uint4*>(ring.tile[s] + threadIdx.x * 32);
-    v0 = src[0];
-    v1 = src[1];
-    if constexpr (sizeof(R) == sizeof(RingWithState))
-      *st = reinterpret_cast<const uint2*>(ring.state[s])[threadIdx.x];
+  if (!mbar_wait(&ring.full[s], (n / kStages) & 1u)) {
+    *static_cast<volatile int*>(&ring.fail) = 1;
+    atomicOr(&p.ws->error, 1u);
+    return false;
   }
-  __syncthreads();
-  if (*static_cast<volatile int*>(&ring.fail)) return false;
-  if (threadIdx.x == 0 && n + kStages < ntile_cta) ring_issue(ring, p, tile_of(p, n + kStages, reverse), s);
+  const uint4* src = reinterpret_cast<const uint4*>(ring.tile[s] + threadIdx.x * 32);
+  v0 = src[0];
+  v1 = src[1];
+  if constexpr (sizeof(R) == sizeof(RingWithState)) *st = reinterpret_cast<const uint2*>(ring.state[s])[threadIdx.x];
+  mbar_arrive(&ring.empty[s]);
   return true;
-}
-
-// After a failed wait: record it, then give copies still in flight a bounded chance to land
-// before the CTA's shared memory is released.
-template <typename R>
-__device__ __forceinline__ void ring_abort(R& ring, const Params& p, unsigned int n, unsigned int ntile_cta) {
-  if (threadIdx.x != 0) return;
-  atomicOr(&p.ws->error, 1u);
-  for (unsigned int m = n; m < ntile_cta && m < n + kStages; ++m)
-    (void)mbar_wait(&ring.full[m % kStages], (m / kStages) & 1u);
 }
 
 // ------------------------------------------------------------------ block helpers
@@ -391,6 +410,7 @@ __device__ __forceinline__ double warp_sum(double v) {
 template <int N>
 __device__ __forceinline__ void cta_accumulate(double (&v)[N], double* const (&dst)[N]) {
   __shared__ double red[N][kThreads / 32];
+  const int nwarp = blockDim.x >> 5;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
 #pragma unroll
   for (int i = 0; i < N; ++i) {
@@ -402,7 +422,7 @@ __device__ __forceinline__ void cta_accumulate(double (&v)[N], double* const (&d
 #pragma unroll
     for (int i = 0; i < N; ++i) {
       double s = 0.0;
-      for (int w = 0; w < kThreads / 32; ++w) s += red[i][w];
+      for (int w = 0; w < nwarp; ++w) s += red[i][w];
       if (dst[i] != nullptr) atomicAdd(dst[i], s);
     }
   }
@@ -450,15 +470,15 @@ __device__ __forceinline__ void sumsq_block(const unsigned int (&u)[8], double& 
 // Eq. 1's tensor maximum, plus sum W^2 (binary64) for the error report.
 __global__ void __launch_bounds__(kThreads) amax_kernel(Params p, int reverse) {
   __shared__ Ring ring;
-  ring_start(ring, p, reverse);
-  const unsigned int ntc = tiles_of_cta(p);
+  ring_init(ring);
+  const unsigned int ntc = is_producer_warp() ? 0u : tiles_of_cta(p);
+  if (threadIdx.x == kTile) ring_produce(ring, p, reverse);
   unsigned int mx = 0;
   double sq[2] = {0.0, 0.0};
-  unsigned int n = 0;
-  for (; n < ntc; ++n) {
+  for (unsigned int n = 0; n < ntc; ++n) {
     uint4 v0, v1;
-    if (!ring_next(ring, p, n, ntc, reverse, v0, v1)) break;
-    const unsigned int b = tile_of(p, n, reverse) * kThreads + threadIdx.x;
+    if (!ring_consume(ring, p, n, v0, v1)) break;
+    const unsigned int b = tile_of(p, n, reverse) * kTile + threadIdx.x;
     if (b >= p.nblk) continue;
     const unsigned int u[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
     unsigned int bmx = 0, bmn = 0x7FFF7FFFu;
@@ -473,7 +493,6 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(Params p, int reverse) {
     if (min(bmn & 0xFFFFu, bmn >> 16) >= 0x80u) sumsq_block<false>(u, sq[0], sq[1]);
     else sumsq_block<true>(u, sq[0], sq[1]);
   }
-  if (n < ntc) ring_abort(ring, p, n, ntc);
   mx = max(mx & 0xFFFFu, mx >> 16);
   mx = __reduce_max_sync(0xFFFFFFFFu, mx);
   if ((threadIdx.x & 31) == 0 && mx) atomicMax(&p.ws->amax_bits, mx);
@@ -490,18 +509,18 @@ __global__ void __launch_bounds__(kThreads) init_kernel(Params p, int reverse, i
   const unsigned int amax_bits = p.ws->amax_bits;
   const int st = status_from_amax(amax_bits);
   if (st & (SOAR_STATUS_NONFINITE | SOAR_STATUS_RANGE)) return;
-  ring_start(ring, p, reverse);
-  const unsigned int ntc = tiles_of_cta(p);
+  ring_init(ring);
+  const unsigned int ntc = is_producer_warp() ? 0u : tiles_of_cta(p);
+  if (threadIdx.x == kTile) ring_produce(ring, p, reverse);
   const float alpha = (st & SOAR_STATUS_ZERO_TENSOR) ? 1.0f : __fdiv_rn(bits_to_mag(amax_bits), 2688.0f);
   const float six_alpha = __fmul_rn(alpha, 6.0f);
   const double alpha_d = static_cast<double>(alpha);
   double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum
   unsigned int zeros = 0, wide = 0;
-  unsigned int n = 0;
-  for (; n < ntc; ++n) {
+  for (unsigned int n = 0; n < ntc; ++n) {
     uint4 v0, v1;
-    if (!ring_next(ring, p, n, ntc, reverse, v0, v1)) break;
-    const unsigned int b = tile_of(p, n, reverse) * kThreads + threadIdx.x;
+    if (!ring_consume(ring, p, n, v0, v1)) break;
+    const unsigned int b = tile_of(p, n, reverse) * kTile + threadIdx.x;
     if (b >= p.nblk) continue;
     Block blk;
     unpack_block(v0, v1, blk);
@@ -537,7 +556,6 @@ __global__ void __launch_bounds__(kThreads) init_kernel(Params p, int reverse, i
     acc[1] = fma(B * vd, vd, acc[1]);
     acc[2] += sd * fma(sd, B, -2.0 * A);
   }
-  if (n < ntc) ring_abort(ring, p, n, ntc);
   double* const dst[3] = {&p.ws->num[0], &p.ws->den[0], &p.ws->gsum[0]};
   cta_accumulate<3>(acc, dst);
   zeros = __reduce_add_sync(0xFFFFFFFFu, zeros);
@@ -618,20 +636,20 @@ iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
   }
   __syncthreads();
   if (!s_run) return;
-  ring_start(ring, p, reverse);
-  const unsigned int ntc = tiles_of_cta(p);
+  ring_init(ring);
+  const unsigned int ntc = is_producer_warp() ? 0u : tiles_of_cta(p);
+  if (threadIdx.x == kTile) ring_produce(ring, p, reverse);
   const float alpha = s_alpha;
   const double alpha_d = static_cast<double>(alpha);
   const int n_dq = p.n_dq, n_beta = p.n_beta;
 
   double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum of stage t+1
   unsigned int wide = 0;
-  unsigned int n = 0;
-  for (; n < ntc; ++n) {
+  for (unsigned int n = 0; n < ntc; ++n) {
     uint4 v0, v1;
     uint2 st;
-    if (!ring_next(ring, p, n, ntc, reverse, v0, v1, &st)) break;
-    const unsigned int b = tile_of(p, n, reverse) * kThreads + threadIdx.x;
+    if (!ring_consume(ring, p, n, v0, v1, &st)) break;
+    const unsigned int b = tile_of(p, n, reverse) * kTile + threadIdx.x;
     if (b >= p.nblk) continue;
     if ((st.y >> 16) == 0) continue;                // all-zero block: nothing to optimise
     Block blk;
@@ -704,7 +722,6 @@ iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
     acc[1] = fma(bestB * vd, vd, acc[1]);
     acc[2] += best;
   }
-  if (n < ntc) ring_abort(ring, p, n, ntc);
   double* const dst[3] = {&p.ws->num[t + 1], &p.ws->den[t + 1], &p.ws->gsum[t + 1]};
   cta_accumulate<3>(acc, dst);
   wide = __reduce_add_sync(0xFFFFFFFFu, wide);
@@ -792,12 +809,12 @@ __global__ void __launch_bounds__(256) swizzle_kernel(const uint8_t* lin, uint8_
 }
 
 // Eq. 3-4 on stored outputs.
-__global__ void __launch_bounds__(kThreads) dequant_error_kernel(Params p, const uint8_t* scales, int swizzled,
+__global__ void __launch_bounds__(kTile) dequant_error_kernel(Params p, const uint8_t* scales, int swizzled,
                                                                  unsigned int col_tiles, const float* alpha_ptr,
                                                                  double* out_sse, double* out_sumsq) {
   const double alpha = static_cast<double>(*alpha_ptr);
   double acc[2] = {0.0, 0.0};
-  for (unsigned int b = blockIdx.x * kThreads + threadIdx.x; b < p.nblk; b += gridDim.x * kThreads) {
+  for (unsigned int b = blockIdx.x * kTile + threadIdx.x; b < p.nblk; b += gridDim.x * kTile) {
     const unsigned int row = b / p.nbc, cb = b - row * p.nbc;
     const uint16_t* src = p.W + static_cast<long long>(row) * p.ld + static_cast<long long>(cb) * 16;
     const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(src));
@@ -881,7 +898,7 @@ unsigned int persistent_grid(K kernel, unsigned int nblk, int threads) {
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, 0) != cudaSuccess || per_sm <= 0)
     per_sm = 2;
   const unsigned long long cap = static_cast<unsigned long long>(sm_count()) * per_sm;
-  const unsigned long long need = (static_cast<unsigned long long>(nblk) + threads - 1) / threads;
+  const unsigned long long need = (static_cast<unsigned long long>(nblk) + kTile - 1) / kTile;
   return static_cast<unsigned int>(need < cap ? (need ? need : 1) : cap);
 }
 
@@ -987,7 +1004,7 @@ int soar_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, co
   p.ld = ld;
   p.nbc = static_cast<unsigned int>(cols / 16);
   p.nblk = static_cast<unsigned int>(rows * (cols / 16));
-  p.ntiles = (p.nblk + kThreads - 1) / kThreads;
+  p.ntiles = (p.nblk + kTile - 1) / kTile;
   p.contiguous = (ld == cols) ? 1 : 0;
   {
     uint8_t* next = static_cast<uint8_t*>(workspace) + kWsFixedBytes;
@@ -1108,7 +1125,7 @@ int soar_dequant_error(const void* W_bf16, int64_t rows, int64_t cols, int64_t l
   if (cudaMemsetAsync(out_sumsq, 0, sizeof(double), st) != cudaSuccess) return SOAR_ERR_CUDA;
   {
     ScopedLaunch sl(K_DEQUANT_ERROR, st);
-    dequant_error_kernel<<<persistent_grid(dequant_error_kernel, p.nblk, kThreads), kThreads, 0, st>>>(
+    dequant_error_kernel<<<persistent_grid(dequant_error_kernel, p.nblk, kTile), kTile, 0, st>>>(
         p, static_cast<const uint8_t*>(e4m3_scales), scale_layout == SOAR_SCALES_SWIZZLED ? 1 : 0,
         (p.nbc + 3) / 4, global_fp32, out_sse, out_sumsq);
   }
