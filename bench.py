@@ -247,7 +247,10 @@ def run_ours(args):
 
     sampler = ClockSampler(local)
     sampler.start()
-    ms, trace = timed(step, args.steps, args.warmup)
+    # headline: K steps with nothing between the kernels; then the same K steps again with an
+    # event pair around every kernel (which costs a few microseconds per launch) for the shares
+    ms, _ = timed(step, args.steps, args.warmup, trace=False)
+    traced_ms, trace = timed(step, args.steps, 0, trace=True)
     clocks = sampler.stop()
     results = [o.read_result() for o in outs]
     iters = [r.iters_run for r in results]
@@ -288,7 +291,8 @@ def run_ours(args):
     extra = {}
     if args.preset == "paper" and not args.no_single_pass:
         sp = preset_cfg(api, "single_pass")
-        sp_ms, sp_tr = timed(lambda: step(sp), max(args.steps, 5), 3)
+        sp_ms, _ = timed(lambda: step(sp), max(args.steps, 5), 3, trace=False)
+        _, sp_tr = timed(lambda: step(sp), max(args.steps, 5), 0, trace=True)
         sp_bytes = elements * call_bytes_per_elem(sp, sp.max_iters)
         gbs = sp_bytes / (sp_ms * 1e-3) / 1e9
         extra["single_pass"] = dict(
@@ -368,7 +372,7 @@ def run_ours(args):
                         parallelism=f"replicated workload x{world}, no collective"),
             elements_per_s=world * elements / (ms * 1e-3),
             hbm_frac_end_to_end_of_measured=value / peaks["hbm_gbs"],
-            roofline=roofline, kernels=kernels, cpu_baseline=cpu, e2e=e2e, gpu_launches=launches,
+            traced_ms_per_step=traced_ms, roofline=roofline, kernels=kernels, cpu_baseline=cpu, e2e=e2e, gpu_launches=launches,
             clocks=clocks, **extra)
         print(json.dumps(line), flush=True)
     if world > 1:
