@@ -60,8 +60,15 @@ def pick_workload(name: str):
     raise SystemExit(f"unknown workload {name}")
 
 
-def preset_cfg(api, preset: str, **over):
+def preset_cfg(api, preset: str, args=None, **over):
+    """The preset's settings; ``--pairs K`` and ``--iters T`` override the candidate grid and the
+    iteration count (K pairs per block = n_beta x n_dq with n_dq = min(2, K); no early stop)."""
     base = api.PRESET_PAPER if preset == "paper" else api.PRESET_SINGLE_PASS
+    if args is not None and args.pairs:
+        n_dq = min(2, args.pairs)
+        over.update(n_dq=n_dq, n_beta=max(1, args.pairs // n_dq))
+    if args is not None and args.iters is not None:
+        over.update(max_iters=args.iters, early_stop_rel=0.0)
     return api.soar_default_cfg(base, **over)
 
 
@@ -157,7 +164,7 @@ def run_reference(args):
     from oracle import soar_ref as R
     from paper_2605_12245_b200 import api
     wl = pick_workload(args.workload)
-    cfg = preset_cfg(api, args.preset)
+    cfg = preset_cfg(api, args.preset, args)
     rcfg = ref_cfg_of(R, cfg)
     spec = wl.tensors[0]
     rows = min(spec.rows, max(1, args.ref_rows))
@@ -201,7 +208,7 @@ def run_ours(args):
     api.lib()
     peaks = load_peaks()
     wl = pick_workload(args.workload)
-    cfg = preset_cfg(api, args.preset)
+    cfg = preset_cfg(api, args.preset, args)
 
     # ---- inputs: generated on the host (seeded), resident in HBM before timing
     host_w, dev_w, outs = [], [], []
@@ -389,6 +396,8 @@ def main():
     ap.add_argument("--preset", default="paper", choices=["paper", "single_pass"])
     ap.add_argument("--cpu-rows", type=int, default=256, help="rows of tensor 0 the CPU baseline quantizes")
     ap.add_argument("--ref-rows", type=int, default=128, help="rows per step of the reference arm")
+    ap.add_argument("--pairs", type=int, default=0, help="candidate pairs per block (overrides the preset's grid)")
+    ap.add_argument("--iters", type=int, default=None, help="iterations T, early stop off (overrides the preset)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-single-pass", action="store_true")

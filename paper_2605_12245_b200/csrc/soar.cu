@@ -281,7 +281,8 @@ template <typename R>
 __device__ __forceinline__ bool ring_consume(R& ring, const Params& p, unsigned int n, uint4& v0, uint4& v1,
                                              uint2* st = nullptr) {
   const int s = static_cast<int>(n % kStages);
-  if (!mbar_wait(&ring.full[s], (n / kStages) & 1u)) {
+  // the outcome is made the same for the whole warp: callers vote across the warp later
+  if (!__all_sync(0xFFFFFFFFu, mbar_wait(&ring.full[s], (n / kStages) & 1u))) {
     *static_cast<volatile int*>(&ring.fail) = 1;
     atomicOr(&p.ws->error, 1u);
     return false;
@@ -650,8 +651,7 @@ iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
     uint2 st;
     if (!ring_consume(ring, p, n, v0, v1, &st)) break;
     const unsigned int b = tile_of(p, n, reverse) * kTile + threadIdx.x;
-    if (b >= p.nblk) continue;
-    if ((st.y >> 16) == 0) continue;                // all-zero block: nothing to optimise
+    if (b >= p.nblk || (st.y >> 16) == 0) continue;   // past the end, or an all-zero block: nothing to optimise
     Block blk;
     unpack_block(v0, v1, blk);
     int d_lo, d_hi;
@@ -676,38 +676,57 @@ iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
         if (g1 < best) { best = g1; best_d = dc1; }
       }
     } else {
-      // Eq. 8 over beta ascending, then scale code ascending; strict '<' keeps the first minimum.
+      // Eq. 8 over beta ascending, then scale code ascending; strict '<' keeps the first
+      // minimum.  Every candidate is scored in full, with no test for "same codes as the
+      // previous beta": under SIMT such a test only saves work when all 32 blocks of a warp
+      // pass it at once, and it costs instructions on every candidate.  The loop keeps just
+      // the best error and its (beta, code) index; the winner is re-made once at the end.
       best = __longlong_as_double(0x7FF0000000000000ll);
-      bestA = 0.0;
-      bestB = 0.0;
-      best0 = best1 = 0;
-      unsigned int prev0 = 0, prev1 = 0;
-      for (int k = 0; k < n_beta; ++k) {
-        const float r = recip_scale(alpha, __fmul_rn(center, s_beta[k]));
-        unsigned int c0, c1;
-        round_block(blk, r, c0, c1);
-        if (k > 0 && c0 == prev0 && c1 == prev1) continue;   // same codes as the previous beta: same errors
-        prev0 = c0;
-        prev1 = c1;
-        double A, B;
-        block_sums(blk, fx, r, c0, c1, A, B, wide);
-        const double A2 = -2.0 * A;
-        if (n_dq <= 2) {
-          const double g0 = sd0 * fma(sd0, B, A2);
-          if (g0 < best) { best = g0; bestA = A; bestB = B; best_d = dc0; best0 = c0; best1 = c1; }
-          if (n_dq == 2) {
-            const double g1 = sd1 * fma(sd1, B, A2);
-            if (g1 < best) { best = g1; bestA = A; bestB = B; best_d = dc1; best0 = c0; best1 = c1; }
+      int best_key = 0;
+      const int nd = d_hi - d_lo + 1;
+      // the reciprocal scale falls as beta grows, so the first candidate decides whether the
+      // exact integer sums hold for all of them
+      const bool all_narrow = fx.ok && __fmul_rn(blk.bmax, recip_scale(alpha, __fmul_rn(center, s_beta[0]))) <= 32.0f;
+      if (all_narrow && nd <= 2) {
+        // error minus sum W^2 = sd^2 B - 2 sd A = p * (4B) - q * afix  with  p = sd^2/4, q = 2 sd unit
+        const double p0 = 0.25 * sd0 * sd0, q0 = 2.0 * sd0 * fx.unit;
+        const double p1 = 0.25 * sd1 * sd1, q1 = 2.0 * sd1 * fx.unit;
+        for (int k = 0; k < n_beta; ++k) {
+          const float r = recip_scale(alpha, __fmul_rn(center, s_beta[k]));
+          unsigned int c0, c1, afix, b4;
+          round_block(blk, r, c0, c1);
+          code_sums(fx, c0, c1, afix, b4);
+          const double ad = uint_to_double(afix), bd = uint_to_double(b4);
+          const double g0 = fma(p0, bd, -(q0 * ad));
+          if (g0 < best) { best = g0; best_key = 2 * k; }
+          if (nd == 2) {
+            const double g1 = fma(p1, bd, -(q1 * ad));
+            if (g1 < best) { best = g1; best_key = 2 * k + 1; }
           }
-        } else {
-          for (int d = d_lo; d <= d_hi; ++d) {
-            const int dc = clip_code(d);
-            const double sd = alpha_d * static_cast<double>(e4m3_value(dc));
+        }
+      } else {
+        for (int k = 0; k < n_beta; ++k) {
+          const float r = recip_scale(alpha, __fmul_rn(center, s_beta[k]));
+          unsigned int c0, c1;
+          round_block(blk, r, c0, c1);
+          double A, B;
+          block_sums(blk, fx, r, c0, c1, A, B, wide);
+          const double A2 = -2.0 * A;
+          for (int d = 0; d < nd; ++d) {
+            const double sd = alpha_d * static_cast<double>(e4m3_value(clip_code(d_lo + d)));
             const double g = sd * fma(sd, B, A2);
-            if (g < best) { best = g; bestA = A; bestB = B; best_d = dc; best0 = c0; best1 = c1; }
+            if (g < best) { best = g; best_key = (nd <= 2 ? 2 : nd) * k + d; }
           }
         }
       }
+      // the winner, made again from its index
+      const int per = nd <= 2 ? 2 : nd;
+      const int bk = best_key / per;
+      best_d = clip_code(d_lo + (best_key - bk * per));
+      const float r = recip_scale(alpha, __fmul_rn(center, s_beta[bk]));
+      round_block(blk, r, best0, best1);
+      unsigned int unused = 0;
+      block_sums(blk, fx, r, best0, best1, bestA, bestB, unused);
     }
     // The winner: codes and scale out, sums kept for the next iteration's Eq. 6.
     if (emit) {
