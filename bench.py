@@ -308,6 +308,18 @@ def run_ours(args):
             frac_of_nominal_8000=gbs / 8000.0,
             kernels={k: dict(launches=v[0], ms_per_step=v[1] / max(args.steps, 5)) for k, v in sp_tr.items()})
 
+    # ---- the error check of Eq. 3-4 on the outputs just produced (its own entry point, not part of a step)
+    err_out = torch.empty(2, dtype=torch.float64, device="cuda")
+
+    def err_step():
+        for W, o in zip(dev_w, outs):
+            api.soar_dequant_error(W, o.packed, o.scales, o.alpha, stream=stream, out=err_out)
+
+    err_ms, _ = timed(err_step, max(args.steps, 5), 3, trace=False)
+    err_bytes = elements * kernel_bytes_per_elem("dequant_error_kernel", cfg)
+    extra["dequant_error"] = dict(ms_per_step=err_ms, achieved_gbs=err_bytes / (err_ms * 1e-3) / 1e9,
+                                  frac_of_measured_hbm=err_bytes / (err_ms * 1e-3) / 1e9 / peaks["hbm_gbs"])
+
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region
     import ctypes
     ctypes_sizeof_result = ctypes.sizeof(api.SoarResult)

@@ -269,7 +269,7 @@ __device__ __forceinline__ void ring_produce(R& ring, const Params& p, int rever
   }
   if (n < ntc) {
     *static_cast<volatile int*>(&ring.fail) = 1;
-    atomicOr(&p.ws->error, 1u);
+    if (p.ws != nullptr) atomicOr(&p.ws->error, 1u);
     for (unsigned int m = (n > static_cast<unsigned int>(kStages) ? n - kStages : 0); m < n; ++m)
       (void)mbar_wait(&ring.full[m % kStages], (m / kStages) & 1u);
   }
@@ -284,7 +284,7 @@ __device__ __forceinline__ bool ring_consume(R& ring, const Params& p, unsigned 
   // the outcome is made the same for the whole warp: callers vote across the warp later
   if (!__all_sync(0xFFFFFFFFu, mbar_wait(&ring.full[s], (n / kStages) & 1u))) {
     *static_cast<volatile int*>(&ring.fail) = 1;
-    atomicOr(&p.ws->error, 1u);
+    if (p.ws != nullptr) atomicOr(&p.ws->error, 1u);
     return false;
   }
   const uint4* src = reinterpret_cast<const uint4*>(ring.tile[s] + threadIdx.x * 32);
@@ -839,33 +839,63 @@ __global__ void __launch_bounds__(256) swizzle_kernel(const uint8_t* lin, uint8_
   }
 }
 
-// Eq. 3-4 on stored outputs.
-__global__ void __launch_bounds__(kTile) dequant_error_kernel(Params p, const uint8_t* scales, int swizzled,
+// Eq. 3-4 on stored outputs: sum (w - q s)^2 and sum w^2, one binary64 fma per term, with the
+// bf16 values widened by bit placement (scaled by 2^-128, undone at the end) and the signed
+// E2M1 values read from a 16-entry table in shared memory.  A wait that gave up turns the
+// results into NaN.
+__global__ void __launch_bounds__(kThreads) dequant_error_kernel(Params p, const uint8_t* scales, int swizzled,
                                                                  unsigned int col_tiles, const float* alpha_ptr,
                                                                  double* out_sse, double* out_sumsq) {
-  const double alpha = static_cast<double>(*alpha_ptr);
-  double acc[2] = {0.0, 0.0};
-  for (unsigned int b = blockIdx.x * kTile + threadIdx.x; b < p.nblk; b += gridDim.x * kTile) {
-    const unsigned int row = b / p.nbc, cb = b - row * p.nbc;
-    const uint16_t* src = p.W + static_cast<long long>(row) * p.ld + static_cast<long long>(cb) * 16;
-    const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(src));
-    const uint4 v1 = __ldg(reinterpret_cast<const uint4*>(src) + 1);
-    const unsigned int w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-    const uint2 cw = reinterpret_cast<const uint2*>(p.packed)[b];
-    const int dc = swizzled ? scales[swizzled_offset(row, cb, col_tiles)] : scales[b];
-    const double s = alpha * static_cast<double>(e4m3_value(dc & 0x7F));
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const unsigned int word = w[j >> 1];
-      const float wf = __uint_as_float((j & 1) ? (word & 0xFFFF0000u) : (word << 16));
-      const unsigned int code = ((j < 8 ? cw.x : cw.y) >> (4 * (j & 7))) & 0xFu;
-      const double q = static_cast<double>(e2m1_code_value(code & 7u)) * ((code & 8u) ? -1.0 : 1.0);
-      const double wd = static_cast<double>(wf);
-      const double e = wd - q * s;
-      acc[0] = fma(e, e, acc[0]);
-      acc[1] = fma(wd, wd, acc[1]);
-    }
+  __shared__ Ring ring;
+  __shared__ double s_q[16];
+  if (threadIdx.x < 16) {
+    const double mag = static_cast<double>(e2m1_code_value(threadIdx.x & 7u));
+    s_q[threadIdx.x] = (threadIdx.x & 8u) ? -mag : mag;
   }
+  ring_init(ring);
+  const unsigned int ntc = is_producer_warp() ? 0u : tiles_of_cta(p);
+  if (threadIdx.x == kTile) ring_produce(ring, p, 0);
+  const double alpha_scaled = static_cast<double>(*alpha_ptr) * 0x1p-128;
+  double acc[2] = {0.0, 0.0};
+  for (unsigned int n = 0; n < ntc; ++n) {
+    uint4 v0, v1;
+    if (!ring_consume(ring, p, n, v0, v1)) break;
+    const unsigned int b = tile_of(p, n, 0) * kTile + threadIdx.x;
+    if (b >= p.nblk) continue;
+    const uint2 cw = reinterpret_cast<const uint2*>(p.packed)[b];
+    int dc;
+    if (swizzled) {
+      const unsigned int row = b / p.nbc, cb = b - row * p.nbc;
+      dc = scales[swizzled_offset(row, cb, col_tiles)];
+    } else {
+      dc = scales[b];
+    }
+    const double s = alpha_scaled * static_cast<double>(e4m3_value(dc & 0x7F));
+    const unsigned int u[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+    double e0 = 0.0, e1 = 0.0, q0 = 0.0, q1 = 0.0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      // magnitude at bits 27..13 with exponent offset 768 (value * 2^-128), sign at bit 31;
+      // zeros and bf16 subnormals become zero
+      unsigned int lo = ((u[i] << 13) & 0x0FFFE000u) | 0x30000000u | ((u[i] << 16) & 0x80000000u);
+      unsigned int hi = ((u[i] >> 3) & 0x0FFFE000u) | 0x30000000u | (u[i] & 0x80000000u);
+      if ((u[i] & 0x00007F80u) == 0) lo = 0;
+      if ((u[i] & 0x7F800000u) == 0) hi = 0;
+      const double wl = __hiloint2double(static_cast<int>(lo), 0), wh = __hiloint2double(static_cast<int>(hi), 0);
+      const unsigned int word = (i < 4) ? cw.x : cw.y;
+      const double ql = s_q[(word >> (8 * (i & 3))) & 0xFu], qh = s_q[(word >> (8 * (i & 3) + 4)) & 0xFu];
+      const double dl = fma(-ql, s, wl), dh = fma(-qh, s, wh);
+      e0 = fma(dl, dl, e0);
+      e1 = fma(dh, dh, e1);
+      q0 = fma(wl, wl, q0);
+      q1 = fma(wh, wh, q1);
+    }
+    acc[0] += e0 + e1;
+    acc[1] += q0 + q1;
+  }
+  const bool failed = *static_cast<volatile int*>(&ring.fail) != 0;
+  acc[0] = failed ? __longlong_as_double(0x7FF8000000000000ll) : acc[0] * 0x1p256;
+  acc[1] = failed ? __longlong_as_double(0x7FF8000000000000ll) : acc[1] * 0x1p256;
   double* const dst[2] = {out_sse, out_sumsq};
   cta_accumulate<2>(acc, dst);
 }
@@ -1152,11 +1182,13 @@ int soar_dequant_error(const void* W_bf16, int64_t rows, int64_t cols, int64_t l
   p.ld = ld;
   p.nbc = static_cast<unsigned int>(cols / 16);
   p.nblk = static_cast<unsigned int>(rows * (cols / 16));
+  p.ntiles = (p.nblk + kTile - 1) / kTile;
+  p.contiguous = (ld == cols) ? 1 : 0;
   if (cudaMemsetAsync(out_sse, 0, sizeof(double), st) != cudaSuccess) return SOAR_ERR_CUDA;
   if (cudaMemsetAsync(out_sumsq, 0, sizeof(double), st) != cudaSuccess) return SOAR_ERR_CUDA;
   {
     ScopedLaunch sl(K_DEQUANT_ERROR, st);
-    dequant_error_kernel<<<persistent_grid(dequant_error_kernel, p.nblk, kTile), kTile, 0, st>>>(
+    dequant_error_kernel<<<persistent_grid(dequant_error_kernel, p.nblk, kThreads), kThreads, 0, st>>>(
         p, static_cast<const uint8_t*>(e4m3_scales), scale_layout == SOAR_SCALES_SWIZZLED ? 1 : 0,
         (p.nbc + 3) / 4, global_fp32, out_sse, out_sumsq);
   }
