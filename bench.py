@@ -196,6 +196,7 @@ def run_ours(args):
     import torch.distributed as dist
 
     from paper_2605_12245_b200 import api
+    from paper_2605_12245_b200 import sharding as SH
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -207,7 +208,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     api.lib()
     peaks = load_peaks()
-    wl = pick_workload(args.workload)
+    wl = SH.rank_workload(pick_workload(args.workload), rank)   # weak scaling: each rank its own layer
     cfg = preset_cfg(api, args.preset, args)
 
     # ---- inputs: generated on the host (seeded), resident in HBM before timing
@@ -245,11 +246,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         tr = api.soar_trace_end() if trace else {}
         barrier()
-        ms = e0.elapsed_time(e1) / steps
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = SH.max_over_ranks(e0.elapsed_time(e1) / steps, "cuda")
         return ms, tr
 
     sampler = ClockSampler(local)
@@ -354,10 +351,7 @@ def run_ours(args):
             e2e_step()
         torch.cuda.synchronize()
         dt = (time.perf_counter() - t0) / args.steps
-        if world > 1:
-            t = torch.tensor([dt], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = SH.max_over_ranks(dt, "cuda")
         # results must equal the resident-input run
         assert hosts[0].read_result().iters_run == iters[0]
         e2e = dict(value=world * 2.0 * elements / dt / 1e9, unit="GB/s", ms_per_step=dt * 1e3,
@@ -388,7 +382,7 @@ def run_ours(args):
                         n_dq=cfg.n_dq, early_stop_rel=cfg.early_stop_rel, tensors=len(wl.tensors),
                         elements=elements, iters_run=iters,
                         l2="inputs (%.2f GB per step) exceed the 126 MB L2" % (2 * elements / 1e9),
-                        parallelism=f"replicated workload x{world}, no collective"),
+                        parallelism=f"{world} rank(s), one layer of these shapes each, no collective"),
             elements_per_s=world * elements / (ms * 1e-3),
             hbm_frac_end_to_end_of_measured=value / peaks["hbm_gbs"],
             traced_ms_per_step=traced_ms, roofline=roofline, kernels=kernels, cpu_baseline=cpu, e2e=e2e, gpu_launches=launches,
