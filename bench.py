@@ -48,15 +48,33 @@ def load_peaks():
     return dict(hbm_gbs=6650.0, sm_max_mhz=1965.0, source="fallback")
 
 
-def pick_workload(name: str):
-    if name == "config1":
-        return WL.config1()
-    if name == "config2":
-        return WL.config2()
-    if name == "config4":
-        return WL.config4()
-    if name == "config5":
-        return WL.config5()
+class FlatWorkload:
+    """The tensors of one or several workloads as one list (config 3 is 36 layer workloads)."""
+
+    def __init__(self, name, parts):
+        self.name = name
+        self.sources = [(wl, i) for wl in parts for i in range(len(wl.tensors))]
+        self.tensors = tuple(wl.tensors[i] for wl, i in self.sources)
+
+    @property
+    def elements(self) -> int:
+        return sum(t.rows * t.cols for t in self.tensors)
+
+    def generate(self, i, *a, **kw):
+        wl, ti = self.sources[i]
+        return WL.generate(wl, ti, *a, **kw)
+
+
+def pick_workload(name: str, rank: int = 0) -> FlatWorkload:
+    """``rank`` > 0 draws the same shapes from a seed of its own (weak scaling: one layer per rank)."""
+    from paper_2605_12245_b200 import sharding as SH
+    single = {"config1": WL.config1, "config2": WL.config2, "config4": WL.config4, "config5": WL.config5}
+    if name in single:
+        wl = SH.rank_workload(single[name](), rank)
+        return FlatWorkload(wl.name, [wl])
+    if name == "config3":
+        return FlatWorkload("config3_qwen3_8b_36_layers" + (f"_rank{rank}" if rank else ""),
+                            [SH.rank_workload(WL.config3_layer(l), rank) for l in range(36)])
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -99,6 +117,31 @@ def kernel_bytes_per_elem(name: str, cfg, t: int = 0) -> float:
     if name == "dequant_error_kernel":
         return 2.0 + OUT_BYTES
     return 0.0
+
+
+# DRAM bytes per element (dram__bytes_read.sum + dram__bytes_write.sum of one launch, ncu, config 5:
+# profiles/single_pass_kernels_config5.md and profiles/iterate_kernel_paper_config5.md).  Traffic grows in
+# proportion to the elements, so a launch's traffic is this figure times its elements.  The figures
+# belong to one version of the kernels: they are dropped when the kernel source no longer matches.
+NCU_TRAFFIC = {
+    "kernel_source_sha256_16": "142b88b6407ddaf7",
+    "bytes_per_elem": {"amax_kernel": 2.02, "init_kernel": 2.43, "iterate_kernel/single": 3.00,
+                       "iterate_kernel/grid": 3.44},
+}
+
+
+def ncu_traffic_per_elem(name: str, cfg):
+    import hashlib
+    src = os.path.join(ROOT, "paper_2605_12245_b200", "csrc", "soar.cu")
+    try:
+        with open(src, "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest()[:16] != NCU_TRAFFIC["kernel_source_sha256_16"]:
+                return None
+    except OSError:
+        return None
+    if name == "iterate_kernel":
+        name += "/single" if (cfg.n_beta == 1 and cfg.n_dq <= 2) else "/grid"
+    return NCU_TRAFFIC["bytes_per_elem"].get(name)
 
 
 def call_bytes_per_elem(cfg, iters_run: int) -> float:
@@ -169,7 +212,7 @@ def run_reference(args):
     spec = wl.tensors[0]
     rows = min(spec.rows, max(1, args.ref_rows))
     rows = max(1, rows // WL._chunk_rows(spec.cols)) * WL._chunk_rows(spec.cols)
-    w = WL.generate(wl, 0, 0, rows)
+    w = wl.generate(0, 0, rows)
     for _ in range(args.warmup):
         R.quantize(w[: max(1, rows // 8)], rcfg)
     t0 = time.perf_counter()
@@ -208,13 +251,13 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     api.lib()
     peaks = load_peaks()
-    wl = SH.rank_workload(pick_workload(args.workload), rank)   # weak scaling: each rank its own layer
+    wl = pick_workload(args.workload, rank)
     cfg = preset_cfg(api, args.preset, args)
 
     # ---- inputs: generated on the host (seeded), resident in HBM before timing
     host_w, dev_w, outs = [], [], []
     for i, spec in enumerate(wl.tensors):
-        bits = WL.generate(wl, i)
+        bits = wl.generate(i)
         h = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
         host_w.append(h)
         dev_w.append(h.cuda())
@@ -264,6 +307,12 @@ def run_ours(args):
     # ---- roofline of the dominant kernel
     dom = max(trace, key=lambda k: trace[k][1])
     n_launch, tot_ms = trace[dom]
+    # DRAM traffic of an average working launch of the dominant kernel (ncu figure per element x elements)
+    active = sum(iters) if dom == "iterate_kernel" else len(wl.tensors)
+    tpe = ncu_traffic_per_elem(dom, cfg)
+    work_elems = (sum(s.rows * s.cols * it for s, it in zip(wl.tensors, iters)) if dom == "iterate_kernel"
+                  else elements)
+    traffic = None if tpe is None or active == 0 else tpe * work_elems / active
     if dom == "iterate_kernel" and iterate_ops_per_block(cfg) > 16 * 180:
         # candidate loop dominates: bound by plain FP32/INT issue
         blocks_iters = sum((s.rows * s.cols // 16) * it for s, it in zip(wl.tensors, iters)) * args.steps
@@ -271,7 +320,7 @@ def run_ours(args):
         achieved = ops / (tot_ms * 1e-3) / 1e12
         peak = SM_COUNT * FP32_LANES_PER_SM * peaks["sm_max_mhz"] * 1e6 / 1e12
         roofline = dict(bound="alu", kernel=dom, achieved=achieved, peak=peak, unit="Tlane-op/s",
-                        frac=achieved / peak, traffic=None, launches=n_launch,
+                        frac=achieved / peak, traffic=traffic, launches=n_launch,
                         active_launches=sum(iters) * args.steps, kernel_ms_per_step=tot_ms / args.steps,
                         peak_source="148 SMs x 128 FP32 lanes x clocks.max.sm",
                         hbm_gbs_for_context=sum(
@@ -285,7 +334,7 @@ def run_ours(args):
             byts = elements * args.steps * kernel_bytes_per_elem(dom, cfg)
         achieved = byts / (tot_ms * 1e-3) / 1e9
         roofline = dict(bound="hbm", kernel=dom, achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
-                        frac=achieved / peaks["hbm_gbs"], traffic=None, launches=n_launch,
+                        frac=achieved / peaks["hbm_gbs"], traffic=traffic, launches=n_launch,
                         kernel_ms_per_step=tot_ms / args.steps, peak_source=peaks["source"],
                         frac_of_nominal_8000=achieved / 8000.0)
     kernels = {k: dict(launches=v[0], ms_per_step=v[1] / args.steps, share=v[1] / sum(x[1] for x in trace.values()))
@@ -303,7 +352,11 @@ def run_ours(args):
             ms_per_step=sp_ms, value=world * 2.0 * elements / (sp_ms * 1e-3) / 1e9, unit="GB/s",
             algorithmic_bytes_per_step=sp_bytes, achieved_gbs=gbs, frac_of_measured_hbm=gbs / peaks["hbm_gbs"],
             frac_of_nominal_8000=gbs / 8000.0,
-            kernels={k: dict(launches=v[0], ms_per_step=v[1] / max(args.steps, 5)) for k, v in sp_tr.items()})
+            kernels={k: dict(launches=v[0], ms_per_step=v[1] / max(args.steps, 5),
+                             achieved_gbs=(elements * kernel_bytes_per_elem(k, sp, 0) * max(args.steps, 5)
+                                           / (v[1] * 1e-3) / 1e9) if v[1] > 0 else None,
+                             traffic_bytes_per_elem=ncu_traffic_per_elem(k, sp))
+                     for k, v in sp_tr.items()})
 
     # ---- the error check of Eq. 3-4 on the outputs just produced (its own entry point, not part of a step)
     err_out = torch.empty(2, dtype=torch.float64, device="cuda")
@@ -321,7 +374,7 @@ def run_ours(args):
     import ctypes
     ctypes_sizeof_result = ctypes.sizeof(api.SoarResult)
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and args.workload != "config3":      # config 3 would pin 18 GB of host memory
         big = max(wl.tensors, key=lambda s: s.rows * s.cols)
         streams = [torch.cuda.Stream(), torch.cuda.Stream()]
         stage = [(torch.empty((big.rows * big.cols,), dtype=torch.bfloat16, device="cuda"),
