@@ -80,8 +80,13 @@ def dq_candidates(center: np.ndarray, n: int, vals: np.ndarray) -> np.ndarray:
 
 
 def quantize(w_bits: np.ndarray, max_iters=15, early_stop_rel=1e-3, n_dq=2, n_beta=101,
-             beta_step_pct=1):
-    """Algorithm 1 on uint16 bf16 bit patterns [rows, cols]; returns a dict."""
+             beta_step_pct=1, coupled_scale=False, keep_alpha=False, keep_block_scale=False):
+    """Algorithm 1 on uint16 bf16 bit patterns [rows, cols]; returns a dict.
+
+    The three switches give the paper's stand-alone arms: ``coupled_scale`` is Sec. 3.2's
+    scheme (one block scale quantizes and dequantizes: a candidate's quantization scale is its
+    own E4M3 value times beta); ``keep_alpha`` and ``keep_block_scale`` together are Sec. 3.3
+    alone (no Eq. 5, no Eq. 6: the search runs around the max-based start)."""
     rows, cols = w_bits.shape
     wf = (w_bits.astype(np.uint32) << np.uint32(16)).view(F32)
     sign = (w_bits >> 15).astype(np.uint8).reshape(-1, 16)
@@ -120,25 +125,34 @@ def quantize(w_bits: np.ndarray, max_iters=15, early_stop_rel=1e-3, n_dq=2, n_be
         num = math.fsum((A * vals[dd])[live])
         den = math.fsum((B * vals[dd] ** 2)[live])
         alpha_new = F32(num / den) if den > 0 else alpha  # Eq. 5
+        if keep_alpha:
+            alpha_new = alpha
         # Eq. 6
         with np.errstate(divide="ignore", invalid="ignore"):
             center = (A.astype(F32) / (alpha_new * B.astype(F32)).astype(F32)).astype(F32)
         center = np.where(B > 0, center, vals[dd].astype(F32)).astype(F32)
+        if keep_block_scale:
+            center = vals[dd].astype(F32)
         cand_d = dq_candidates(center, n_dq, vals)         # [nblk, nd]
-        cand_q = (center[:, None] * bet[None, :]).astype(F32)  # [nblk, nb]
-        mk = reround(mag[:, None, :], alpha_new, cand_q)   # [nblk, nb, 16]
+        nd = cand_d.shape[1]
+        if coupled_scale:                                  # quantization scale = the candidate's own E4M3 value
+            base = vals[cand_d].astype(F32)                # [nblk, nd]
+        else:                                              # quantization scale around the unrounded solution
+            base = np.repeat(center[:, None], nd, axis=1)
+        cand_q = (base[:, None, :] * bet[None, :, None]).astype(F32)   # [nblk, nb, nd]
+        mk = reround(mag[:, None, None, :], alpha_new, cand_q)         # [nblk, nb, nd, 16]
         best = np.full(nblk, np.inf)
         bk = np.zeros(nblk, np.int64)
         bd = np.zeros(nblk, np.int64)
         for k in range(n_beta):                            # beta ascending, then d ascending
-            for j in range(cand_d.shape[1]):
-                L = err(mk[:, k, :], alpha_new, cand_d[:, j])
+            for j in range(nd):
+                L = err(mk[:, k, j, :], alpha_new, cand_d[:, j])
                 better = L < best                          # strict: first minimum wins
                 best = np.where(better, L, best)
                 bk = np.where(better, k, bk)
                 bd = np.where(better, j, bd)
         ar = np.arange(nblk)
-        dq = np.where(live, cand_q[ar, bk], dq).astype(F32)
+        dq = np.where(live, cand_q[ar, bk, bd], dq).astype(F32)
         dd = np.where(live, cand_d[ar, bd], dd)
         alpha = alpha_new
         sse_new = math.fsum(best[live])

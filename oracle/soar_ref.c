@@ -53,7 +53,18 @@ typedef struct soar_ref_cfg {
   int32_t n_dq;           /* E4M3 dequantization candidates per block (App. B.3)  */
   int32_t n_beta;         /* multipliers for the quantization scale (App. B.3)    */
   int32_t beta_step_pct;  /* grid step in hundredths (App. B.3: 0.01)             */
+  int32_t flags;          /* REF_FLAG_* : the paper's stand-alone arms (Sec. 3.2, 3.3) */
 } soar_ref_cfg;
+
+/* Sec. 3.2 alone ("Refinement Scheme"): one block scale plays both roles, so a candidate's
+ * quantization scale is its own E4M3 dequantization value (times beta) instead of the
+ * unrounded Eq. 6 solution. */
+#define REF_FLAG_COUPLED_SCALE 1
+/* Sec. 3.3 alone ((i),(ii)): the search runs around the max-based start, so Eq. 5 is
+ * skipped (alpha stays Eq. 1's) ... */
+#define REF_FLAG_KEEP_ALPHA 2
+/* ... and Eq. 6 is skipped (the candidate sets are centred on the stored scale). */
+#define REF_FLAG_KEEP_BLOCK_SCALE 4
 
 /* ------------------------------------------------------------------ formats */
 
@@ -203,35 +214,39 @@ static void dss_block(const uint16_t* w, float alpha, float center, const soar_r
   uint8_t dc[REF_MAX_DQ];
   int nd = soar_ref_dq_candidates(center, cfg->n_dq, dc);
   int nb = cfg->n_beta;
-  static _Thread_local double mk[REF_MAX_BETA][REF_BLOCK];
+  const int coupled = (cfg->flags & REF_FLAG_COUPLED_SCALE) != 0;
+  /* one entry per candidate pair (k, d); without coupling the codes of a beta are the same
+   * for every d and are simply made again */
+  static _Thread_local double mk[REF_MAX_BETA][REF_MAX_DQ][REF_BLOCK];
   static _Thread_local double Lk[REF_MAX_BETA][REF_MAX_DQ];
-  static _Thread_local double Ak[REF_MAX_BETA], Bk[REF_MAX_BETA];
-  static _Thread_local float dqk[REF_MAX_BETA];
+  static _Thread_local double Ak[REF_MAX_BETA][REF_MAX_DQ], Bk[REF_MAX_BETA][REF_MAX_DQ];
+  static _Thread_local float dqk[REF_MAX_BETA][REF_MAX_DQ];
   double best = 0.0;
   int bk = -1, bd = -1;
   for (int k = 0; k < nb; ++k) {
-    float dq = center * soar_ref_beta(k, nb, cfg->beta_step_pct);
-    dqk[k] = dq;
-    soar_ref_round_block(w, alpha, dq, mk[k], &Ak[k], &Bk[k]);
+    float beta = soar_ref_beta(k, nb, cfg->beta_step_pct);
     for (int d = 0; d < nd; ++d) {
-      double L = soar_ref_block_error(w, mk[k], alpha, dc[d]);
+      float dq = (coupled ? soar_ref_e4m3_decode(dc[d]) : center) * beta;
+      dqk[k][d] = dq;
+      soar_ref_round_block(w, alpha, dq, mk[k][d], &Ak[k][d], &Bk[k][d]);
+      double L = soar_ref_block_error(w, mk[k][d], alpha, dc[d]);
       Lk[k][d] = L;
       if (bk < 0 || L < best) { best = L; bk = k; bd = d; }
     }
   }
   double second = 1e300;
   for (int k = 0; k < nb; ++k) {
-    int same_codes = memcmp(mk[k], mk[bk], sizeof(mk[k])) == 0;
     for (int d = 0; d < nd; ++d) {
-      if (same_codes && d == bd) continue;
+      int same_codes = memcmp(mk[k][d], mk[bk][bd], sizeof(mk[k][d])) == 0;
+      if (same_codes && dc[d] == dc[bd]) continue;
       if (Lk[k][d] < second) second = Lk[k][d];
     }
   }
-  *dq_out = dqk[bk];
+  *dq_out = dqk[bk][bd];
   *d_out = dc[bd];
   *L_out = best;
-  *A_out = Ak[bk];
-  *B_out = Bk[bk];
+  *A_out = Ak[bk][bd];
+  *B_out = Bk[bk][bd];
   if (second >= 1e300) *gap_rel = 1e300;
   else if (best > 0.0) *gap_rel = (second - best) / best;
   else *gap_rel = (second > 0.0) ? 1e300 : 0.0;
@@ -354,6 +369,7 @@ int soar_ref_quantize(const uint16_t* W, int64_t rows, int64_t cols, int64_t ld,
     /* Eq. 5: alpha^(t+1); one rounding of the binary64 quotient. A zero
      * denominator (every code zero) keeps alpha. */
     float alpha_new = (den > 0.0) ? (float)(num / den) : alpha;
+    if (cfg->flags & REF_FLAG_KEEP_ALPHA) alpha_new = alpha;      /* Sec. 3.3 alone: alpha stays Eq. 1's */
 
     /* Eq. 6 with the same codes and the new alpha, then DSS per block. */
 #pragma omp parallel for schedule(dynamic, 1)
@@ -365,7 +381,9 @@ int soar_ref_quantize(const uint16_t* W, int64_t rows, int64_t cols, int64_t ld,
         const uint16_t* w = W + r * ld + b * REF_BLOCK;
         double m[REF_BLOCK], A, B;
         soar_ref_round_block(w, alpha, dq[i], m, &A, &B);
-        float center = soar_ref_block_scale(A, B, alpha_new, dd[i]);
+        float center = (cfg->flags & REF_FLAG_KEEP_BLOCK_SCALE)
+                           ? soar_ref_e4m3_decode(dd[i])                  /* Sec. 3.3 alone: around the stored scale */
+                           : soar_ref_block_scale(A, B, alpha_new, dd[i]);
         float ndq;
         uint8_t nd;
         double L, wA, wB, gap;

@@ -23,6 +23,8 @@ STATUS_ZERO_TENSOR = 1
 STATUS_NONFINITE = 2
 STATUS_RANGE = 4
 
+FLAG_COUPLED_SCALE, FLAG_KEEP_ALPHA, FLAG_KEEP_BLOCK_SCALE = 1, 2, 4
+
 GCC_FLAGS = ["-O2", "-msse4.1", "-fopenmp", "-ffp-contract=off", "-fPIC", "-shared"]
 
 
@@ -42,6 +44,7 @@ class _Cfg(C.Structure):
         ("n_dq", C.c_int32),
         ("n_beta", C.c_int32),
         ("beta_step_pct", C.c_int32),
+        ("flags", C.c_int32),
     ]
 
 
@@ -54,9 +57,11 @@ class RefCfg:
     n_dq: int = 2
     n_beta: int = 101
     beta_step_pct: int = 1
+    flags: int = 0            # FLAG_* bits: the paper's stand-alone arms (Sec. 3.2, Sec. 3.3)
 
     def c(self) -> _Cfg:
-        return _Cfg(self.max_iters, self.early_stop_rel, self.n_dq, self.n_beta, self.beta_step_pct)
+        return _Cfg(self.max_iters, self.early_stop_rel, self.n_dq, self.n_beta, self.beta_step_pct,
+                    self.flags)
 
 
 @dataclass
