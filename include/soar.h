@@ -49,6 +49,16 @@ extern "C" {
 #define SOAR_PRESET_PAPER 0            /* T=15, stop 1e-3, 2 E4M3 neighbours, 101 beta (Sec. 4.1, App. B.3) */
 #define SOAR_PRESET_SINGLE_PASS 1      /* T=1, no early stop, 2 neighbours, beta = {1}       */
 #define SOAR_PRESET_RTN 2              /* T=0: the max-based rule of Eq. 1-3 only            */
+#define SOAR_PRESET_CJSO_ONLY 3        /* Sec. 3.2 alone: T=15, stop 1e-3, nearest E4M3 code, coupled scale */
+#define SOAR_PRESET_DSS_ONLY 4         /* Sec. 3.3 alone: one search (2 x 101) around the max-based start   */
+
+/* soar_cfg.flags bits: the stand-alone arms of the paper's ablation (Table 4) */
+#define SOAR_FLAG_COUPLED_SCALE 1      /* Sec. 3.2 "Refinement Scheme": one block scale quantizes and
+                                          dequantizes; a candidate's quantization scale is its own E4M3
+                                          value times beta, not the unrounded Eq. 6 solution times beta */
+#define SOAR_FLAG_KEEP_ALPHA 2         /* skip Eq. 5: alpha stays the max-based value of Eq. 1 */
+#define SOAR_FLAG_KEEP_BLOCK_SCALE 4   /* skip Eq. 6: candidate sets are centred on the stored scale
+                                          (with KEEP_ALPHA: Sec. 3.3 (i),(ii) alone) */
 
 #define SOAR_MAX_ITERS 64
 #define SOAR_MAX_BETA 512
@@ -68,7 +78,7 @@ typedef struct soar_cfg {
                              (App. B.3: 101, i.e. 0.50 .. 1.50); centred on 1.00            */
   int32_t beta_step_pct;  /* multiplier step in hundredths (App. B.3: 1)                     */
   int32_t scale_layout;   /* SOAR_SCALES_* bits: which scale outputs to write               */
-  int32_t flags;          /* reserved, must be 0                                            */
+  int32_t flags;          /* SOAR_FLAG_* bits; 0 = Algorithm 1                              */
 } soar_cfg;
 
 /* Per-call report (device memory, written by the last kernel of soar_quantize). */

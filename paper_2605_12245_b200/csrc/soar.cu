@@ -74,6 +74,7 @@ struct Params {
   int n_dq;
   int n_beta;
   int beta_step_pct;
+  int flags;           // SOAR_FLAG_* bits
 };
 
 // ------------------------------------------------------------------ number formats
@@ -597,8 +598,9 @@ __device__ __forceinline__ void iteration_head(const Params& p, int t, float& al
       if (stops_after(prev, cur, p.early_stop_rel)) { run = 0; break; }
       prev = cur;
     }
-    for (int i = 0; i <= t; ++i)            // Eq. 5: alpha^(i+1) from stage-i sums
-      if (ws->den[i] > 0.0) alpha = static_cast<float>(ws->num[i] / ws->den[i]);
+    if (!(p.flags & SOAR_FLAG_KEEP_ALPHA))
+      for (int i = 0; i <= t; ++i)          // Eq. 5: alpha^(i+1) from stage-i sums
+        if (ws->den[i] > 0.0) alpha = static_cast<float>(ws->num[i] / ws->den[i]);
   }
   alpha_out = alpha;
   run_out = run;
@@ -606,10 +608,12 @@ __device__ __forceinline__ void iteration_head(const Params& p, int t, float& al
 
 // Eq. 6 with the new alpha from the previous winner's sums (all codes zero keeps the stored
 // scale), and App. B.3's E4M3 codes around it: d_lo .. d_hi before clipping.
-__device__ __forceinline__ float block_center(const uint2 st, float alpha, int n_dq, int& d_lo, int& d_hi) {
+__device__ __forceinline__ float block_center(const uint2 st, float alpha, int n_dq, bool keep, int& d_lo,
+                                              int& d_hi) {
   const int d_cur = static_cast<int>(st.y >> 16);
   const float B0 = 0.25f * static_cast<float>(st.y & 0xFFFFu);
-  const float center = (B0 > 0.0f) ? __fdiv_rn(__uint_as_float(st.x), __fmul_rn(alpha, B0)) : e4m3_value(d_cur);
+  const float center = (B0 > 0.0f && !keep) ? __fdiv_rn(__uint_as_float(st.x), __fmul_rn(alpha, B0))
+                                             : e4m3_value(d_cur);
   const int cn = e4m3_encode(center);
   if (n_dq <= 1) {
     d_lo = d_hi = cn;
@@ -667,7 +671,7 @@ iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
     Block blk;
     unpack_block(v0, v1, blk);
     int d_lo, d_hi;
-    const float center = block_center(st, alpha, n_dq, d_lo, d_hi);
+    const float center = block_center(st, alpha, n_dq, (p.flags & SOAR_FLAG_KEEP_BLOCK_SCALE) != 0, d_lo, d_hi);
     const int dc0 = clip_code(d_lo), dc1 = clip_code(d_lo + 1);
     const double sd0 = alpha_d * static_cast<double>(e4m3_value(dc0));
     const double sd1 = alpha_d * static_cast<double>(e4m3_value(dc1));
@@ -698,8 +702,9 @@ iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
       const int nd = d_hi - d_lo + 1;
       // the reciprocal scale falls as beta grows, so the first candidate decides whether the
       // exact integer sums hold for all of them
+      const bool coupled = (p.flags & SOAR_FLAG_COUPLED_SCALE) != 0;
       const bool all_narrow = fx.ok && __fmul_rn(blk.bmax, recip_scale(alpha, __fmul_rn(center, s_beta[0]))) <= 32.0f;
-      if (all_narrow && nd <= 2) {
+      if (all_narrow && nd <= 2 && !coupled) {
         // error minus sum W^2 = sd^2 B - 2 sd A = p * (4B) - q * afix  with  p = sd^2/4, q = 2 sd unit
         const double p0 = 0.25 * sd0 * sd0, q0 = 2.0 * sd0 * fx.unit;
         const double p1 = 0.25 * sd1 * sd1, q1 = 2.0 * sd1 * fx.unit;
@@ -717,16 +722,25 @@ iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
           }
         }
       } else {
+        // general form: any number of E4M3 candidates, scales far below the block maximum, and the
+        // coupled arm of Sec. 3.2, where each E4M3 candidate rounds the block with its own value
         for (int k = 0; k < n_beta; ++k) {
-          const float r = recip_scale(alpha, __fmul_rn(center, s_beta[k]));
+          float r = recip_scale(alpha, __fmul_rn(center, s_beta[k]));
           unsigned int c0, c1;
-          round_block(blk, r, c0, c1);
-          double A, B;
-          block_sums(blk, fx, r, c0, c1, A, B, wide);
-          const double A2 = -2.0 * A;
+          double A = 0.0, B = 0.0;
+          if (!coupled) {
+            round_block(blk, r, c0, c1);
+            block_sums(blk, fx, r, c0, c1, A, B, wide);
+          }
           for (int d = 0; d < nd; ++d) {
-            const double sd = alpha_d * static_cast<double>(e4m3_value(clip_code(d_lo + d)));
-            const double g = sd * fma(sd, B, A2);
+            const float dv = e4m3_value(clip_code(d_lo + d));
+            if (coupled) {
+              r = recip_scale(alpha, __fmul_rn(dv, s_beta[k]));
+              round_block(blk, r, c0, c1);
+              block_sums(blk, fx, r, c0, c1, A, B, wide);
+            }
+            const double sd = alpha_d * static_cast<double>(dv);
+            const double g = sd * fma(sd, B, -2.0 * A);
             if (g < best) { best = g; best_key = (nd <= 2 ? 2 : nd) * k + d; }
           }
         }
@@ -735,7 +749,7 @@ iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
       const int per = nd <= 2 ? 2 : nd;
       const int bk = best_key / per;
       best_d = clip_code(d_lo + (best_key - bk * per));
-      const float r = recip_scale(alpha, __fmul_rn(center, s_beta[bk]));
+      const float r = recip_scale(alpha, __fmul_rn(coupled ? e4m3_value(best_d) : center, s_beta[bk]));
       round_block(blk, r, best0, best1);
       unsigned int unused = 0;
       block_sums(blk, fx, r, best0, best1, bestA, bestB, unused);
@@ -782,7 +796,7 @@ __global__ void __launch_bounds__(128) finalize_kernel(Params p, float* out_alph
     if (st == 0 && ws->error == 0) {
       double prev = s_sse[0];
       for (int i = 0; i < p.max_iters; ++i) {
-        if (s_den[i] > 0.0) alpha = static_cast<float>(s_num[i] / s_den[i]);
+        if (s_den[i] > 0.0 && !(p.flags & SOAR_FLAG_KEEP_ALPHA)) alpha = static_cast<float>(s_num[i] / s_den[i]);
         const double cur = s_sse[i + 1];
         iters = i + 1;
         s_ta[iters] = static_cast<double>(alpha);
@@ -988,7 +1002,8 @@ int check_cfg(const soar_cfg* cfg) {
   if (100 - (cfg->n_beta / 2) * cfg->beta_step_pct <= 0) return SOAR_ERR_INVALID_ARG;
   if ((cfg->scale_layout & ~(SOAR_SCALES_LINEAR | SOAR_SCALES_SWIZZLED)) != 0 || cfg->scale_layout == 0)
     return SOAR_ERR_INVALID_ARG;
-  if (cfg->flags != 0) return SOAR_ERR_INVALID_ARG;
+  if ((cfg->flags & ~(SOAR_FLAG_COUPLED_SCALE | SOAR_FLAG_KEEP_ALPHA | SOAR_FLAG_KEEP_BLOCK_SCALE)) != 0)
+    return SOAR_ERR_INVALID_ARG;
   return SOAR_OK;
 }
 
@@ -1012,6 +1027,14 @@ int soar_default_cfg(soar_cfg* cfg, int preset) {
       return SOAR_OK;
     case SOAR_PRESET_RTN:
       cfg->max_iters = 0; cfg->early_stop_rel = 0.0f; cfg->n_dq = 1; cfg->n_beta = 1;
+      return SOAR_OK;
+    case SOAR_PRESET_CJSO_ONLY:
+      cfg->max_iters = 15; cfg->early_stop_rel = 1e-3f; cfg->n_dq = 1; cfg->n_beta = 1;
+      cfg->flags = SOAR_FLAG_COUPLED_SCALE;
+      return SOAR_OK;
+    case SOAR_PRESET_DSS_ONLY:
+      cfg->max_iters = 1; cfg->early_stop_rel = 0.0f; cfg->n_dq = 2; cfg->n_beta = 101;
+      cfg->flags = SOAR_FLAG_KEEP_ALPHA | SOAR_FLAG_KEEP_BLOCK_SCALE;
       return SOAR_OK;
     default:
       return SOAR_ERR_INVALID_ARG;
@@ -1081,6 +1104,7 @@ int soar_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, co
   p.n_dq = cfg->n_dq;
   p.n_beta = cfg->n_beta;
   p.beta_step_pct = cfg->beta_step_pct;
+  p.flags = cfg->flags;
 
   if (cudaMemsetAsync(workspace, 0, kWsFixedBytes, st) != cudaSuccess) return SOAR_ERR_CUDA;
   // Passes alternate direction over the tiles: each starts where the previous one ended,
@@ -1096,7 +1120,7 @@ int soar_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, co
     init_kernel<<<persistent_grid(init_kernel, p.nblk, kThreads), kThreads, 0, st>>>(p, reverse,
                                                                                      cfg->max_iters == 0 ? 1 : 0);
   }
-  const bool single = cfg->n_beta == 1 && cfg->n_dq <= 2;
+  const bool single = cfg->n_beta == 1 && cfg->n_dq <= 2 && !(cfg->flags & SOAR_FLAG_COUPLED_SCALE);
   const unsigned int g_it = single ? persistent_grid(iterate_kernel<true>, p.nblk, kThreads)
                                    : persistent_grid(iterate_kernel<false>, p.nblk, kThreads);
   const bool may_stop = cfg->early_stop_rel > 0.0f;

@@ -37,7 +37,7 @@ def cfg_pair(**kw):
     ref = R.RefCfg(**kw)
     cfg = api.soar_default_cfg(api.PRESET_PAPER, max_iters=ref.max_iters,
                                early_stop_rel=ref.early_stop_rel, n_dq=ref.n_dq,
-                               n_beta=ref.n_beta, beta_step_pct=ref.beta_step_pct)
+                               n_beta=ref.n_beta, beta_step_pct=ref.beta_step_pct, flags=ref.flags)
     return cfg, ref
 
 

@@ -27,6 +27,10 @@ pytestmark = pytest.mark.gpu
     dict(max_iters=1, early_stop_rel=0.0, n_dq=2, n_beta=1),  # single pass
     dict(max_iters=3, early_stop_rel=0.0, n_dq=1, n_beta=1),  # CJSO with the nearest scale
     dict(max_iters=2, early_stop_rel=0.0, n_dq=4, n_beta=6, beta_step_pct=3),
+    dict(flags=1, n_dq=1, n_beta=1),                                        # Sec. 3.2 alone (coupled scale)
+    dict(flags=1, max_iters=2, early_stop_rel=0.0, n_dq=2, n_beta=3, beta_step_pct=5),
+    dict(flags=6, max_iters=1, early_stop_rel=0.0),                          # Sec. 3.3 alone (2 x 101 search)
+    dict(flags=6, max_iters=2, early_stop_rel=0.0, n_dq=4, n_beta=7, beta_step_pct=4),
 ])
 def test_parity_small(rows, cols, ld, seed, kw, cfgkw):
     w = WL.small_case(rows, cols, seed, **kw)
@@ -107,6 +111,15 @@ def test_wide_candidates_take_the_exact_path():
     P.assert_parity(gpu, R.quantize(bits, ref_cfg))
 
 
+def test_presets_of_the_stand_alone_arms_match_the_oracle():
+    w = WL.small_case(96, 1024, 61, outlier_cols_frac=0.004, outlier_scale=20.0)
+    for preset, ref_cfg in (
+            (api.PRESET_CJSO_ONLY, R.RefCfg(n_dq=1, n_beta=1, flags=R.FLAG_COUPLED_SCALE)),
+            (api.PRESET_DSS_ONLY, R.RefCfg(max_iters=1, early_stop_rel=0.0,
+                                           flags=R.FLAG_KEEP_ALPHA | R.FLAG_KEEP_BLOCK_SCALE))):
+        P.assert_parity(P.run_gpu(w, api.soar_default_cfg(preset)), R.quantize(w, ref_cfg))
+
+
 def test_argument_errors_are_reported_on_the_host():
     w = P.to_device(WL.small_case(4, 64, 0))
     cfg = api.soar_default_cfg()
@@ -115,6 +128,8 @@ def test_argument_errors_are_reported_on_the_host():
     bad = api.soar_default_cfg(block=32)
     with pytest.raises(api.SoarError):
         api.soar_quantize(w, bad)
+    with pytest.raises(api.SoarError):
+        api.soar_quantize(w, api.soar_default_cfg(flags=8))    # unknown flag bit
     out = api.alloc_buffers(4, 64, cfg)
     out.workspace = out.workspace[:16]
     with pytest.raises(api.SoarError):
