@@ -220,6 +220,17 @@ typedef struct soar_trace_entry {
 int soar_trace_begin(void);
 int soar_trace_end(soar_trace_entry* out, int capacity, int* count);
 
+/*
+ * Self-test of an arithmetic shortcut (no counterpart in the paper).  The candidate loop of
+ * soar_quantize needs 1/(alpha * dq) rounded to nearest (the reciprocal of Eq. 2's divisor) for
+ * every candidate; it computes it as the hardware's approximate reciprocal plus one Newton
+ * step, which on sm_100a equals the correctly rounded reciprocal for every input of the range
+ * it is used on.  This call counts, on the device, the binary32 inputs with biased exponent
+ * lo_exp..hi_exp (2 <= lo_exp <= hi_exp <= 252; all 2^23 significands each) on which the two
+ * differ, into *out_mismatches (device, 8 bytes).  The full range takes about two seconds.
+ */
+int soar_selftest_reciprocal(int lo_exp, int hi_exp, unsigned long long* out_mismatches, void* stream);
+
 /* Text for a host-side return value. */
 const char* soar_status_string(int status);
 

@@ -26,7 +26,7 @@ MAX_ITERS = 64
 EXPORTS = (
     "soar_default_cfg", "soar_workspace_bytes", "soar_swizzled_scale_bytes", "soar_quantize",
     "soar_dequant_error", "soar_quantize_launches", "soar_status_string", "soar_quantize_host",
-    "soar_trace_begin", "soar_trace_end", "soar_quantize_static",
+    "soar_trace_begin", "soar_trace_end", "soar_quantize_static", "soar_selftest_reciprocal",
 )
 
 
@@ -100,6 +100,8 @@ def lib() -> C.CDLL:
                                          C.POINTER(SoarStaging), vp]
         L.soar_quantize_static.restype = C.c_int
         L.soar_quantize_static.argtypes = [vp, i64, i64, i64, C.POINTER(SoarCfg), vp, vp, vp, vp, vp, vp]
+        L.soar_selftest_reciprocal.restype = C.c_int
+        L.soar_selftest_reciprocal.argtypes = [C.c_int, C.c_int, vp, vp]
         L.soar_trace_begin.restype = C.c_int
         L.soar_trace_begin.argtypes = []
         L.soar_trace_end.restype = C.c_int
@@ -281,6 +283,13 @@ def soar_quantize_host(host: HostBuffers, cfg: SoarCfg, dev_W: torch.Tensor, dev
         _ptr(host.W), rows, cols, cols, C.byref(cfg), _ptr(host.packed), _ptr(host.scales),
         _ptr(host.scales_sw), _ptr(host.alpha), _ptr(host.result), C.byref(st), _stream_ptr(stream))
     _check(rc, "soar_quantize_host")
+
+
+def soar_selftest_reciprocal(lo_exp: int = 2, hi_exp: int = 252, stream=None) -> int:
+    """Runs ``soar_selftest_reciprocal`` and returns the mismatch count (synchronizes)."""
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    _check(lib().soar_selftest_reciprocal(lo_exp, hi_exp, _ptr(out), _stream_ptr(stream)), "soar_selftest_reciprocal")
+    return int(out.cpu()[0])
 
 
 def soar_trace_begin() -> None:

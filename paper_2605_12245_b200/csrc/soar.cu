@@ -414,6 +414,19 @@ __device__ __forceinline__ float recip_scale(float alpha, float dq) {
   return __frcp_rn(__fmul_rn(alpha, dq));
 }
 
+// 1/s rounded to nearest for s in [2^-125, 2^126): the hardware's approximate reciprocal
+// followed by one Newton step, y + y * (1 - s y), both as fused multiply-adds.  On sm_100a this
+// equals rcp.rn for every binary32 input of that range (soar_selftest_reciprocal compares all
+// of them); it is a third of the instructions.  Callers check the range (recip_fast_ok).
+__device__ __forceinline__ float recip_fast(float s) {
+  float y;
+  asm("rcp.approx.f32 %0, %1;" : "=f"(y) : "f"(s));
+  return __fmaf_rn(y, __fmaf_rn(-s, y, 1.0f), y);
+}
+__device__ __forceinline__ bool recip_fast_ok(float s) {
+  return ((__float_as_uint(s) >> 23) - 2u) <= 250u;   // positive, biased exponent 2 .. 252
+}
+
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
@@ -704,12 +717,15 @@ iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
       // exact integer sums hold for all of them
       const bool coupled = (p.flags & SOAR_FLAG_COUPLED_SCALE) != 0;
       const bool all_narrow = fx.ok && __fmul_rn(blk.bmax, recip_scale(alpha, __fmul_rn(center, s_beta[0]))) <= 32.0f;
-      if (all_narrow && nd <= 2 && !coupled) {
+      // the products alpha * center * beta are monotone in beta: the end points bound them all
+      const bool fast_rcp = recip_fast_ok(__fmul_rn(alpha, __fmul_rn(center, s_beta[0]))) &&
+                            recip_fast_ok(__fmul_rn(alpha, __fmul_rn(center, s_beta[n_beta - 1])));
+      if (all_narrow && nd <= 2 && !coupled && fast_rcp) {
         // error minus sum W^2 = sd^2 B - 2 sd A = p * (4B) - q * afix  with  p = sd^2/4, q = 2 sd unit
         const double p0 = 0.25 * sd0 * sd0, q0 = 2.0 * sd0 * fx.unit;
         const double p1 = 0.25 * sd1 * sd1, q1 = 2.0 * sd1 * fx.unit;
         for (int k = 0; k < n_beta; ++k) {
-          const float r = recip_scale(alpha, __fmul_rn(center, s_beta[k]));
+          const float r = recip_fast(__fmul_rn(alpha, __fmul_rn(center, s_beta[k])));
           unsigned int c0, c1, afix, b4;
           round_block(blk, r, c0, c1);
           code_sums(fx, c0, c1, afix, b4);
@@ -912,6 +928,19 @@ __global__ void __launch_bounds__(kThreads) dequant_error_kernel(Params p, const
   acc[1] = failed ? __longlong_as_double(0x7FF8000000000000ll) : acc[1] * 0x1p256;
   double* const dst[2] = {out_sse, out_sumsq};
   cta_accumulate<2>(acc, dst);
+}
+
+// Counts the binary32 inputs with biased exponent lo_exp..hi_exp (all 2^23 significands each)
+// on which recip_fast differs from rcp.rn.
+__global__ void selftest_reciprocal_kernel(unsigned int lo_exp, unsigned int hi_exp, unsigned long long* mismatches) {
+  const unsigned long long total = static_cast<unsigned long long>(hi_exp - lo_exp + 1) << 23;
+  unsigned long long bad = 0;
+  for (unsigned long long i = blockIdx.x * static_cast<unsigned long long>(blockDim.x) + threadIdx.x; i < total;
+       i += static_cast<unsigned long long>(gridDim.x) * blockDim.x) {
+    const float s = __uint_as_float((lo_exp << 23) + static_cast<unsigned int>(i));
+    if (__float_as_uint(recip_fast(s)) != __float_as_uint(__frcp_rn(s))) ++bad;
+  }
+  if (bad) atomicAdd(mismatches, bad);
 }
 
 // ------------------------------------------------------------------ host side
@@ -1252,6 +1281,15 @@ int soar_quantize_host(const void* W_host, int64_t rows, int64_t cols, int64_t l
     ok = ok && cudaMemcpyAsync(out_result_host, dev->result, sizeof(soar_result), cudaMemcpyDeviceToHost, st) ==
                    cudaSuccess;
   return ok ? SOAR_OK : SOAR_ERR_CUDA;
+}
+
+int soar_selftest_reciprocal(int lo_exp, int hi_exp, unsigned long long* out_mismatches, void* stream) {
+  if (out_mismatches == nullptr || lo_exp < 2 || hi_exp > 252 || lo_exp > hi_exp) return SOAR_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(out_mismatches, 0, sizeof(unsigned long long), st) != cudaSuccess) return SOAR_ERR_CUDA;
+  selftest_reciprocal_kernel<<<sm_count() * 8, 256, 0, st>>>(static_cast<unsigned int>(lo_exp),
+                                                             static_cast<unsigned int>(hi_exp), out_mismatches);
+  return cudaGetLastError() == cudaSuccess ? SOAR_OK : SOAR_ERR_CUDA;
 }
 
 int soar_trace_begin(void) {

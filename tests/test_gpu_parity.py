@@ -120,6 +120,13 @@ def test_presets_of_the_stand_alone_arms_match_the_oracle():
         P.assert_parity(P.run_gpu(w, api.soar_default_cfg(preset)), R.quantize(w, ref_cfg))
 
 
+def test_fast_reciprocal_equals_the_correctly_rounded_one_everywhere_it_is_used():
+    """All 2^23 significands of every exponent the shortcut is allowed on: 2.1e9 inputs."""
+    assert api.soar_selftest_reciprocal(2, 252) == 0
+    with pytest.raises(api.SoarError):
+        api.soar_selftest_reciprocal(1, 252)
+
+
 def test_argument_errors_are_reported_on_the_host():
     w = P.to_device(WL.small_case(4, 64, 0))
     cfg = api.soar_default_cfg()
