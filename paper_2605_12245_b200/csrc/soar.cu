@@ -342,6 +342,7 @@ __device__ __forceinline__ void round_block(const Block& blk, float r, unsigned 
 struct Fixed {
   unsigned int pair[8];
   double unit;   // 2^(e - 16): A = unit * sum fix_j * (2 m_j)
+  double inv8;   // 1 / (8 unit)
   bool ok;       // false for block maxima below 2^-110, which take the binary64 path
 };
 
@@ -351,6 +352,7 @@ __device__ __forceinline__ void make_fixed(const Block& blk, Fixed& fx) {
   const unsigned int ebc = max(eb, 17u);
   const float S = __uint_as_float((269u - ebc) << 23);       // 2^(15 - e)
   fx.unit = __hiloint2double(static_cast<int>((ebc + 880u) << 20), 0);
+  fx.inv8 = __hiloint2double(static_cast<int>((1163u - ebc) << 20), 0);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const unsigned int lo = __float_as_uint(__fmaf_rn(fabsf(blk.w[2 * i]), S, 8388608.0f));
@@ -721,22 +723,31 @@ iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
       const bool fast_rcp = recip_fast_ok(__fmul_rn(alpha, __fmul_rn(center, s_beta[0]))) &&
                             recip_fast_ok(__fmul_rn(alpha, __fmul_rn(center, s_beta[n_beta - 1])));
       if (all_narrow && nd <= 2 && !coupled && fast_rcp) {
-        // error minus sum W^2 = sd^2 B - 2 sd A = p * (4B) - q * afix  with  p = sd^2/4, q = 2 sd unit
-        const double p0 = 0.25 * sd0 * sd0, q0 = 2.0 * sd0 * fx.unit;
-        const double p1 = 0.25 * sd1 * sd1, q1 = 2.0 * sd1 * fx.unit;
+        // error minus sum W^2 = sd^2 B - 2 sd A = q * (rho * (4B) - afix)  with  q = 2 sd unit > 0 and
+        // rho = sd / (8 unit): per E4M3 code the candidates are ranked by rho * 4B - afix alone (one fma),
+        // and the two codes' winners are compared once after the loop
+        const double rho0 = sd0 * fx.inv8, rho1 = sd1 * fx.inv8;
+        double h0 = best, h1 = best;
+        int k0 = 0, k1 = 0;
         for (int k = 0; k < n_beta; ++k) {
           const float r = recip_fast(__fmul_rn(alpha, __fmul_rn(center, s_beta[k])));
           unsigned int c0, c1, afix, b4;
           round_block(blk, r, c0, c1);
           code_sums(fx, c0, c1, afix, b4);
           const double ad = uint_to_double(afix), bd = uint_to_double(b4);
-          const double g0 = fma(p0, bd, -(q0 * ad));
-          if (g0 < best) { best = g0; best_key = 2 * k; }
+          const double e0 = fma(rho0, bd, -ad);
+          if (e0 < h0) { h0 = e0; k0 = k; }
           if (nd == 2) {
-            const double g1 = fma(p1, bd, -(q1 * ad));
-            if (g1 < best) { best = g1; best_key = 2 * k + 1; }
+            const double e1 = fma(rho1, bd, -ad);
+            if (e1 < h1) { h1 = e1; k1 = k; }
           }
         }
+        const double g0 = 2.0 * sd0 * fx.unit * h0;
+        const double g1 = (nd == 2) ? 2.0 * sd1 * fx.unit * h1 : best;
+        // first minimum in (beta, code) order
+        const bool second = g1 < g0 || (g1 == g0 && k1 < k0);
+        best = second ? g1 : g0;
+        best_key = second ? 2 * k1 + 1 : 2 * k0;
       } else {
         // general form: any number of E4M3 candidates, scales far below the block maximum, and the
         // coupled arm of Sec. 3.2, where each E4M3 candidate rounds the block with its own value
