@@ -370,6 +370,20 @@ def run_ours(args):
     extra["dequant_error"] = dict(ms_per_step=err_ms, achieved_gbs=err_bytes / (err_ms * 1e-3) / 1e9,
                                   frac_of_measured_hbm=err_bytes / (err_ms * 1e-3) / 1e9 / peaks["hbm_gbs"])
 
+    # ---- candidate-count sweep (config 5's purpose: where the search loop overtakes HBM); one iteration each
+    if args.sweep:
+        rows_out = []
+        for K in [int(x) for x in args.sweep.split(",")]:
+            n_dq = min(2, K)
+            c = api.soar_default_cfg(api.PRESET_SINGLE_PASS, n_dq=n_dq, n_beta=max(1, K // n_dq))
+            k_ms, _ = timed(lambda: step(c), max(args.steps, 5), 3, trace=False)
+            k_bytes = elements * call_bytes_per_elem(c, 1)
+            rows_out.append(dict(pairs=c.n_dq * c.n_beta, n_beta=c.n_beta, n_dq=c.n_dq, ms_per_step=k_ms,
+                                 value=world * 2.0 * elements / (k_ms * 1e-3) / 1e9, unit="GB/s",
+                                 achieved_gbs=k_bytes / (k_ms * 1e-3) / 1e9,
+                                 frac_of_measured_hbm=k_bytes / (k_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]))
+        extra["sweep"] = rows_out
+
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region
     import ctypes
     ctypes_sizeof_result = ctypes.sizeof(api.SoarResult)
@@ -457,6 +471,7 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=128, help="rows per step of the reference arm")
     ap.add_argument("--pairs", type=int, default=0, help="candidate pairs per block (overrides the preset's grid)")
     ap.add_argument("--iters", type=int, default=None, help="iterations T, early stop off (overrides the preset)")
+    ap.add_argument("--sweep", default="", help="comma-separated candidate-pair counts to time, one iteration each")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-single-pass", action="store_true")
