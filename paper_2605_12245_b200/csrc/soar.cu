@@ -357,7 +357,7 @@ __device__ __forceinline__ void make_fixed(const Block& blk, Fixed& fx) {
   for (int i = 0; i < 8; ++i) {
     const unsigned int lo = __float_as_uint(__fmaf_rn(fabsf(blk.w[2 * i]), S, 8388608.0f));
     const unsigned int hi = __float_as_uint(__fmaf_rn(fabsf(blk.w[2 * i + 1]), S, 8388608.0f));
-    fx.pair[i] = (lo & 0xFFFFu) | (hi << 16);
+    fx.pair[i] = __byte_perm(lo, hi, 0x5410);   // low halves of lo and hi side by side
   }
 }
 
@@ -510,13 +510,17 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(Params p, int reverse) {
     const unsigned int b = tile_of(p, n, reverse) * kTile + threadIdx.x;
     if (b >= p.nblk) continue;
     const unsigned int u[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-    unsigned int bmx = 0, bmn = 0x7FFF7FFFu;
+    // largest and smallest magnitude of the block with packed bf16 min/max (a NaN input comes out
+    // of the maximum as NaN, whose bits are above the infinity pattern)
+    unsigned int bmx = 0, bmn = 0x7F7F7F7Fu;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const unsigned int m = u[i] & 0x7FFF7FFFu;
-      bmx = __vmaxu2(bmx, m);
-      bmn = __vminu2(bmn, m);
+      unsigned int m;
+      asm("abs.bf16x2 %0, %1;" : "=r"(m) : "r"(u[i]));
+      asm("max.NaN.bf16x2 %0, %0, %1;" : "+r"(bmx) : "r"(m));
+      asm("min.bf16x2 %0, %0, %1;" : "+r"(bmn) : "r"(m));
     }
+    bmx &= 0x7FFF7FFFu;
     mx = __vmaxu2(mx, bmx);
     // a magnitude below 0x0080 has a zero exponent field: zero or subnormal
     if (min(bmn & 0xFFFFu, bmn >> 16) >= 0x80u) sumsq_block<false>(u, sq[0], sq[1]);
