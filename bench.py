@@ -124,9 +124,9 @@ def kernel_bytes_per_elem(name: str, cfg, t: int = 0) -> float:
 # proportion to the elements, so a launch's traffic is this figure times its elements.  The figures
 # belong to one version of the kernels: they are dropped when the kernel source no longer matches.
 NCU_TRAFFIC = {
-    "kernel_source_sha256_16": "142b88b6407ddaf7",
-    "bytes_per_elem": {"amax_kernel": 2.02, "init_kernel": 2.43, "iterate_kernel/single": 3.00,
-                       "iterate_kernel/grid": 3.44},
+    "kernel_source_sha256_16": "c2f1a82793df3685",
+    "bytes_per_elem": {"amax_kernel": 2.02, "init_kernel": 2.44, "iterate_kernel/single": 3.00,
+                       "iterate_kernel/grid": 3.45},
 }
 
 
@@ -467,8 +467,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config4")
     ap.add_argument("--preset", default="paper", choices=["paper", "single_pass"])
-    ap.add_argument("--cpu-rows", type=int, default=256, help="rows of tensor 0 the CPU baseline quantizes")
-    ap.add_argument("--ref-rows", type=int, default=128, help="rows per step of the reference arm")
+    ap.add_argument("--cpu-rows", type=int, default=4096, help="rows of tensor 0 the CPU baseline quantizes")
+    ap.add_argument("--ref-rows", type=int, default=1024, help="rows per step of the reference arm")
     ap.add_argument("--pairs", type=int, default=0, help="candidate pairs per block (overrides the preset's grid)")
     ap.add_argument("--iters", type=int, default=None, help="iterations T, early stop off (overrides the preset)")
     ap.add_argument("--sweep", default="", help="comma-separated candidate-pair counts to time, one iteration each")
