@@ -95,7 +95,7 @@ def ref_cfg_of(R, cfg):
                     n_beta=cfg.n_beta, beta_step_pct=cfg.beta_step_pct)
 
 
-# Algorithmic work per 16-element block (what the method itself demands)
+# Algorithmic work per 16-element block: what the method itself demands, not what a kernel happens to execute
 def iterate_ops_per_block(cfg) -> float:
     return cfg.n_beta * (16 * OPS_PER_ELEMENT_EVAL + cfg.n_dq * OPS_PER_PAIR_SCORE)
 
