@@ -92,7 +92,7 @@ def preset_cfg(api, preset: str, args=None, **over):
 
 def ref_cfg_of(R, cfg):
     return R.RefCfg(max_iters=cfg.max_iters, early_stop_rel=cfg.early_stop_rel, n_dq=cfg.n_dq,
-                    n_beta=cfg.n_beta, beta_step_pct=cfg.beta_step_pct)
+                    n_beta=cfg.n_beta, beta_step_pct=cfg.beta_step_pct, flags=cfg.flags)
 
 
 # Algorithmic work per 16-element block: what the method itself demands, not what a kernel happens to execute
@@ -269,6 +269,27 @@ def run_ours(args):
         for W, o in zip(dev_w, outs):
             api.soar_quantize(W, c, o, stream)
 
+    if args.graph:
+        # replay the step's launches from a CUDA graph: takes the host's launch cost out of the picture
+        side = torch.cuda.Stream()
+        graphs = {}
+
+        def graphed(c):
+            key = (c.max_iters, c.n_beta, c.n_dq, c.early_stop_rel)
+            if key not in graphs:
+                g = torch.cuda.CUDAGraph()
+                torch.cuda.synchronize()
+                with torch.cuda.graph(g, stream=side):
+                    for W, o in zip(dev_w, outs):
+                        api.soar_quantize(W, c, o, side)
+                graphs[key] = g
+            return graphs[key]
+
+        eager_step = step
+
+        def step(c=cfg):  # noqa: F811
+            graphed(c).replay()
+
     def barrier():
         torch.cuda.synchronize()
         if world > 1:
@@ -297,7 +318,7 @@ def run_ours(args):
     # headline: K steps with nothing between the kernels; then the same K steps again with an
     # event pair around every kernel (which costs a few microseconds per launch) for the shares
     ms, _ = timed(step, args.steps, args.warmup, trace=False)
-    traced_ms, trace = timed(step, args.steps, 0, trace=True)
+    traced_ms, trace = timed(eager_step if args.graph else step, args.steps, 0, trace=True)
     clocks = sampler.stop()
     results = [o.read_result() for o in outs]
     iters = [r.iters_run for r in results]
@@ -345,7 +366,7 @@ def run_ours(args):
     if args.preset == "paper" and not args.no_single_pass:
         sp = preset_cfg(api, "single_pass")
         sp_ms, _ = timed(lambda: step(sp), max(args.steps, 5), 3, trace=False)
-        _, sp_tr = timed(lambda: step(sp), max(args.steps, 5), 0, trace=True)
+        _, sp_tr = timed(lambda: (eager_step if args.graph else step)(sp), max(args.steps, 5), 0, trace=True)
         sp_bytes = elements * call_bytes_per_elem(sp, sp.max_iters)
         gbs = sp_bytes / (sp_ms * 1e-3) / 1e9
         extra["single_pass"] = dict(
@@ -452,7 +473,7 @@ def run_ours(args):
                         parallelism=f"{world} rank(s), one layer of these shapes each, no collective"),
             elements_per_s=world * elements / (ms * 1e-3),
             hbm_frac_end_to_end_of_measured=value / peaks["hbm_gbs"],
-            traced_ms_per_step=traced_ms, roofline=roofline, kernels=kernels, cpu_baseline=cpu, e2e=e2e, gpu_launches=launches,
+            traced_ms_per_step=traced_ms, cuda_graph=bool(args.graph), roofline=roofline, kernels=kernels, cpu_baseline=cpu, e2e=e2e, gpu_launches=launches,
             clocks=clocks, **extra)
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -472,6 +493,7 @@ def main():
     ap.add_argument("--pairs", type=int, default=0, help="candidate pairs per block (overrides the preset's grid)")
     ap.add_argument("--iters", type=int, default=None, help="iterations T, early stop off (overrides the preset)")
     ap.add_argument("--sweep", default="", help="comma-separated candidate-pair counts to time, one iteration each")
+    ap.add_argument("--graph", action="store_true", help="replay each step from a CUDA graph (no per-kernel trace)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-single-pass", action="store_true")
