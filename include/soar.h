@@ -138,6 +138,33 @@ int soar_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld,
                   void* out_e4m3_scales_sw, float* out_global_fp32, void* workspace,
                   size_t workspace_bytes, soar_result* out_result, void* stream);
 
+/* One matrix of a batch: the arguments of soar_quantize that differ per matrix. */
+typedef struct soar_tensor_desc {
+  const void* W_bf16;        /* device, rows x cols bf16, row stride ld                       */
+  int64_t rows, cols, ld;
+  void* out_fp4_packed;      /* device, rows*cols/2 bytes                                     */
+  void* out_e4m3_scales;     /* device, rows*cols/16 bytes, or NULL (see soar_quantize)       */
+  void* out_e4m3_scales_sw;  /* device, soar_swizzled_scale_bytes(), or NULL                  */
+  float* out_global_fp32;    /* device, one float                                             */
+  soar_result* out_result;   /* device, or NULL                                               */
+} soar_tensor_desc;
+
+/* Bytes of device scratch soar_quantize_batch needs: the sum of soar_workspace_bytes over the
+ * matrices (0 on bad arguments). */
+size_t soar_batch_workspace_bytes(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg);
+
+/*
+ * Algorithm 1 on n independent matrices with shared settings; every matrix gets exactly the
+ * outputs soar_quantize would give it.  The matrices' tiles are walked as one sequence by the
+ * same kernels (up to 16 matrices per launch), so a model's many small matrices cost a few
+ * launches per group instead of a few per matrix; matrices that stop early (Sec. 4.1) drop
+ * out of later iterations on their own.  `tensors` is host memory (n descriptors, read before
+ * the call returns); `workspace` is device scratch of soar_batch_workspace_bytes(), 256-byte
+ * aligned.  Argument errors of any matrix are returned before anything is enqueued.
+ */
+int soar_quantize_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void* workspace,
+                        size_t workspace_bytes, void* stream);
+
 /* Device staging buffers for soar_quantize_host (all device memory, caller-owned, same sizes
  * and alignment as the matching soar_quantize arguments; W holds rows*ld bf16 elements). */
 typedef struct soar_staging {

@@ -27,6 +27,7 @@ EXPORTS = (
     "soar_default_cfg", "soar_workspace_bytes", "soar_swizzled_scale_bytes", "soar_quantize",
     "soar_dequant_error", "soar_quantize_launches", "soar_status_string", "soar_quantize_host",
     "soar_trace_begin", "soar_trace_end", "soar_quantize_static", "soar_selftest_reciprocal",
+    "soar_batch_workspace_bytes", "soar_quantize_batch",
 )
 
 
@@ -48,6 +49,16 @@ class SoarResult(C.Structure):
         ("sse", C.c_double), ("sse_init", C.c_double), ("sumsq", C.c_double),
         ("zero_blocks", C.c_int64), ("wide_candidates", C.c_int64),
         ("trace_alpha", C.c_double * (MAX_ITERS + 1)), ("trace_sse", C.c_double * (MAX_ITERS + 1)),
+    ]
+
+
+class SoarTensorDesc(C.Structure):
+    """Mirror of ``soar_tensor_desc``."""
+
+    _fields_ = [
+        ("W_bf16", C.c_void_p), ("rows", C.c_int64), ("cols", C.c_int64), ("ld", C.c_int64),
+        ("out_fp4_packed", C.c_void_p), ("out_e4m3_scales", C.c_void_p), ("out_e4m3_scales_sw", C.c_void_p),
+        ("out_global_fp32", C.c_void_p), ("out_result", C.c_void_p),
     ]
 
 
@@ -100,6 +111,10 @@ def lib() -> C.CDLL:
                                          C.POINTER(SoarStaging), vp]
         L.soar_quantize_static.restype = C.c_int
         L.soar_quantize_static.argtypes = [vp, i64, i64, i64, C.POINTER(SoarCfg), vp, vp, vp, vp, vp, vp]
+        L.soar_batch_workspace_bytes.restype = C.c_size_t
+        L.soar_batch_workspace_bytes.argtypes = [C.POINTER(SoarTensorDesc), C.c_int, C.POINTER(SoarCfg)]
+        L.soar_quantize_batch.restype = C.c_int
+        L.soar_quantize_batch.argtypes = [C.POINTER(SoarTensorDesc), C.c_int, C.POINTER(SoarCfg), vp, C.c_size_t, vp]
         L.soar_selftest_reciprocal.restype = C.c_int
         L.soar_selftest_reciprocal.argtypes = [C.c_int, C.c_int, vp, vp]
         L.soar_trace_begin.restype = C.c_int
@@ -204,6 +219,39 @@ def soar_quantize(W: torch.Tensor, cfg: SoarCfg, out: QuantBuffers | None = None
         _ptr(out.result), _stream_ptr(stream))
     _check(rc, "soar_quantize")
     return out
+
+
+def _descs(Ws, outs):
+    d = (SoarTensorDesc * len(Ws))()
+    for i, (W, o) in enumerate(zip(Ws, outs)):
+        _require_cuda(W, o.packed, o.scales, o.scales_sw, o.alpha, o.result)
+        if W.dtype != torch.bfloat16 or W.dim() != 2 or W.stride(1) != 1:
+            raise SoarError("W must be a 2-D bf16 tensor with unit column stride")
+        nul = lambda t: None if t is None else t.data_ptr()  # noqa: E731
+        d[i] = SoarTensorDesc(W.data_ptr(), W.shape[0], W.shape[1], W.stride(0), o.packed.data_ptr(),
+                              nul(o.scales), nul(o.scales_sw), o.alpha.data_ptr(), nul(o.result))
+    return d
+
+
+def soar_batch_workspace_bytes(Ws, outs, cfg: SoarCfg) -> int:
+    d = _descs(Ws, outs)
+    return int(lib().soar_batch_workspace_bytes(d, len(Ws), C.byref(cfg)))
+
+
+def soar_quantize_batch(Ws, cfg: SoarCfg, outs, workspace: torch.Tensor | None = None, stream=None):
+    """Enqueue ``soar_quantize_batch`` for a list of bf16 CUDA matrices; ``outs`` are their
+    ``QuantBuffers`` (their own ``workspace`` fields are not used), ``workspace`` one uint8 CUDA
+    tensor of ``soar_batch_workspace_bytes`` (allocated here when omitted).  Returns it."""
+    d = _descs(Ws, outs)
+    if workspace is None:
+        need = int(lib().soar_batch_workspace_bytes(d, len(Ws), C.byref(cfg)))
+        if need == 0:
+            raise SoarError("soar_batch_workspace_bytes rejected the shapes or cfg")
+        workspace = torch.empty(need, dtype=torch.uint8, device=Ws[0].device)
+    _require_cuda(workspace)
+    rc = lib().soar_quantize_batch(d, len(Ws), C.byref(cfg), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    _check(rc, "soar_quantize_batch")
+    return workspace
 
 
 STATIC_MAX_ELEMENTS = 1 << 24

@@ -77,6 +77,17 @@ struct Params {
   int flags;           // SOAR_FLAG_* bits
 };
 
+// One launch works on up to kMaxBatch tensors: their tiles form one sequence (tensor 0's tiles,
+// then tensor 1's, ...), which the CTAs of the persistent grid walk together.
+constexpr int kMaxBatch = 16;
+struct Batch {
+  int n;
+  unsigned int total_tiles;
+  unsigned int tile_end[kMaxBatch];   // running sum of the tensors' tile counts
+  Params t[kMaxBatch];
+};
+static_assert(sizeof(Batch) <= 3072, "kernel parameter block too large");
+
 // ------------------------------------------------------------------ number formats
 
 __device__ __forceinline__ float bits_to_mag(unsigned int bf16_bits) {
@@ -184,6 +195,8 @@ struct __align__(128) Ring {
   unsigned char tile[kStages][kTileBytes];
   unsigned long long full[kStages];    // producer -> consumers: the stage's bytes have landed
   unsigned long long empty[kStages];   // consumers -> producer: every consumer has read the stage
+  int meta_tensor[kStages];            // tensor the stage's tile belongs to; -1 ends the sequence
+  unsigned int meta_tile[kStages];     // and which of its tiles
   int fail;
 };
 
@@ -193,11 +206,13 @@ struct __align__(128) RingWithState {
   unsigned char state[kStages][kTile * 8];
   unsigned long long full[kStages];
   unsigned long long empty[kStages];
+  int meta_tensor[kStages];
+  unsigned int meta_tile[kStages];
   int fail;
 };
 
-// Thread 0: start the copies of tile `tile` into stage `s` (one copy when rows are
-// contiguous, else one per row segment) and arm the stage's barrier with the byte count.
+// Producer: start the copies of tile `tile` of tensor `p` into stage `s` (one copy when rows
+// are contiguous, else one per row segment) and arm the stage's barrier with the byte count.
 template <typename R>
 __device__ __forceinline__ void ring_issue(R& ring, const Params& p, unsigned int tile, int s) {
   const unsigned int b0 = tile * kTile;
@@ -227,15 +242,16 @@ __device__ __forceinline__ void ring_issue(R& ring, const Params& p, unsigned in
   }
 }
 
-// Order in which a CTA visits its tiles: n-th tile of this CTA, forward or from the end.
-// Consecutive passes alternate direction so that a pass starts on what the previous pass
-// left in L2.
-__device__ __forceinline__ unsigned int tile_of(const Params& p, unsigned int n, int reverse) {
-  const unsigned int t = blockIdx.x + n * gridDim.x;
-  return reverse ? p.ntiles - 1 - t : t;
-}
-__device__ __forceinline__ unsigned int tiles_of_cta(const Params& p) {
-  return blockIdx.x < p.ntiles ? (p.ntiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+// Tensor and tile-within-tensor of position g of the batch's tile sequence.
+__device__ __forceinline__ int tensor_of(const Batch& bt, unsigned int g, unsigned int& tile) {
+  int ti = 0;
+  unsigned int base = 0;
+  while (g >= bt.tile_end[ti]) {
+    base = bt.tile_end[ti];
+    ++ti;
+  }
+  tile = g - base;
+  return ti;
 }
 
 // All threads: barriers ready before anyone uses them.
@@ -254,46 +270,72 @@ __device__ __forceinline__ void ring_init(R& ring) {
 
 __device__ __forceinline__ bool is_producer_warp() { return threadIdx.x >= kTile; }
 
-// Producer (one thread): walks the CTA's tile sequence, refilling a stage as soon as every
-// consumer has handed it back.  A wait that gives up records the failure, lets copies still
-// in flight land (bounded) and ends the sequence; the consumers then give up on their own.
+__device__ __forceinline__ void record_failure(const Batch& bt) {
+  for (int i = 0; i < bt.n; ++i)
+    if (bt.t[i].ws != nullptr) atomicOr(&bt.t[i].ws->error, 1u);
+}
+
+// Producer (one thread): walks the CTA's share of the tile sequence (positions blockIdx.x,
+// + gridDim.x, ..., from the front or, for `reverse`, from the back: consecutive passes
+// alternate so that a pass starts on what the previous one left in L2), skipping tensors
+// whose bit in `run_mask` is clear, and refills a stage as soon as every consumer has handed it
+// back.  After the last tile it posts an end marker.  A wait that gives up records the
+// failure, lets copies still in flight land (bounded) and ends the sequence; the consumers
+// then give up on their own.
 template <typename R>
-__device__ __forceinline__ void ring_produce(R& ring, const Params& p, int reverse) {
-  const unsigned int ntc = tiles_of_cta(p);
+__device__ __forceinline__ void ring_produce(R& ring, const Batch& bt, int reverse, unsigned int run_mask) {
   unsigned int n = 0;
   bool ok = true;
-  for (; n < ntc; ++n) {
+  for (unsigned int g0 = blockIdx.x; g0 < bt.total_tiles; g0 += gridDim.x) {
+    unsigned int tile;
+    const int ti = tensor_of(bt, reverse ? bt.total_tiles - 1 - g0 : g0, tile);
+    if (!((run_mask >> ti) & 1u)) continue;
     const int s = static_cast<int>(n % kStages);
     if (n >= static_cast<unsigned int>(kStages)) ok = mbar_wait(&ring.empty[s], (n / kStages - 1) & 1u);
-    if (!ok || *static_cast<volatile int*>(&ring.fail)) break;
-    ring_issue(ring, p, tile_of(p, n, reverse), s);
+    if (!ok || *static_cast<volatile int*>(&ring.fail)) { ok = false; break; }
+    ring.meta_tensor[s] = ti;
+    ring.meta_tile[s] = tile;
+    ring_issue(ring, bt.t[ti], tile, s);
+    ++n;
   }
-  if (n < ntc) {
+  if (ok) {   // end marker: completes the stage's phase with no bytes
+    const int s = static_cast<int>(n % kStages);
+    if (n >= static_cast<unsigned int>(kStages)) ok = mbar_wait(&ring.empty[s], (n / kStages - 1) & 1u);
+    if (ok) {
+      ring.meta_tensor[s] = -1;
+      mbar_arrive(&ring.full[s]);
+    }
+  }
+  if (!ok) {
     *static_cast<volatile int*>(&ring.fail) = 1;
-    if (p.ws != nullptr) atomicOr(&p.ws->error, 1u);
+    record_failure(bt);
     for (unsigned int m = (n > static_cast<unsigned int>(kStages) ? n - kStages : 0); m < n; ++m)
       (void)mbar_wait(&ring.full[m % kStages], (m / kStages) & 1u);
   }
 }
 
-// Consumer: this thread's 32 bytes (and block state) of the CTA's n-th tile, then the stage
-// is handed back.  Returns false when the wait gave up; the caller leaves its tile loop.
+// Consumer: the CTA's n-th stage.  Returns 0 with this thread's 32 bytes (and block state), the
+// tile's tensor and its number, the stage handed back; 1 at the end marker; 2 when the wait
+// gave up.  On 1 and 2 the caller leaves its tile loop.
 template <typename R>
-__device__ __forceinline__ bool ring_consume(R& ring, const Params& p, unsigned int n, uint4& v0, uint4& v1,
-                                             uint2* st = nullptr) {
+__device__ __forceinline__ int ring_consume(R& ring, const Batch& bt, unsigned int n, uint4& v0, uint4& v1,
+                                            int& ti, unsigned int& tile, uint2* st = nullptr) {
   const int s = static_cast<int>(n % kStages);
-  // the outcome is made the same for the whole warp: callers vote across the warp later
+  // the outcome is made the same for the whole warp
   if (!__all_sync(0xFFFFFFFFu, mbar_wait(&ring.full[s], (n / kStages) & 1u))) {
     *static_cast<volatile int*>(&ring.fail) = 1;
-    if (p.ws != nullptr) atomicOr(&p.ws->error, 1u);
-    return false;
+    record_failure(bt);
+    return 2;
   }
+  ti = ring.meta_tensor[s];
+  if (ti < 0) return 1;
+  tile = ring.meta_tile[s];
   const uint4* src = reinterpret_cast<const uint4*>(ring.tile[s] + threadIdx.x * 32);
   v0 = src[0];
   v1 = src[1];
   if constexpr (sizeof(R) == sizeof(RingWithState)) *st = reinterpret_cast<const uint2*>(ring.state[s])[threadIdx.x];
   mbar_arrive(&ring.empty[s]);
-  return true;
+  return 0;
 }
 
 // ------------------------------------------------------------------ block helpers
@@ -435,26 +477,40 @@ __device__ __forceinline__ double warp_sum(double v) {
   return v;
 }
 
-// CTA-wide sums of N doubles, then one atomicAdd each from thread 0.
+// Per-tensor partial sums of a CTA, in shared memory.  Each consumer warp adds its sums for a
+// tensor once (when the CTA's tile sequence leaves the tensor, or ends); the warp that arrives
+// last forwards the CTA's total to the tensor's global accumulators, one atomicAdd each.  No
+// CTA-wide barrier is involved.
 template <int N>
-__device__ __forceinline__ void cta_accumulate(double (&v)[N], double* const (&dst)[N]) {
-  __shared__ double red[N][kThreads / 32];
-  const int nwarp = blockDim.x >> 5;
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+struct Slots {
+  double acc[kMaxBatch][N];
+  unsigned int count[kMaxBatch];
+};
+
+// All threads, before the tile loop (a __syncthreads follows in ring_init).
+template <int N>
+__device__ __forceinline__ void slots_clear(Slots<N>& sl) {
+  for (int i = threadIdx.x; i < kMaxBatch * N; i += blockDim.x) (&sl.acc[0][0])[i] = 0.0;
+  for (int i = threadIdx.x; i < kMaxBatch; i += blockDim.x) sl.count[i] = 0;
+}
+
+// Whole consumer warp: adds v[] for tensor `ti` and clears it.
+template <int N>
+__device__ __forceinline__ void slots_add(Slots<N>& sl, int ti, double (&v)[N], double* const (&dst)[N]) {
 #pragma unroll
-  for (int i = 0; i < N; ++i) {
-    double s = warp_sum(v[i]);
-    if (lane == 0) red[i][wid] = s;
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
+  for (int i = 0; i < N; ++i) v[i] = warp_sum(v[i]);
+  if ((threadIdx.x & 31) == 0) {
 #pragma unroll
-    for (int i = 0; i < N; ++i) {
-      double s = 0.0;
-      for (int w = 0; w < nwarp; ++w) s += red[i][w];
-      if (dst[i] != nullptr) atomicAdd(dst[i], s);
+    for (int i = 0; i < N; ++i) atomicAdd(&sl.acc[ti][i], v[i]);
+    __threadfence_block();
+    if (atomicAdd(&sl.count[ti], 1u) == kTile / 32 - 1) {
+      __threadfence_block();
+#pragma unroll
+      for (int i = 0; i < N; ++i) atomicAdd(dst[i], atomicAdd(&sl.acc[ti][i], 0.0));
     }
   }
+#pragma unroll
+  for (int i = 0; i < N; ++i) v[i] = 0.0;
 }
 
 // Data-dependent status from the tensor maximum (bf16 magnitude bits).
@@ -497,18 +553,39 @@ __device__ __forceinline__ void sumsq_block(const unsigned int (&u)[8], double& 
 }
 
 // Eq. 1's tensor maximum, plus sum W^2 (binary64) for the error report.
-__global__ void __launch_bounds__(kThreads) amax_kernel(Params p, int reverse) {
+__global__ void __launch_bounds__(kThreads) amax_kernel(const __grid_constant__ Batch bt, int reverse) {
   __shared__ Ring ring;
+  __shared__ Slots<1> slots;
+  slots_clear(slots);
   ring_init(ring);
-  const unsigned int ntc = is_producer_warp() ? 0u : tiles_of_cta(p);
-  if (threadIdx.x == kTile) ring_produce(ring, p, reverse);
+  if (is_producer_warp()) {
+    if (threadIdx.x == kTile) ring_produce(ring, bt, reverse, 0xFFFFFFFFu);
+    return;
+  }
   unsigned int mx = 0;
   double sq[2] = {0.0, 0.0};
-  for (unsigned int n = 0; n < ntc; ++n) {
+  int cur = -1;
+  for (unsigned int n = 0;; ++n) {
     uint4 v0, v1;
-    if (!ring_consume(ring, p, n, v0, v1)) break;
-    const unsigned int b = tile_of(p, n, reverse) * kTile + threadIdx.x;
-    if (b >= p.nblk) continue;
+    int ti = -1;
+    unsigned int tile = 0;
+    const int rc = ring_consume(ring, bt, n, v0, v1, ti, tile);
+    if (rc != 0 || ti != cur) {
+      if (cur >= 0) {   // leaving tensor `cur`: hand over its maximum and sum
+        mx = max(mx & 0xFFFFu, mx >> 16);
+        mx = __reduce_max_sync(0xFFFFFFFFu, mx);
+        if ((threadIdx.x & 31) == 0 && mx) atomicMax(&bt.t[cur].ws->amax_bits, mx);
+        double acc[1] = {(sq[0] + sq[1]) * 0x1p256};   // undo the 2^-128 scaling of the values
+        double* const dst[1] = {&bt.t[cur].ws->sumsq};
+        slots_add(slots, cur, acc, dst);
+        mx = 0;
+        sq[0] = sq[1] = 0.0;
+      }
+      if (rc != 0) break;
+      cur = ti;
+    }
+    const unsigned int b = tile * kTile + threadIdx.x;
+    if (b >= bt.t[ti].nblk) continue;
     const unsigned int u[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
     // largest and smallest magnitude of the block with packed bf16 min/max (a NaN input comes out
     // of the maximum as NaN, whose bits are above the infinity pattern)
@@ -526,34 +603,63 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(Params p, int reverse) {
     if (min(bmn & 0xFFFFu, bmn >> 16) >= 0x80u) sumsq_block<false>(u, sq[0], sq[1]);
     else sumsq_block<true>(u, sq[0], sq[1]);
   }
-  mx = max(mx & 0xFFFFu, mx >> 16);
-  mx = __reduce_max_sync(0xFFFFFFFFu, mx);
-  if ((threadIdx.x & 31) == 0 && mx) atomicMax(&p.ws->amax_bits, mx);
-  double acc[1] = {(sq[0] + sq[1]) * 0x1p256};   // undo the 2^-128 scaling of the values
-  double* const dst[1] = {&p.ws->sumsq};
-  cta_accumulate<1>(acc, dst);
+}
+
+// Warp-level hand-over of two counters to a tensor's workspace.
+__device__ __forceinline__ void add_counters(Ws* ws, unsigned int& zeros, unsigned int& wide) {
+  zeros = __reduce_add_sync(0xFFFFFFFFu, zeros);
+  wide = __reduce_add_sync(0xFFFFFFFFu, wide);
+  if ((threadIdx.x & 31) == 0) {
+    if (zeros) atomicAdd(&ws->zero_blocks, static_cast<unsigned long long>(zeros));
+    if (wide) atomicAdd(&ws->wide, static_cast<unsigned long long>(wide));
+  }
+  zeros = wide = 0;
 }
 
 // Algorithm 1 "Initialization" (Eq. 1): alpha0 = amax/(6*448), dd0 = E4M3(bmax/(6 alpha0)),
 // dq0 = dd0; first codes (Eq. 2); stage-0 sums for Eq. 5 and the starting error.  Codes and
-// scales are written here only when no iteration follows (final != 0).
-__global__ void __launch_bounds__(kThreads) init_kernel(Params p, int reverse, int final) {
+// scales are written here only when no iteration follows (final != 0).  Tensors with
+// non-finite or out-of-range input are skipped.
+__global__ void __launch_bounds__(kThreads) init_kernel(const __grid_constant__ Batch bt, int reverse, int final) {
   __shared__ Ring ring;
-  const unsigned int amax_bits = p.ws->amax_bits;
-  const int st = status_from_amax(amax_bits);
-  if (st & (SOAR_STATUS_NONFINITE | SOAR_STATUS_RANGE)) return;
+  __shared__ Slots<3> slots;
+  slots_clear(slots);
   ring_init(ring);
-  const unsigned int ntc = is_producer_warp() ? 0u : tiles_of_cta(p);
-  if (threadIdx.x == kTile) ring_produce(ring, p, reverse);
-  const float alpha = (st & SOAR_STATUS_ZERO_TENSOR) ? 1.0f : __fdiv_rn(bits_to_mag(amax_bits), 2688.0f);
-  const float six_alpha = __fmul_rn(alpha, 6.0f);
-  const double alpha_d = static_cast<double>(alpha);
+  if (is_producer_warp()) {
+    if (threadIdx.x == kTile) {
+      unsigned int run = 0;
+      for (int i = 0; i < bt.n; ++i)
+        if (!(status_from_amax(bt.t[i].ws->amax_bits) & (SOAR_STATUS_NONFINITE | SOAR_STATUS_RANGE))) run |= 1u << i;
+      ring_produce(ring, bt, reverse, run);
+    }
+    return;
+  }
+  float alpha = 1.0f, six_alpha = 6.0f;
+  double alpha_d = 1.0;
   double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum
   unsigned int zeros = 0, wide = 0;
-  for (unsigned int n = 0; n < ntc; ++n) {
+  int cur = -1;
+  for (unsigned int n = 0;; ++n) {
     uint4 v0, v1;
-    if (!ring_consume(ring, p, n, v0, v1)) break;
-    const unsigned int b = tile_of(p, n, reverse) * kTile + threadIdx.x;
+    int ti = -1;
+    unsigned int tile = 0;
+    const int rc = ring_consume(ring, bt, n, v0, v1, ti, tile);
+    if (rc != 0 || ti != cur) {
+      if (cur >= 0) {
+        Ws* ws = bt.t[cur].ws;
+        double* const dst[3] = {&ws->num[0], &ws->den[0], &ws->gsum[0]};
+        slots_add(slots, cur, acc, dst);
+        add_counters(ws, zeros, wide);
+      }
+      if (rc != 0) break;
+      cur = ti;
+      const unsigned int amax_bits = bt.t[ti].ws->amax_bits;
+      alpha = amax_bits == 0 ? 1.0f : __fdiv_rn(bits_to_mag(amax_bits), 2688.0f);
+      six_alpha = __fmul_rn(alpha, 6.0f);
+      alpha_d = static_cast<double>(alpha);
+    }
+    const Params& p = bt.t[ti];
+    const unsigned int b = tile * kTile + threadIdx.x;
     if (b >= p.nblk) continue;
     Block blk;
     unpack_block(v0, v1, blk);
@@ -589,12 +695,6 @@ __global__ void __launch_bounds__(kThreads) init_kernel(Params p, int reverse, i
     acc[1] = fma(B * vd, vd, acc[1]);
     acc[2] += sd * fma(sd, B, -2.0 * A);
   }
-  double* const dst[3] = {&p.ws->num[0], &p.ws->den[0], &p.ws->gsum[0]};
-  cta_accumulate<3>(acc, dst);
-  zeros = __reduce_add_sync(0xFFFFFFFFu, zeros);
-  if ((threadIdx.x & 31) == 0 && zeros) atomicAdd(&p.ws->zero_blocks, static_cast<unsigned long long>(zeros));
-  wide = __reduce_add_sync(0xFFFFFFFFu, wide);
-  if ((threadIdx.x & 31) == 0 && wide) atomicAdd(&p.ws->wide, static_cast<unsigned long long>(wide));
 }
 
 // Error of stage s (Eq. 4) from the tensor sums.
@@ -654,38 +754,60 @@ __device__ __forceinline__ int clip_code(int d) { return max(1, min(0x7E, d)); }
 // dequantization codes, whose passes are bound by HBM rather than by the candidate loop.
 template <bool kSingle>
 __global__ void __launch_bounds__(kThreads, kSingle ? 3 : 2)
-iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
+iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, int keep) {
   __shared__ RingWithState ring;
+  __shared__ Slots<3> slots;
   __shared__ float s_beta[kSingle ? 1 : SOAR_MAX_BETA];
-  __shared__ float s_alpha;
-  __shared__ int s_run;
-  if (threadIdx.x == 0) {
+  __shared__ float s_alpha[kMaxBatch];
+  __shared__ unsigned int s_run;
+  if (threadIdx.x == 0) s_run = 0;
+  __syncthreads();
+  if (threadIdx.x < bt.n) {   // per tensor: still running?  its alpha for this iteration
     float a;
     int run;
-    iteration_head(p, t, a, run);
-    s_alpha = a;
-    s_run = run;
+    iteration_head(bt.t[threadIdx.x], t, a, run);
+    s_alpha[threadIdx.x] = a;
+    if (run) atomicOr(&s_run, 1u << threadIdx.x);
   }
+  const int n_dq = bt.t[0].n_dq, n_beta = bt.t[0].n_beta;
   if (!kSingle) {
-    for (int k = threadIdx.x; k < p.n_beta; k += kThreads)
-      s_beta[k] = static_cast<float>((100.0 + static_cast<double>((k - p.n_beta / 2) * p.beta_step_pct)) / 100.0);
+    for (int k = threadIdx.x; k < n_beta; k += kThreads)
+      s_beta[k] = static_cast<float>((100.0 + static_cast<double>((k - n_beta / 2) * bt.t[0].beta_step_pct)) / 100.0);
   }
+  slots_clear(slots);
   __syncthreads();
-  if (!s_run) return;
+  if (s_run == 0) return;   // every tensor of the batch has stopped
   ring_init(ring);
-  const unsigned int ntc = is_producer_warp() ? 0u : tiles_of_cta(p);
-  if (threadIdx.x == kTile) ring_produce(ring, p, reverse);
-  const float alpha = s_alpha;
-  const double alpha_d = static_cast<double>(alpha);
-  const int n_dq = p.n_dq, n_beta = p.n_beta;
+  if (is_producer_warp()) {
+    if (threadIdx.x == kTile) ring_produce(ring, bt, reverse, s_run);
+    return;
+  }
+  float alpha = 1.0f;
+  double alpha_d = 1.0;
 
   double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum of stage t+1
-  unsigned int wide = 0;
-  for (unsigned int n = 0; n < ntc; ++n) {
+  unsigned int wide = 0, unused_zeros = 0;
+  int cur = -1;
+  for (unsigned int n = 0;; ++n) {
     uint4 v0, v1;
     uint2 st;
-    if (!ring_consume(ring, p, n, v0, v1, &st)) break;
-    const unsigned int b = tile_of(p, n, reverse) * kTile + threadIdx.x;
+    int ti = -1;
+    unsigned int tile = 0;
+    const int rc = ring_consume(ring, bt, n, v0, v1, ti, tile, &st);
+    if (rc != 0 || ti != cur) {
+      if (cur >= 0) {
+        Ws* ws = bt.t[cur].ws;
+        double* const dst[3] = {&ws->num[t + 1], &ws->den[t + 1], &ws->gsum[t + 1]};
+        slots_add(slots, cur, acc, dst);
+        add_counters(ws, unused_zeros, wide);
+      }
+      if (rc != 0) break;
+      cur = ti;
+      alpha = s_alpha[ti];
+      alpha_d = static_cast<double>(alpha);
+    }
+    const Params& p = bt.t[ti];
+    const unsigned int b = tile * kTile + threadIdx.x;
     if (b >= p.nblk || (st.y >> 16) == 0) continue;   // past the end, or an all-zero block: nothing to optimise
     Block blk;
     unpack_block(v0, v1, blk);
@@ -798,14 +920,20 @@ iterate_kernel(Params p, int t, int reverse, int emit, int keep) {
     acc[1] = fma(bestB * vd, vd, acc[1]);
     acc[2] += best;
   }
-  double* const dst[3] = {&p.ws->num[t + 1], &p.ws->den[t + 1], &p.ws->gsum[t + 1]};
-  cta_accumulate<3>(acc, dst);
-  wide = __reduce_add_sync(0xFFFFFFFFu, wide);
-  if ((threadIdx.x & 31) == 0 && wide) atomicAdd(&p.ws->wide, static_cast<unsigned long long>(wide));
 }
 
-// Replays the early-stop rule over the stage sums, writes alpha and the report.
-__global__ void __launch_bounds__(128) finalize_kernel(Params p, float* out_alpha, soar_result* res) {
+// Where each tensor of a batch wants its alpha and its report (report may be null).
+struct Reports {
+  float* alpha[kMaxBatch];
+  soar_result* result[kMaxBatch];
+};
+
+// Replays the early-stop rule over the stage sums, writes alpha and the report; one CTA per tensor.
+__global__ void __launch_bounds__(128) finalize_kernel(const __grid_constant__ Batch bt,
+                                                       const __grid_constant__ Reports rp) {
+  const Params& p = bt.t[blockIdx.x];
+  float* out_alpha = rp.alpha[blockIdx.x];
+  soar_result* res = rp.result[blockIdx.x];
   __shared__ double s_num[SOAR_MAX_ITERS + 1], s_den[SOAR_MAX_ITERS + 1], s_sse[SOAR_MAX_ITERS + 1];
   __shared__ double s_ta[SOAR_MAX_ITERS + 1];
   __shared__ int s_iters;
@@ -888,24 +1016,32 @@ __global__ void __launch_bounds__(256) swizzle_kernel(const uint8_t* lin, uint8_
 // bf16 values widened by bit placement (scaled by 2^-128, undone at the end) and the signed
 // E2M1 values read from a 16-entry table in shared memory.  A wait that gave up turns the
 // results into NaN.
-__global__ void __launch_bounds__(kThreads) dequant_error_kernel(Params p, const uint8_t* scales, int swizzled,
+__global__ void __launch_bounds__(kThreads) dequant_error_kernel(const __grid_constant__ Batch bt,
+                                                                 const uint8_t* scales, int swizzled,
                                                                  unsigned int col_tiles, const float* alpha_ptr,
                                                                  double* out_sse, double* out_sumsq) {
   __shared__ Ring ring;
+  __shared__ Slots<2> slots;
   __shared__ double s_q[16];
+  const Params& p = bt.t[0];
+  slots_clear(slots);
   if (threadIdx.x < 16) {
     const double mag = static_cast<double>(e2m1_code_value(threadIdx.x & 7u));
     s_q[threadIdx.x] = (threadIdx.x & 8u) ? -mag : mag;
   }
   ring_init(ring);
-  const unsigned int ntc = is_producer_warp() ? 0u : tiles_of_cta(p);
-  if (threadIdx.x == kTile) ring_produce(ring, p, 0);
+  if (is_producer_warp()) {
+    if (threadIdx.x == kTile) ring_produce(ring, bt, 0, 1u);
+    return;
+  }
   const double alpha_scaled = static_cast<double>(*alpha_ptr) * 0x1p-128;
   double acc[2] = {0.0, 0.0};
-  for (unsigned int n = 0; n < ntc; ++n) {
+  for (unsigned int n = 0;; ++n) {
     uint4 v0, v1;
-    if (!ring_consume(ring, p, n, v0, v1)) break;
-    const unsigned int b = tile_of(p, n, 0) * kTile + threadIdx.x;
+    int ti;
+    unsigned int tile;
+    if (ring_consume(ring, bt, n, v0, v1, ti, tile) != 0) break;
+    const unsigned int b = tile * kTile + threadIdx.x;
     if (b >= p.nblk) continue;
     const uint2 cw = reinterpret_cast<const uint2*>(p.packed)[b];
     int dc;
@@ -942,7 +1078,7 @@ __global__ void __launch_bounds__(kThreads) dequant_error_kernel(Params p, const
   acc[0] = failed ? __longlong_as_double(0x7FF8000000000000ll) : acc[0] * 0x1p256;
   acc[1] = failed ? __longlong_as_double(0x7FF8000000000000ll) : acc[1] * 0x1p256;
   double* const dst[2] = {out_sse, out_sumsq};
-  cta_accumulate<2>(acc, dst);
+  slots_add(slots, 0, acc, dst);
 }
 
 // Counts the binary32 inputs with biased exponent lo_exp..hi_exp (all 2^23 significands each)
@@ -1012,13 +1148,12 @@ int sm_count() {
 // Grid of a persistent kernel: every SM filled to the kernel's occupancy, never more CTAs
 // than tiles.
 template <typename K>
-unsigned int persistent_grid(K kernel, unsigned int nblk, int threads) {
+unsigned int persistent_grid(K kernel, unsigned int tiles, int threads) {
   int per_sm = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, 0) != cudaSuccess || per_sm <= 0)
     per_sm = 2;
-  const unsigned long long cap = static_cast<unsigned long long>(sm_count()) * per_sm;
-  const unsigned long long need = (static_cast<unsigned long long>(nblk) + kTile - 1) / kTile;
-  return static_cast<unsigned int>(need < cap ? (need ? need : 1) : cap);
+  const unsigned int cap = static_cast<unsigned int>(sm_count() * per_sm);
+  return tiles < cap ? (tiles ? tiles : 1u) : cap;
 }
 
 size_t round256(size_t n) { return (n + 255) / 256 * 256; }
@@ -1106,92 +1241,149 @@ int soar_quantize_launches(const soar_cfg* cfg) {
   return 3 + cfg->max_iters + ((cfg->scale_layout & SOAR_SCALES_SWIZZLED) ? 1 : 0);
 }
 
+size_t soar_batch_workspace_bytes(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg) {
+  if (tensors == nullptr || n <= 0) return 0;
+  size_t total = 0;
+  for (int i = 0; i < n; ++i) {
+    const size_t b = soar_workspace_bytes(tensors[i].rows, tensors[i].cols, cfg);
+    if (b == 0) return 0;
+    total += b;
+  }
+  return total;
+}
+
+int soar_quantize_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+  int rc = check_cfg(cfg);
+  if (rc != SOAR_OK) return rc;
+  if (tensors == nullptr || n <= 0) return SOAR_ERR_INVALID_ARG;
+  const bool want_lin = (cfg->scale_layout & SOAR_SCALES_LINEAR) != 0;
+  const bool want_sw = (cfg->scale_layout & SOAR_SCALES_SWIZZLED) != 0;
+  for (int i = 0; i < n; ++i) {   // every argument is checked before anything is enqueued
+    const soar_tensor_desc& d = tensors[i];
+    rc = check_shape(d.W_bf16, d.rows, d.cols, d.ld);
+    if (rc != SOAR_OK) return rc;
+    if (d.out_fp4_packed == nullptr || d.out_global_fp32 == nullptr) return SOAR_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d.out_fp4_packed) % 16 != 0) return SOAR_ERR_UNSUPPORTED;
+    if (want_lin && d.out_e4m3_scales == nullptr) return SOAR_ERR_INVALID_ARG;
+    if (want_sw && d.out_e4m3_scales_sw == nullptr) return SOAR_ERR_INVALID_ARG;
+  }
+  const size_t need = soar_batch_workspace_bytes(tensors, n, cfg);
+  if (workspace == nullptr || need == 0 || workspace_bytes < need) return SOAR_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return SOAR_ERR_UNSUPPORTED;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // workspace: the n headers first (one memset clears them all), then each tensor's arrays
+  uint8_t* const headers = static_cast<uint8_t*>(workspace);
+  uint8_t* next = headers + static_cast<size_t>(n) * kWsFixedBytes;
+  if (cudaMemsetAsync(headers, 0, static_cast<size_t>(n) * kWsFixedBytes, st) != cudaSuccess) return SOAR_ERR_CUDA;
+
+  const bool single = cfg->n_beta == 1 && cfg->n_dq <= 2 && !(cfg->flags & SOAR_FLAG_COUPLED_SCALE);
+  const bool may_stop = cfg->early_stop_rel > 0.0f;
+  for (int first = 0; first < n; first += kMaxBatch) {
+    Batch bt;
+    Reports rp;
+    memset(&bt, 0, sizeof(bt));
+    memset(&rp, 0, sizeof(rp));
+    bt.n = (n - first < kMaxBatch) ? n - first : kMaxBatch;
+    unsigned int tiles = 0;
+    for (int j = 0; j < bt.n; ++j) {
+      const soar_tensor_desc& d = tensors[first + j];
+      Params& p = bt.t[j];
+      p.W = static_cast<const uint16_t*>(d.W_bf16);
+      p.packed = static_cast<uint8_t*>(d.out_fp4_packed);
+      p.ws = reinterpret_cast<Ws*>(headers + static_cast<size_t>(first + j) * kWsFixedBytes);
+      p.ld = d.ld;
+      p.nbc = static_cast<unsigned int>(d.cols / 16);
+      p.nblk = static_cast<unsigned int>(d.rows * (d.cols / 16));
+      p.ntiles = (p.nblk + kTile - 1) / kTile;
+      p.contiguous = (d.ld == d.cols) ? 1 : 0;
+      p.state = nullptr;
+      if (cfg->max_iters > 0) {
+        p.state = reinterpret_cast<uint2*>(next);
+        next += round256(static_cast<size_t>(p.nblk) * sizeof(uint2));
+      }
+      if (want_lin) {
+        p.scales = static_cast<uint8_t*>(d.out_e4m3_scales);
+      } else {
+        p.scales = next;
+        next += round256(p.nblk);
+      }
+      p.max_iters = cfg->max_iters;
+      p.early_stop_rel = cfg->early_stop_rel;
+      p.n_dq = cfg->n_dq;
+      p.n_beta = cfg->n_beta;
+      p.beta_step_pct = cfg->beta_step_pct;
+      p.flags = cfg->flags;
+      tiles += p.ntiles;
+      bt.tile_end[j] = tiles;
+      rp.alpha[j] = d.out_global_fp32;
+      rp.result[j] = d.out_result;
+    }
+    for (int j = bt.n; j < kMaxBatch; ++j) bt.tile_end[j] = 0xFFFFFFFFu;   // never reached by a tile index
+    bt.total_tiles = tiles;
+
+    // Passes alternate direction over the tiles: each starts where the previous one ended,
+    // on data still in L2.
+    int reverse = 0;
+    {
+      ScopedLaunch sl(K_AMAX, st);
+      amax_kernel<<<persistent_grid(amax_kernel, tiles, kThreads), kThreads, 0, st>>>(bt, reverse);
+    }
+    reverse ^= 1;
+    {
+      ScopedLaunch sl(K_INIT, st);
+      init_kernel<<<persistent_grid(init_kernel, tiles, kThreads), kThreads, 0, st>>>(bt, reverse,
+                                                                                      cfg->max_iters == 0 ? 1 : 0);
+    }
+    const unsigned int g_it = single ? persistent_grid(iterate_kernel<true>, tiles, kThreads)
+                                     : persistent_grid(iterate_kernel<false>, tiles, kThreads);
+    for (int t = 0; t < cfg->max_iters; ++t) {
+      reverse ^= 1;
+      // with the early stop on, any iteration may turn out to be the last one
+      const int last = (t == cfg->max_iters - 1) ? 1 : 0;
+      const int emit = (may_stop || last) ? 1 : 0;
+      ScopedLaunch sl(K_ITERATE, st);
+      if (single) iterate_kernel<true><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
+      else iterate_kernel<false><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
+    }
+    {
+      ScopedLaunch sl(K_FINALIZE, st);
+      finalize_kernel<<<bt.n, 128, 0, st>>>(bt, rp);
+    }
+    if (want_sw) {
+      for (int j = 0; j < bt.n; ++j) {
+        const soar_tensor_desc& d = tensors[first + j];
+        const Params& p = bt.t[j];
+        const unsigned int rt = static_cast<unsigned int>((d.rows + 127) / 128);
+        const unsigned int ct = (p.nbc + 3) / 4;
+        const size_t total = static_cast<size_t>(rt) * ct * 512;
+        const size_t blocks = (total + 255) / 256;
+        const unsigned int grid = static_cast<unsigned int>(blocks < 65535u * 16u ? blocks : 65535u * 16u);
+        ScopedLaunch sl(K_SWIZZLE, st);
+        swizzle_kernel<<<grid, 256, 0, st>>>(p.scales, static_cast<uint8_t*>(d.out_e4m3_scales_sw),
+                                             static_cast<unsigned int>(d.rows), p.nbc, rt, ct);
+      }
+    }
+  }
+  return cudaGetLastError() == cudaSuccess ? SOAR_OK : SOAR_ERR_CUDA;
+}
+
 int soar_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, const soar_cfg* cfg,
                   void* out_fp4_packed, void* out_e4m3_scales, void* out_e4m3_scales_sw,
                   float* out_global_fp32, void* workspace, size_t workspace_bytes,
                   soar_result* out_result, void* stream) {
-  int rc = check_cfg(cfg);
-  if (rc != SOAR_OK) return rc;
-  rc = check_shape(W_bf16, rows, cols, ld);
-  if (rc != SOAR_OK) return rc;
-  if (out_fp4_packed == nullptr || out_global_fp32 == nullptr) return SOAR_ERR_INVALID_ARG;
-  if (reinterpret_cast<uintptr_t>(out_fp4_packed) % 16 != 0) return SOAR_ERR_UNSUPPORTED;
-  const bool want_lin = (cfg->scale_layout & SOAR_SCALES_LINEAR) != 0;
-  const bool want_sw = (cfg->scale_layout & SOAR_SCALES_SWIZZLED) != 0;
-  if (want_lin && out_e4m3_scales == nullptr) return SOAR_ERR_INVALID_ARG;
-  if (want_sw && out_e4m3_scales_sw == nullptr) return SOAR_ERR_INVALID_ARG;
-  const size_t need = soar_workspace_bytes(rows, cols, cfg);
-  if (workspace == nullptr || workspace_bytes < need) return SOAR_ERR_WORKSPACE;
-  if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return SOAR_ERR_UNSUPPORTED;
-
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  Params p;
-  p.W = static_cast<const uint16_t*>(W_bf16);
-  p.packed = static_cast<uint8_t*>(out_fp4_packed);
-  p.ws = static_cast<Ws*>(workspace);
-  p.ld = ld;
-  p.nbc = static_cast<unsigned int>(cols / 16);
-  p.nblk = static_cast<unsigned int>(rows * (cols / 16));
-  p.ntiles = (p.nblk + kTile - 1) / kTile;
-  p.contiguous = (ld == cols) ? 1 : 0;
-  {
-    uint8_t* next = static_cast<uint8_t*>(workspace) + kWsFixedBytes;
-    p.state = nullptr;
-    if (cfg->max_iters > 0) {
-      p.state = reinterpret_cast<uint2*>(next);
-      next += round256(static_cast<size_t>(p.nblk) * sizeof(uint2));
-    }
-    p.scales = want_lin ? static_cast<uint8_t*>(out_e4m3_scales) : next;
-  }
-  p.max_iters = cfg->max_iters;
-  p.early_stop_rel = cfg->early_stop_rel;
-  p.n_dq = cfg->n_dq;
-  p.n_beta = cfg->n_beta;
-  p.beta_step_pct = cfg->beta_step_pct;
-  p.flags = cfg->flags;
-
-  if (cudaMemsetAsync(workspace, 0, kWsFixedBytes, st) != cudaSuccess) return SOAR_ERR_CUDA;
-  // Passes alternate direction over the tiles: each starts where the previous one ended,
-  // on data still in L2.
-  int reverse = 0;
-  {
-    ScopedLaunch sl(K_AMAX, st);
-    amax_kernel<<<persistent_grid(amax_kernel, p.nblk, kThreads), kThreads, 0, st>>>(p, reverse);
-  }
-  reverse ^= 1;
-  {
-    ScopedLaunch sl(K_INIT, st);
-    init_kernel<<<persistent_grid(init_kernel, p.nblk, kThreads), kThreads, 0, st>>>(p, reverse,
-                                                                                     cfg->max_iters == 0 ? 1 : 0);
-  }
-  const bool single = cfg->n_beta == 1 && cfg->n_dq <= 2 && !(cfg->flags & SOAR_FLAG_COUPLED_SCALE);
-  const unsigned int g_it = single ? persistent_grid(iterate_kernel<true>, p.nblk, kThreads)
-                                   : persistent_grid(iterate_kernel<false>, p.nblk, kThreads);
-  const bool may_stop = cfg->early_stop_rel > 0.0f;
-  for (int t = 0; t < cfg->max_iters; ++t) {
-    reverse ^= 1;
-    // with the early stop on, any iteration may turn out to be the last one
-    const int last = (t == cfg->max_iters - 1) ? 1 : 0;
-    const int emit = (may_stop || last) ? 1 : 0;
-    ScopedLaunch sl(K_ITERATE, st);
-    if (single) iterate_kernel<true><<<g_it, kThreads, 0, st>>>(p, t, reverse, emit, !last);
-    else iterate_kernel<false><<<g_it, kThreads, 0, st>>>(p, t, reverse, emit, !last);
-  }
-  {
-    ScopedLaunch sl(K_FINALIZE, st);
-    finalize_kernel<<<1, 128, 0, st>>>(p, out_global_fp32, out_result);
-  }
-  if (want_sw) {
-    const unsigned int rt = static_cast<unsigned int>((rows + 127) / 128);
-    const unsigned int ct = (p.nbc + 3) / 4;
-    const size_t total = static_cast<size_t>(rt) * ct * 512;
-    const size_t blocks = (total + 255) / 256;
-    const unsigned int grid = static_cast<unsigned int>(blocks < 65535u * 16u ? blocks : 65535u * 16u);
-    ScopedLaunch sl(K_SWIZZLE, st);
-    swizzle_kernel<<<grid, 256, 0, st>>>(p.scales, static_cast<uint8_t*>(out_e4m3_scales_sw),
-                                         static_cast<unsigned int>(rows), p.nbc, rt, ct);
-  }
-  return cudaGetLastError() == cudaSuccess ? SOAR_OK : SOAR_ERR_CUDA;
+  soar_tensor_desc d;
+  d.W_bf16 = W_bf16;
+  d.rows = rows;
+  d.cols = cols;
+  d.ld = ld;
+  d.out_fp4_packed = out_fp4_packed;
+  d.out_e4m3_scales = out_e4m3_scales;
+  d.out_e4m3_scales_sw = out_e4m3_scales_sw;
+  d.out_global_fp32 = out_global_fp32;
+  d.out_result = out_result;
+  return soar_quantize_batch(&d, 1, cfg, workspace, workspace_bytes, stream);
 }
 
 // Built-in scratch of soar_quantize_static.  In host code the symbol below is only a handle:
@@ -1256,8 +1448,14 @@ int soar_dequant_error(const void* W_bf16, int64_t rows, int64_t cols, int64_t l
   if (cudaMemsetAsync(out_sumsq, 0, sizeof(double), st) != cudaSuccess) return SOAR_ERR_CUDA;
   {
     ScopedLaunch sl(K_DEQUANT_ERROR, st);
-    dequant_error_kernel<<<persistent_grid(dequant_error_kernel, p.nblk, kThreads), kThreads, 0, st>>>(
-        p, static_cast<const uint8_t*>(e4m3_scales), scale_layout == SOAR_SCALES_SWIZZLED ? 1 : 0,
+    Batch bt;
+    memset(&bt, 0, sizeof(bt));
+    bt.n = 1;
+    bt.t[0] = p;
+    bt.total_tiles = p.ntiles;
+    for (int j = 0; j < kMaxBatch; ++j) bt.tile_end[j] = j == 0 ? p.ntiles : 0xFFFFFFFFu;
+    dequant_error_kernel<<<persistent_grid(dequant_error_kernel, p.ntiles, kThreads), kThreads, 0, st>>>(
+        bt, static_cast<const uint8_t*>(e4m3_scales), scale_layout == SOAR_SCALES_SWIZZLED ? 1 : 0,
         (p.nbc + 3) / 4, global_fp32, out_sse, out_sumsq);
   }
   return cudaGetLastError() == cudaSuccess ? SOAR_OK : SOAR_ERR_CUDA;

@@ -127,6 +127,42 @@ def test_fast_reciprocal_equals_the_correctly_rounded_one_everywhere_it_is_used(
         api.soar_selftest_reciprocal(1, 252)
 
 
+@pytest.mark.parametrize("cfgkw", [
+    dict(),                                                   # the paper's preset: tensors stop after different iterations
+    dict(max_iters=1, early_stop_rel=0.0, n_dq=2, n_beta=1),  # single pass
+    dict(max_iters=0),
+])
+def test_batch_gives_each_matrix_what_a_single_call_gives(cfgkw):
+    """20 matrices (more than one launch group), from one block to several tiles, one all zero,
+    one with a NaN, one with a padded row stride: same bytes as 20 separate calls, and the oracle's."""
+    shapes = [(1, 16), (3, 48), (37, 1040), (130, 2064), (64, 4096), (5, 16), (257, 512), (8, 8192)] * 2 + \
+             [(16, 64), (96, 1024), (33, 272), (512, 256)]
+    ws = [WL.small_case(r, c, 100 + i, dist=("laplace" if i % 3 == 0 else "student_t4"),
+                        outlier_entry_frac=0.005 * (i % 2), outlier_scale=40.0)
+          for i, (r, c) in enumerate(shapes)]
+    ws[5][:] = 0
+    ws[9] = ws[9].copy(); ws[9][1, 3] = 0x7FC0
+    cfg, ref_cfg = P.cfg_pair(**cfgkw)
+    dev = [P.to_device(w, ld=(w.shape[1] + 24 if i == 3 else None)) for i, w in enumerate(ws)]
+    outs = [api.alloc_buffers(w.shape[0], w.shape[1], cfg) for w in ws]
+    api.soar_quantize_batch(dev, cfg, outs)
+    torch.cuda.synchronize()
+    for i, (w, W, o) in enumerate(zip(ws, dev, outs)):
+        one = api.soar_quantize(W, cfg)
+        torch.cuda.synchronize()
+        r1, rb = one.read_result(), o.read_result()
+        assert rb.status == r1.status and rb.iters_run == r1.iters_run, i
+        if rb.status & api.STATUS_NONFINITE:
+            continue
+        assert np.array_equal(o.packed.cpu().numpy(), one.packed.cpu().numpy()), i
+        assert np.array_equal(o.scales.cpu().numpy(), one.scales.cpu().numpy()), i
+        assert float(o.alpha.cpu()[0]) == float(one.alpha.cpu()[0]), i
+        assert rb.sse == pytest.approx(r1.sse, rel=1e-12), i
+        if rb.status == 0 and i % 4 == 0:
+            g = P.GpuOut(o.packed.cpu().numpy(), o.scales.cpu().numpy(), float(o.alpha.cpu()[0]), rb, o)
+            P.assert_parity(g, R.quantize(w, ref_cfg))
+
+
 def test_argument_errors_are_reported_on_the_host():
     w = P.to_device(WL.small_case(4, 64, 0))
     cfg = api.soar_default_cfg()
