@@ -265,10 +265,21 @@ def run_ours(args):
     elements = wl.elements
     stream = torch.cuda.current_stream()
 
-    def step(c=cfg):
-        for W, o in zip(dev_w, outs):
-            api.soar_quantize(W, c, o, stream)
+    batch_ws = {}
 
+    def step(c=cfg, st=None):
+        """One pass over the workload: one batched call (or one call per tensor with --no-batch)."""
+        st = stream if st is None else st
+        if args.no_batch:
+            for W, o in zip(dev_w, outs):
+                api.soar_quantize(W, c, o, st)
+            return
+        key = (c.max_iters, c.scale_layout)
+        if key not in batch_ws:
+            batch_ws[key] = torch.empty(api.soar_batch_workspace_bytes(dev_w, outs, c), dtype=torch.uint8, device="cuda")
+        api.soar_quantize_batch(dev_w, c, outs, batch_ws[key], st)
+
+    eager_step = step
     if args.graph:
         # replay the step's launches from a CUDA graph: takes the host's launch cost out of the picture
         side = torch.cuda.Stream()
@@ -279,13 +290,12 @@ def run_ours(args):
             if key not in graphs:
                 g = torch.cuda.CUDAGraph()
                 torch.cuda.synchronize()
+                eager_step(c, side)                      # allocate the workspace outside the capture
+                torch.cuda.synchronize()
                 with torch.cuda.graph(g, stream=side):
-                    for W, o in zip(dev_w, outs):
-                        api.soar_quantize(W, c, o, side)
+                    eager_step(c, side)
                 graphs[key] = g
             return graphs[key]
-
-        eager_step = step
 
         def step(c=cfg):  # noqa: F811
             graphed(c).replay()
@@ -329,7 +339,11 @@ def run_ours(args):
     dom = max(trace, key=lambda k: trace[k][1])
     n_launch, tot_ms = trace[dom]
     # DRAM traffic of an average working launch of the dominant kernel (ncu figure per element x elements)
-    active = sum(iters) if dom == "iterate_kernel" else len(wl.tensors)
+    if args.no_batch:
+        active = sum(iters) if dom == "iterate_kernel" else len(wl.tensors)
+    else:      # one launch serves a group of up to 16 tensors; an iteration launch works while any of them runs
+        groups = [iters[i:i + 16] for i in range(0, len(iters), 16)]
+        active = sum(max(g) for g in groups) if dom == "iterate_kernel" else len(groups)
     tpe = ncu_traffic_per_elem(dom, cfg)
     work_elems = (sum(s.rows * s.cols * it for s, it in zip(wl.tensors, iters)) if dom == "iterate_kernel"
                   else elements)
@@ -342,7 +356,7 @@ def run_ours(args):
         peak = SM_COUNT * FP32_LANES_PER_SM * peaks["sm_max_mhz"] * 1e6 / 1e12
         roofline = dict(bound="alu", kernel=dom, achieved=achieved, peak=peak, unit="Tlane-op/s",
                         frac=achieved / peak, traffic=traffic, launches=n_launch,
-                        active_launches=sum(iters) * args.steps, kernel_ms_per_step=tot_ms / args.steps,
+                        active_launches=active * args.steps, kernel_ms_per_step=tot_ms / args.steps,
                         peak_source="148 SMs x 128 FP32 lanes x clocks.max.sm",
                         hbm_gbs_for_context=sum(
                             s.rows * s.cols * kernel_bytes_per_elem(dom, cfg, t)
@@ -473,7 +487,7 @@ def run_ours(args):
                         parallelism=f"{world} rank(s), one layer of these shapes each, no collective"),
             elements_per_s=world * elements / (ms * 1e-3),
             hbm_frac_end_to_end_of_measured=value / peaks["hbm_gbs"],
-            traced_ms_per_step=traced_ms, cuda_graph=bool(args.graph), roofline=roofline, kernels=kernels, cpu_baseline=cpu, e2e=e2e, gpu_launches=launches,
+            traced_ms_per_step=traced_ms, cuda_graph=bool(args.graph), batched=not args.no_batch, roofline=roofline, kernels=kernels, cpu_baseline=cpu, e2e=e2e, gpu_launches=launches,
             clocks=clocks, **extra)
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -493,6 +507,7 @@ def main():
     ap.add_argument("--pairs", type=int, default=0, help="candidate pairs per block (overrides the preset's grid)")
     ap.add_argument("--iters", type=int, default=None, help="iterations T, early stop off (overrides the preset)")
     ap.add_argument("--sweep", default="", help="comma-separated candidate-pair counts to time, one iteration each")
+    ap.add_argument("--no-batch", action="store_true", help="one soar_quantize call per tensor instead of soar_quantize_batch")
     ap.add_argument("--graph", action="store_true", help="replay each step from a CUDA graph (no per-kernel trace)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
