@@ -88,6 +88,22 @@ struct Batch {
 };
 static_assert(sizeof(Batch) <= 3072, "kernel parameter block too large");
 
+// What a consumer needs of its current tensor, copied out of the parameter block once per tensor.
+struct Tensor {
+  uint8_t* packed;
+  uint8_t* scales;
+  uint2* state;
+  unsigned int nblk;
+};
+__device__ __forceinline__ Tensor tensor_view(const Params& p) {
+  Tensor v;
+  v.packed = p.packed;
+  v.scales = p.scales;
+  v.state = p.state;
+  v.nblk = p.nblk;
+  return v;
+}
+
 // ------------------------------------------------------------------ number formats
 
 __device__ __forceinline__ float bits_to_mag(unsigned int bf16_bits) {
@@ -562,7 +578,7 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const __grid_constant__ 
     if (threadIdx.x == kTile) ring_produce(ring, bt, reverse, 0xFFFFFFFFu);
     return;
   }
-  unsigned int mx = 0;
+  unsigned int mx = 0, nblk = 0;
   double sq[2] = {0.0, 0.0};
   int cur = -1;
   for (unsigned int n = 0;; ++n) {
@@ -583,9 +599,9 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const __grid_constant__ 
       }
       if (rc != 0) break;
       cur = ti;
+      nblk = bt.t[ti].nblk;
     }
-    const unsigned int b = tile * kTile + threadIdx.x;
-    if (b >= bt.t[ti].nblk) continue;
+    if (tile * kTile + threadIdx.x >= nblk) continue;
     const unsigned int u[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
     // largest and smallest magnitude of the block with packed bf16 min/max (a NaN input comes out
     // of the maximum as NaN, whose bits are above the infinity pattern)
@@ -639,6 +655,7 @@ __global__ void __launch_bounds__(kThreads) init_kernel(const __grid_constant__ 
   double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum
   unsigned int zeros = 0, wide = 0;
   int cur = -1;
+  Tensor p = {};   // the current tensor's pointers and size, kept in registers
   for (unsigned int n = 0;; ++n) {
     uint4 v0, v1;
     int ti = -1;
@@ -657,8 +674,8 @@ __global__ void __launch_bounds__(kThreads) init_kernel(const __grid_constant__ 
       alpha = amax_bits == 0 ? 1.0f : __fdiv_rn(bits_to_mag(amax_bits), 2688.0f);
       six_alpha = __fmul_rn(alpha, 6.0f);
       alpha_d = static_cast<double>(alpha);
+      p = tensor_view(bt.t[ti]);
     }
-    const Params& p = bt.t[ti];
     const unsigned int b = tile * kTile + threadIdx.x;
     if (b >= p.nblk) continue;
     Block blk;
@@ -788,6 +805,8 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
   double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum of stage t+1
   unsigned int wide = 0, unused_zeros = 0;
   int cur = -1;
+  Tensor p = {};   // the current tensor's pointers and size, kept in registers
+  const int flags = bt.t[0].flags;
   for (unsigned int n = 0;; ++n) {
     uint4 v0, v1;
     uint2 st;
@@ -805,14 +824,17 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
       cur = ti;
       alpha = s_alpha[ti];
       alpha_d = static_cast<double>(alpha);
+      if (kSingle) p = tensor_view(bt.t[ti]);
     }
-    const Params& p = bt.t[ti];
+    // the long candidate loop does better re-reading these from the parameter block per tile than
+    // carrying them in registers
+    if (!kSingle) p = tensor_view(bt.t[ti]);
     const unsigned int b = tile * kTile + threadIdx.x;
     if (b >= p.nblk || (st.y >> 16) == 0) continue;   // past the end, or an all-zero block: nothing to optimise
     Block blk;
     unpack_block(v0, v1, blk);
     int d_lo, d_hi;
-    const float center = block_center(st, alpha, n_dq, (p.flags & SOAR_FLAG_KEEP_BLOCK_SCALE) != 0, d_lo, d_hi);
+    const float center = block_center(st, alpha, n_dq, (flags & SOAR_FLAG_KEEP_BLOCK_SCALE) != 0, d_lo, d_hi);
     const int dc0 = clip_code(d_lo), dc1 = clip_code(d_lo + 1);
     const double sd0 = alpha_d * static_cast<double>(e4m3_value(dc0));
     const double sd1 = alpha_d * static_cast<double>(e4m3_value(dc1));
@@ -843,7 +865,7 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
       const int nd = d_hi - d_lo + 1;
       // the reciprocal scale falls as beta grows, so the first candidate decides whether the
       // exact integer sums hold for all of them
-      const bool coupled = (p.flags & SOAR_FLAG_COUPLED_SCALE) != 0;
+      const bool coupled = (flags & SOAR_FLAG_COUPLED_SCALE) != 0;
       const bool all_narrow = fx.ok && __fmul_rn(blk.bmax, recip_scale(alpha, __fmul_rn(center, s_beta[0]))) <= 32.0f;
       // the products alpha * center * beta are monotone in beta: the end points bound them all
       const bool fast_rcp = recip_fast_ok(__fmul_rn(alpha, __fmul_rn(center, s_beta[0]))) &&
