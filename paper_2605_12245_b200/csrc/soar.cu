@@ -569,7 +569,7 @@ __device__ __forceinline__ void sumsq_block(const unsigned int (&u)[8], double& 
 }
 
 // Eq. 1's tensor maximum, plus sum W^2 (binary64) for the error report.
-__global__ void __launch_bounds__(kThreads) amax_kernel(const __grid_constant__ Batch bt, int reverse) {
+__global__ void __launch_bounds__(kThreads, 6) amax_kernel(const __grid_constant__ Batch bt, int reverse) {
   __shared__ Ring ring;
   __shared__ Slots<1> slots;
   slots_clear(slots);
