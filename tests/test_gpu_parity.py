@@ -163,6 +163,44 @@ def test_batch_gives_each_matrix_what_a_single_call_gives(cfgkw):
             P.assert_parity(g, R.quantize(w, ref_cfg))
 
 
+def test_calls_on_two_streams_with_their_own_workspaces_do_not_disturb_each_other():
+    w1 = WL.small_case(300, 2048, 81, outlier_entry_frac=0.003, outlier_scale=30.0)
+    w2 = WL.small_case(200, 4096, 82, dist="laplace")
+    cfg, _ = P.cfg_pair(max_iters=3)
+    W1, W2 = P.to_device(w1), P.to_device(w2)
+    want1, want2 = api.soar_quantize(W1, cfg), api.soar_quantize(W2, cfg)
+    torch.cuda.synchronize()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    o1, o2 = api.alloc_buffers(*w1.shape, cfg), api.alloc_buffers(*w2.shape, cfg)
+    for _ in range(3):
+        api.soar_quantize(W1, cfg, o1, s1)
+        api.soar_quantize(W2, cfg, o2, s2)
+    torch.cuda.synchronize()
+    for got, want in ((o1, want1), (o2, want2)):
+        assert torch.equal(got.packed, want.packed) and torch.equal(got.scales, want.scales)
+        assert torch.equal(got.alpha, want.alpha)
+
+
+def test_a_call_replays_from_a_cuda_graph():
+    """Nothing in a call synchronizes or allocates, so it can be captured once and replayed."""
+    w = WL.small_case(128, 2048, 83, outlier_cols_frac=0.002, outlier_scale=20.0)
+    cfg, ref_cfg = P.cfg_pair()
+    W = P.to_device(w)
+    out = api.alloc_buffers(*w.shape, cfg)
+    side = torch.cuda.Stream()
+    api.soar_quantize(W, cfg, out, side)                  # first call outside the capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        api.soar_quantize(W, cfg, out, side)
+    out.packed.zero_(); out.scales.zero_(); out.alpha.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    gpu = P.GpuOut(out.packed.cpu().numpy(), out.scales.cpu().numpy(), float(out.alpha.cpu()[0]),
+                   out.read_result(), out)
+    P.assert_parity(gpu, R.quantize(w, ref_cfg))
+
+
 def test_argument_errors_are_reported_on_the_host():
     w = P.to_device(WL.small_case(4, 64, 0))
     cfg = api.soar_default_cfg()
