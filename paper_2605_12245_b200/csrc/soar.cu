@@ -439,6 +439,30 @@ __device__ __forceinline__ void code_sums(const Fixed& fx, unsigned int c0, unsi
   afix = __dp2a_hi(fx.pair[7], t3, a);
 }
 
+// The integer sums of the block's code vector under reciprocal scale r, from the magnitudes
+// alone: afix = sum fix_j * (2 m_j), b4 = sum (2 m_j)^2 with m_j = E2M1(fl(a_j * r)).  Without sign
+// bits the codes feed the byte permute as they are (the candidate loop only ranks; the signed
+// winner is re-made later).
+__device__ __forceinline__ void magnitude_sums(const float (&a)[16], const Fixed& fx, float r, unsigned int& afix,
+                                               unsigned int& b4) {
+  float x[16];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) mul2(a[2 * i], a[2 * i + 1], r, x[2 * i], x[2 * i + 1]);
+  const unsigned int c0 = e2m1x8(x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7]);
+  const unsigned int c1 = e2m1x8(x[8], x[9], x[10], x[11], x[12], x[13], x[14], x[15]);
+  const unsigned int t[4] = {twice_magnitude_x4(c0), twice_magnitude_x4(c0 >> 16), twice_magnitude_x4(c1),
+                             twice_magnitude_x4(c1 >> 16)};
+  unsigned int acc_a = 0, acc_b = 0;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    acc_b = __dp4a(t[q], t[q], acc_b);
+    acc_a = __dp2a_lo(fx.pair[2 * q], t[q], acc_a);
+    acc_a = __dp2a_hi(fx.pair[2 * q + 1], t[q], acc_a);
+  }
+  afix = acc_a;
+  b4 = acc_b;
+}
+
 // The same sums for a code vector whose scale lies far below the block maximum: binary64
 // accumulation in element order.
 __device__ __forceinline__ void code_sums_wide(const float (&w)[16], unsigned int c0, unsigned int c1, double& A,
@@ -877,11 +901,13 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
         const double rho0 = sd0 * fx.inv8, rho1 = sd1 * fx.inv8;
         double h0 = best, h1 = best;
         int k0 = 0, k1 = 0;
+        float mag[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) mag[j] = fabsf(blk.w[j]);
         for (int k = 0; k < n_beta; ++k) {
           const float r = recip_fast(__fmul_rn(alpha, __fmul_rn(center, s_beta[k])));
-          unsigned int c0, c1, afix, b4;
-          round_block(blk, r, c0, c1);
-          code_sums(fx, c0, c1, afix, b4);
+          unsigned int afix, b4;
+          magnitude_sums(mag, fx, r, afix, b4);
           const double ad = uint_to_double(afix), bd = uint_to_double(b4);
           const double e0 = fma(rho0, bd, -ad);
           if (e0 < h0) { h0 = e0; k0 = k; }
