@@ -424,10 +424,7 @@ def run_ours(args):
     ctypes_sizeof_result = ctypes.sizeof(api.SoarResult)
     e2e = None
     if not args.no_e2e and args.workload != "config3":      # config 3 would pin 18 GB of host memory
-        big = max(wl.tensors, key=lambda s: s.rows * s.cols)
-        streams = [torch.cuda.Stream(), torch.cuda.Stream()]
-        stage = [(torch.empty((big.rows * big.cols,), dtype=torch.bfloat16, device="cuda"),
-                  api.alloc_buffers(big.rows, big.cols, cfg)) for _ in streams]
+        pipe = api.HostPipeline([(s.rows, s.cols) for s in wl.tensors], cfg, depth=4)
         hosts = []
         for h, spec in zip(host_w, wl.tensors):
             hb = api.alloc_host_buffers(spec.rows, spec.cols, cfg)
@@ -435,15 +432,7 @@ def run_ours(args):
             hosts.append(hb)
 
         def e2e_step():
-            for i, (hb, spec) in enumerate(zip(hosts, wl.tensors)):
-                s = streams[i % 2]
-                dW, big_out = stage[i % 2]
-                n = spec.rows * spec.cols
-                view = api.QuantBuffers(
-                    packed=big_out.packed.view(-1)[: n // 2].view(spec.rows, spec.cols // 2),
-                    scales=big_out.scales.view(-1)[: n // 16].view(spec.rows, spec.cols // 16),
-                    scales_sw=None, alpha=big_out.alpha, result=big_out.result, workspace=big_out.workspace)
-                api.soar_quantize_host(hb, cfg, dW[:n].view(spec.rows, spec.cols), view, s)
+            pipe.run(hosts)
 
         for _ in range(2):
             e2e_step()
@@ -459,7 +448,7 @@ def run_ours(args):
         e2e = dict(value=world * 2.0 * elements / dt / 1e9, unit="GB/s", ms_per_step=dt * 1e3,
                    h2d_bytes_per_step=2 * elements,
                    d2h_bytes_per_step=elements // 2 + elements // 16 + len(wl.tensors) * (4 + ctypes_sizeof_result),
-                   api="soar_quantize_host, two streams, pinned host buffers")
+                   api="HostPipeline: pinned host buffers, copy-in / soar_quantize / copy-out on three streams, 4 slots")
 
     # ---- the oracle on the host cores, bounded sample (rank 0, single GPU only)
     cpu = None

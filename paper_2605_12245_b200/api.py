@@ -333,6 +333,61 @@ def soar_quantize_host(host: HostBuffers, cfg: SoarCfg, dev_W: torch.Tensor, dev
     _check(rc, "soar_quantize_host")
 
 
+class HostPipeline:
+    """Quantizes matrices that live in pinned host memory with the three legs overlapped:
+    host-to-device copies on one stream, ``soar_quantize`` on a second, device-to-host copies of
+    the results on a third, chained by events over ``depth`` device staging slots sized for the
+    largest matrix.  Stream plumbing only; the work is ``soar_quantize``."""
+
+    def __init__(self, shapes, cfg: SoarCfg, depth: int = 3, device="cuda"):
+        self.cfg = cfg
+        rows, cols = max(shapes, key=lambda rc: rc[0] * rc[1])
+        self.slots = []
+        for _ in range(depth):
+            self.slots.append(dict(
+                W=torch.empty(rows * cols, dtype=torch.bfloat16, device=device),
+                out=alloc_buffers(rows, cols, cfg, device),
+                loaded=torch.cuda.Event(), computed=torch.cuda.Event(), stored=torch.cuda.Event()))
+        self.h2d, self.compute, self.d2h = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+        for sl in self.slots:
+            sl["stored"].record(self.d2h)
+
+    def run(self, hosts) -> None:
+        """Enqueue the whole list (``HostBuffers`` each); results are in the host buffers once
+        ``synchronize()`` returns."""
+        for i, hb in enumerate(hosts):
+            sl = self.slots[i % len(self.slots)]
+            rows, cols = hb.W.shape
+            n = rows * cols
+            big = sl["out"]
+            W = sl["W"][:n].view(rows, cols)
+            view = QuantBuffers(
+                packed=big.packed.view(-1)[: n // 2].view(rows, cols // 2),
+                scales=None if big.scales is None else big.scales.view(-1)[: n // 16].view(rows, cols // 16),
+                scales_sw=None if big.scales_sw is None else big.scales_sw[: soar_swizzled_scale_bytes(rows, cols)],
+                alpha=big.alpha, result=big.result, workspace=big.workspace)
+            self.h2d.wait_event(sl["stored"])            # the slot's previous results have left
+            with torch.cuda.stream(self.h2d):
+                W.copy_(hb.W, non_blocking=True)
+                sl["loaded"].record(self.h2d)
+            self.compute.wait_event(sl["loaded"])
+            soar_quantize(W, self.cfg, view, self.compute)
+            sl["computed"].record(self.compute)
+            self.d2h.wait_event(sl["computed"])
+            with torch.cuda.stream(self.d2h):
+                hb.packed.copy_(view.packed, non_blocking=True)
+                if view.scales is not None:
+                    hb.scales.copy_(view.scales, non_blocking=True)
+                if view.scales_sw is not None:
+                    hb.scales_sw.copy_(view.scales_sw, non_blocking=True)
+                hb.alpha.copy_(view.alpha, non_blocking=True)
+                hb.result.copy_(view.result, non_blocking=True)
+                sl["stored"].record(self.d2h)
+
+    def synchronize(self) -> None:
+        self.d2h.synchronize()
+
+
 def soar_selftest_reciprocal(lo_exp: int = 2, hi_exp: int = 252, stream=None) -> int:
     """Runs ``soar_selftest_reciprocal`` and returns the mismatch count (synchronizes)."""
     out = torch.zeros(1, dtype=torch.int64, device="cuda")

@@ -201,6 +201,28 @@ def test_a_call_replays_from_a_cuda_graph():
     P.assert_parity(gpu, R.quantize(w, ref_cfg))
 
 
+def test_host_pipeline_returns_what_direct_calls_return():
+    """Seven matrices through three staging slots: every slot is reused, sizes differ."""
+    shapes = [(64, 1024), (16, 256), (300, 512), (8, 4096), (130, 2064), (1, 16), (257, 1024)]
+    ws = [WL.small_case(r, c, 200 + i, outlier_entry_frac=0.004, outlier_scale=30.0) for i, (r, c) in enumerate(shapes)]
+    cfg, _ = P.cfg_pair(max_iters=3)
+    hosts = []
+    for w in ws:
+        hb = api.alloc_host_buffers(w.shape[0], w.shape[1], cfg)
+        hb.W.copy_(torch.from_numpy(w.view(np.int16)).view(torch.bfloat16))
+        hosts.append(hb)
+    pipe = api.HostPipeline(shapes, cfg, depth=3)
+    for _ in range(2):                                   # the second round reuses everything once more
+        pipe.run(hosts)
+    pipe.synchronize()
+    for w, hb in zip(ws, hosts):
+        want = P.run_gpu(w, cfg)
+        assert np.array_equal(hb.packed.numpy(), want.packed)
+        assert np.array_equal(hb.scales.numpy(), want.scales)
+        assert float(hb.alpha[0]) == want.alpha
+        assert hb.read_result().iters_run == want.result.iters_run
+
+
 def test_argument_errors_are_reported_on_the_host():
     w = P.to_device(WL.small_case(4, 64, 0))
     cfg = api.soar_default_cfg()
