@@ -274,6 +274,39 @@ def test_swizzled_scale_layout(rows, cols):
     assert e_lin[0] == pytest.approx(g.result.sse, rel=1e-9)
 
 
+@pytest.mark.parametrize("M,K,N", [(256, 512, 128), (128, 2048, 256)])
+def test_outputs_feed_the_hardware_block_scaled_gemm(M, K, N):
+    """The packed codes and the 128x4-tiled scales go, as they are, into the library's block-scaled FP4
+    matrix product (Blackwell's block-scaled MMA underneath); the result must equal the product with
+    the matrix dequantized by Eq. 3 on the host.  This pins the nibble order and the tiled scale
+    layout against the consumer they are meant for.  The other operand is made of exact E2M1 values
+    with unit scales, so the only rounding is the product's binary32 accumulation."""
+    if not hasattr(torch, "float4_e2m1fn_x2"):
+        pytest.skip("this torch has no packed FP4 dtype")
+    w = WL.small_case(M, K, 7, outlier_entry_frac=0.002, outlier_scale=20.0)
+    cfg = api.soar_default_cfg(api.PRESET_PAPER, scale_layout=api.SCALES_LINEAR | api.SCALES_SWIZZLED)
+    g = P.run_gpu(w, cfg)
+    grid = np.array([0, .5, 1, 1.5, 2, 3, 4, 6])
+    codes = np.stack([g.packed & 0xF, g.packed >> 4], axis=-1).reshape(M, K)
+    e4 = np.arange(0x7F, dtype=np.uint8).view(ml_dtypes.float8_e4m3fn).astype(np.float64)
+    Wd = grid[codes & 7] * np.where(codes & 8, -1.0, 1.0) * np.repeat(e4[g.scales], 16, axis=1)   # Eq. 3 without alpha
+    rng = np.random.default_rng(0)
+    xc = rng.integers(0, 16, size=(N, K)).astype(np.uint8)
+    X = grid[xc & 7] * np.where(xc & 8, -1.0, 1.0)
+    xp = (xc[:, 0::2] | (xc[:, 1::2] << 4)).astype(np.uint8)
+    ones = swizzle_reference(np.full((N, K // 16), 0x38, np.uint8))                               # E4M3 1.0
+    a = torch.from_numpy(xp).cuda().view(torch.float4_e2m1fn_x2)
+    b = g.buffers.packed.view(torch.float4_e2m1fn_x2)
+    sa = torch.from_numpy(ones).cuda().view(torch.float8_e4m3fn)
+    sb = g.buffers.scales_sw.view(torch.float8_e4m3fn)
+    try:
+        out = torch._scaled_mm(a, b.t(), sa, sb, out_dtype=torch.float32)
+    except (RuntimeError, NotImplementedError) as e:      # no block-scaled FP4 product on this device / build
+        pytest.skip(f"block-scaled FP4 product unavailable: {str(e)[:80]}")
+    ref = X @ Wd.T
+    assert np.abs(out.double().cpu().numpy() - ref).max() <= 1e-6 * np.abs(ref).max()
+
+
 def test_dequant_error_matches_oracle():
     w = WL.small_case(96, 1024, 41, outlier_entry_frac=0.002, outlier_scale=50.0)
     cfg, ref_cfg = P.cfg_pair(max_iters=2)
