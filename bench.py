@@ -81,7 +81,8 @@ def pick_workload(name: str, rank: int = 0) -> FlatWorkload:
 def preset_cfg(api, preset: str, args=None, **over):
     """The preset's settings; ``--pairs K`` and ``--iters T`` override the candidate grid and the
     iteration count (K pairs per block = n_beta x n_dq with n_dq = min(2, K); no early stop)."""
-    base = api.PRESET_PAPER if preset == "paper" else api.PRESET_SINGLE_PASS
+    base = {"paper": api.PRESET_PAPER, "single_pass": api.PRESET_SINGLE_PASS,
+            "coupled_pair": api.PRESET_COUPLED_PAIR}[preset]
     if args is not None and args.pairs:
         n_dq = min(2, args.pairs)
         over.update(n_dq=n_dq, n_beta=max(1, args.pairs // n_dq))
@@ -490,7 +491,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config4")
-    ap.add_argument("--preset", default="paper", choices=["paper", "single_pass"])
+    ap.add_argument("--preset", default="paper", choices=["paper", "single_pass", "coupled_pair"])
     ap.add_argument("--cpu-rows", type=int, default=4096, help="rows of tensor 0 the CPU baseline quantizes")
     ap.add_argument("--ref-rows", type=int, default=1024, help="rows per step of the reference arm")
     ap.add_argument("--pairs", type=int, default=0, help="candidate pairs per block (overrides the preset's grid)")

@@ -51,6 +51,10 @@ extern "C" {
 #define SOAR_PRESET_RTN 2              /* T=0: the max-based rule of Eq. 1-3 only            */
 #define SOAR_PRESET_CJSO_ONLY 3        /* Sec. 3.2 alone: T=15, stop 1e-3, nearest E4M3 code, coupled scale */
 #define SOAR_PRESET_DSS_ONLY 4         /* Sec. 3.3 alone: one search (2 x 101) around the max-based start   */
+#define SOAR_PRESET_COUPLED_PAIR 5     /* closed-form updates with both E4M3 codes bracketing the Eq. 6 solution,
+                                          each tried with itself as the quantization scale (2 candidates per
+                                          block instead of 202): T=15, stop 1e-3, coupled scale.  Not an arm of
+                                          the paper; on synthetic weights it ends at the full search's error  */
 
 /* soar_cfg.flags bits: the stand-alone arms of the paper's ablation (Table 4) */
 #define SOAR_FLAG_COUPLED_SCALE 1      /* Sec. 3.2 "Refinement Scheme": one block scale quantizes and

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(HERE, "libsoar.so")
 SOAR_OK = 0
 STATUS_ZERO_TENSOR, STATUS_NONFINITE, STATUS_RANGE, STATUS_INTERNAL = 1, 2, 4, 8
 SCALES_LINEAR, SCALES_SWIZZLED = 1, 2
-PRESET_PAPER, PRESET_SINGLE_PASS, PRESET_RTN, PRESET_CJSO_ONLY, PRESET_DSS_ONLY = 0, 1, 2, 3, 4
+PRESET_PAPER, PRESET_SINGLE_PASS, PRESET_RTN, PRESET_CJSO_ONLY, PRESET_DSS_ONLY, PRESET_COUPLED_PAIR = 0, 1, 2, 3, 4, 5
 FLAG_COUPLED_SCALE, FLAG_KEEP_ALPHA, FLAG_KEEP_BLOCK_SCALE = 1, 2, 4
 MAX_ITERS = 64
 

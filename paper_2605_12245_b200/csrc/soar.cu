@@ -791,11 +791,12 @@ __device__ __forceinline__ int clip_code(int d) { return max(1, min(0x7E, d)); }
 // App. B.3 candidate sets, Eq. 8 search, winner stored, stage-(t+1) sums accumulated.
 // Codes and scale bytes are written when `emit` is set (the state after this iteration may
 // be the one returned); the per-block sums are kept when `keep` is set (another iteration
-// may follow).  kSingle is the shape with one quantization scale (beta = 1) and at most two
-// dequantization codes, whose passes are bound by HBM rather than by the candidate loop.
-template <bool kSingle>
-__global__ void __launch_bounds__(kThreads, kSingle ? 3 : 2)
+// may follow).  Modes 1 and 2 are the shapes with one quantization scale per E4M3 code and at most two
+// codes, whose passes are bound by HBM rather than by the candidate loop.
+template <int kMode>   // 0: candidate grid; 1: one candidate scale (beta = 1); 2: the same with the coupled scale
+__global__ void __launch_bounds__(kThreads, kMode == 1 ? 3 : 2)
 iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, int keep) {
+  constexpr bool kSingle = kMode != 0;
   __shared__ RingWithState ring;
   __shared__ Slots<3> slots;
   __shared__ float s_beta[kSingle ? 1 : SOAR_MAX_BETA];
@@ -867,7 +868,23 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
     double best, bestA, bestB;
     int best_d = dc0;
     unsigned int best0, best1;
-    if (kSingle) {
+    if (kMode == 2) {
+      // beta = 1 and the coupled scale of Sec. 3.2: each E4M3 candidate rounds the block with its
+      // own value and is scored with it
+      const float r0 = recip_scale(alpha, e4m3_value(dc0));
+      round_block(blk, r0, best0, best1);
+      block_sums(blk, fx, r0, best0, best1, bestA, bestB, wide);
+      best = sd0 * fma(sd0, bestB, -2.0 * bestA);
+      if (n_dq == 2) {
+        const float r1 = recip_scale(alpha, e4m3_value(dc1));
+        unsigned int c0, c1;
+        double A, B;
+        round_block(blk, r1, c0, c1);
+        block_sums(blk, fx, r1, c0, c1, A, B, wide);
+        const double g1 = sd1 * fma(sd1, B, -2.0 * A);
+        if (g1 < best) { best = g1; best_d = dc1; bestA = A; bestB = B; best0 = c0; best1 = c1; }
+      }
+    } else if (kSingle) {
       // one quantization scale (beta = 1): the codes are fixed, only the E4M3 code is chosen
       const float r = recip_scale(alpha, center);
       round_block(blk, r, best0, best1);
@@ -1259,6 +1276,10 @@ int soar_default_cfg(soar_cfg* cfg, int preset) {
       cfg->max_iters = 15; cfg->early_stop_rel = 1e-3f; cfg->n_dq = 1; cfg->n_beta = 1;
       cfg->flags = SOAR_FLAG_COUPLED_SCALE;
       return SOAR_OK;
+    case SOAR_PRESET_COUPLED_PAIR:
+      cfg->max_iters = 15; cfg->early_stop_rel = 1e-3f; cfg->n_dq = 2; cfg->n_beta = 1;
+      cfg->flags = SOAR_FLAG_COUPLED_SCALE;
+      return SOAR_OK;
     case SOAR_PRESET_DSS_ONLY:
       cfg->max_iters = 1; cfg->early_stop_rel = 0.0f; cfg->n_dq = 2; cfg->n_beta = 101;
       cfg->flags = SOAR_FLAG_KEEP_ALPHA | SOAR_FLAG_KEEP_BLOCK_SCALE;
@@ -1326,7 +1347,7 @@ int soar_quantize_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* 
   uint8_t* next = headers + static_cast<size_t>(n) * kWsFixedBytes;
   if (cudaMemsetAsync(headers, 0, static_cast<size_t>(n) * kWsFixedBytes, st) != cudaSuccess) return SOAR_ERR_CUDA;
 
-  const bool single = cfg->n_beta == 1 && cfg->n_dq <= 2 && !(cfg->flags & SOAR_FLAG_COUPLED_SCALE);
+  const bool single = cfg->n_beta == 1 && cfg->n_dq <= 2;
   const bool may_stop = cfg->early_stop_rel > 0.0f;
   for (int first = 0; first < n; first += kMaxBatch) {
     Batch bt;
@@ -1384,16 +1405,19 @@ int soar_quantize_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* 
       init_kernel<<<persistent_grid(init_kernel, tiles, kThreads), kThreads, 0, st>>>(bt, reverse,
                                                                                       cfg->max_iters == 0 ? 1 : 0);
     }
-    const unsigned int g_it = single ? persistent_grid(iterate_kernel<true>, tiles, kThreads)
-                                     : persistent_grid(iterate_kernel<false>, tiles, kThreads);
+    const int mode = !single ? 0 : ((cfg->flags & SOAR_FLAG_COUPLED_SCALE) ? 2 : 1);
+    const unsigned int g_it = mode == 0   ? persistent_grid(iterate_kernel<0>, tiles, kThreads)
+                              : mode == 1 ? persistent_grid(iterate_kernel<1>, tiles, kThreads)
+                                          : persistent_grid(iterate_kernel<2>, tiles, kThreads);
     for (int t = 0; t < cfg->max_iters; ++t) {
       reverse ^= 1;
       // with the early stop on, any iteration may turn out to be the last one
       const int last = (t == cfg->max_iters - 1) ? 1 : 0;
       const int emit = (may_stop || last) ? 1 : 0;
       ScopedLaunch sl(K_ITERATE, st);
-      if (single) iterate_kernel<true><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
-      else iterate_kernel<false><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
+      if (mode == 0) iterate_kernel<0><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
+      else if (mode == 1) iterate_kernel<1><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
+      else iterate_kernel<2><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
     }
     {
       ScopedLaunch sl(K_FINALIZE, st);

@@ -35,6 +35,16 @@ def test_config4_whole_tensors_paper_preset(tensor):
     print(wl.tensors[tensor].name, rep)
 
 
+def test_config4_whole_tensor_coupled_pair_preset():
+    """q (8192 x 8192) with two coupled candidates per block: several HBM-bound iterations."""
+    wl = WL.config4()
+    w = WL.generate(wl, 0)
+    cfg = api.soar_default_cfg(api.PRESET_COUPLED_PAIR)
+    ref_cfg = R.RefCfg(n_dq=2, n_beta=1, flags=R.FLAG_COUPLED_SCALE)
+    rep = P.assert_parity(P.run_gpu(w, cfg), R.quantize(w, ref_cfg))
+    print("q, coupled pair:", rep)
+
+
 def test_config4_largest_tensor():
     """gate: 28672 x 8192 (470 MB, several times the L2)."""
     wl = WL.config4()

@@ -28,6 +28,7 @@ pytestmark = pytest.mark.gpu
     dict(max_iters=3, early_stop_rel=0.0, n_dq=1, n_beta=1),  # CJSO with the nearest scale
     dict(max_iters=2, early_stop_rel=0.0, n_dq=4, n_beta=6, beta_step_pct=3),
     dict(flags=1, n_dq=1, n_beta=1),                                        # Sec. 3.2 alone (coupled scale)
+    dict(flags=1, n_dq=2, n_beta=1),                                        # both bracketing codes, coupled
     dict(flags=1, max_iters=2, early_stop_rel=0.0, n_dq=2, n_beta=3, beta_step_pct=5),
     dict(flags=6, max_iters=1, early_stop_rel=0.0),                          # Sec. 3.3 alone (2 x 101 search)
     dict(flags=6, max_iters=2, early_stop_rel=0.0, n_dq=4, n_beta=7, beta_step_pct=4),
@@ -115,6 +116,7 @@ def test_presets_of_the_stand_alone_arms_match_the_oracle():
     w = WL.small_case(96, 1024, 61, outlier_cols_frac=0.004, outlier_scale=20.0)
     for preset, ref_cfg in (
             (api.PRESET_CJSO_ONLY, R.RefCfg(n_dq=1, n_beta=1, flags=R.FLAG_COUPLED_SCALE)),
+            (api.PRESET_COUPLED_PAIR, R.RefCfg(n_dq=2, n_beta=1, flags=R.FLAG_COUPLED_SCALE)),
             (api.PRESET_DSS_ONLY, R.RefCfg(max_iters=1, early_stop_rel=0.0,
                                            flags=R.FLAG_KEEP_ALPHA | R.FLAG_KEEP_BLOCK_SCALE))):
         P.assert_parity(P.run_gpu(w, api.soar_default_cfg(preset)), R.quantize(w, ref_cfg))

@@ -90,3 +90,17 @@ def test_full_method_beats_both_arms_on_a_synthetic_tensor():
     dss = R.quantize(w, R.RefCfg(flags=R.FLAG_KEEP_ALPHA | R.FLAG_KEEP_BLOCK_SCALE, **DSS)).trace_sse[-1]
     full = R.quantize(w, R.RefCfg()).trace_sse[-1]
     assert full <= min(cjso.trace_sse.min(), dss) and max(cjso.trace_sse.min(), dss) <= rtn
+
+
+def test_two_coupled_candidates_end_where_the_full_search_ends():
+    """An observation on synthetic weights, not a claim of the paper: for a fixed dequantization
+    scale the best codes are the nearest ones under that same scale, so trying each of the two
+    bracketing E4M3 codes with itself as quantization scale (2 candidates per block) reaches the
+    error the 202-pair search reaches."""
+    for seed, kw in ((13, dict(outlier_cols_frac=0.004, outlier_scale=20.0)),
+                     (5, dict(dist="laplace", outlier_entry_frac=0.0005, outlier_scale=50.0)),
+                     (7, dict(dist="gauss_t2mix"))):
+        w = WL.small_case(96, 1024, seed, **kw)
+        full = R.quantize(w, R.RefCfg()).trace_sse[-1]
+        pair = R.quantize(w, R.RefCfg(flags=R.FLAG_COUPLED_SCALE, n_dq=2, n_beta=1)).trace_sse[-1]
+        assert pair <= full * 1.003
