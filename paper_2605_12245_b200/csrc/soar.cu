@@ -9,6 +9,10 @@
 //   finalize_kernel  early-stop bookkeeping (Sec. 4.1), alpha and the report
 //   swizzle_kernel   optional 128x4-tiled copy of the block scales
 //
+// Batches.  Every kernel works on up to 16 matrices at once: their tiles form one sequence
+// walked by one persistent grid, so a model's many small matrices share launches; a single
+// matrix is a batch of one.  Matrices that have stopped early drop out of later iterations.
+//
 // Data movement.  The three passes over W are persistent, warp-specialised kernels: each CTA
 // walks tiles of 256 blocks (8 KB of bf16).  One thread of a producer warp fetches them with
 // bulk asynchronous copies (cp.async.bulk, completion on a "full" mbarrier) into a
