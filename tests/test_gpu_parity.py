@@ -203,6 +203,28 @@ def test_a_call_replays_from_a_cuda_graph():
     P.assert_parity(gpu, R.quantize(w, ref_cfg))
 
 
+def test_host_entry_point_and_launch_trace():
+    """soar_quantize_host (copies in, quantizes, copies out on one stream) against a direct call;
+    the launch trace names every kernel of the call."""
+    w = WL.small_case(130, 2064, 91, outlier_entry_frac=0.003, outlier_scale=30.0)
+    cfg, _ = P.cfg_pair(max_iters=2, early_stop_rel=0.0)
+    want = P.run_gpu(w, cfg)
+    hb = api.alloc_host_buffers(w.shape[0], w.shape[1], cfg)
+    hb.W.copy_(torch.from_numpy(w.view(np.int16)).view(torch.bfloat16))
+    dev_W = torch.empty(w.shape, dtype=torch.bfloat16, device="cuda")
+    dev = api.alloc_buffers(w.shape[0], w.shape[1], cfg)
+    api.soar_trace_begin()
+    api.soar_quantize_host(hb, cfg, dev_W, dev)
+    torch.cuda.synchronize()
+    trace = api.soar_trace_end()
+    assert np.array_equal(hb.packed.numpy(), want.packed) and np.array_equal(hb.scales.numpy(), want.scales)
+    assert float(hb.alpha[0]) == want.alpha and hb.read_result().iters_run == 2
+    assert {k: v[0] for k, v in trace.items()} == {"amax_kernel": 1, "init_kernel": 1, "iterate_kernel": 2,
+                                                   "finalize_kernel": 1}
+    assert sum(v[0] for v in trace.values()) == api.soar_quantize_launches(cfg)
+    assert all(v[1] > 0 for v in trace.values())
+
+
 def test_host_pipeline_returns_what_direct_calls_return():
     """Seven matrices through three staging slots: every slot is reused, sizes differ."""
     shapes = [(64, 1024), (16, 256), (300, 512), (8, 4096), (130, 2064), (1, 16), (257, 1024)]
