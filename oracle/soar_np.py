@@ -80,14 +80,19 @@ def dq_candidates(center: np.ndarray, n: int, vals: np.ndarray) -> np.ndarray:
 
 
 def quantize(w_bits: np.ndarray, max_iters=15, early_stop_rel=1e-3, n_dq=2, n_beta=101,
-             beta_step_pct=1, coupled_scale=False, keep_alpha=False, keep_block_scale=False):
+             beta_step_pct=1, coupled_scale=False, keep_alpha=False, keep_block_scale=False, h=None):
     """Algorithm 1 on uint16 bf16 bit patterns [rows, cols]; returns a dict.
 
     The three switches give the paper's stand-alone arms: ``coupled_scale`` is Sec. 3.2's
     scheme (one block scale quantizes and dequantizes: a candidate's quantization scale is its
     own E4M3 value times beta); ``keep_alpha`` and ``keep_block_scale`` together are Sec. 3.3
-    alone (no Eq. 5, no Eq. 6: the search runs around the max-based start)."""
+    alone (no Eq. 5, no Eq. 6: the search runs around the max-based start).
+
+    ``h`` (float32, one per column, optional) weights every element's term of the objective:
+    the diagonal form of the output-distortion objective of Sec. 5."""
     rows, cols = w_bits.shape
+    hb = (np.ones(cols) if h is None else np.asarray(h, np.float32).astype(np.float64))
+    hb = np.tile(hb.reshape(-1, 16), (rows, 1))           # [nblk, 16] weights of each block's columns
     wf = (w_bits.astype(np.uint32) << np.uint32(16)).view(F32)
     sign = (w_bits >> 15).astype(np.uint8).reshape(-1, 16)
     mag = np.abs(wf).reshape(-1, 16).astype(F32)
@@ -109,7 +114,7 @@ def quantize(w_bits: np.ndarray, max_iters=15, early_stop_rel=1e-3, n_dq=2, n_be
     def err(m, a, d):
         s = np.float64(a) * vals[d]
         e = mag64 - m * s[:, None]
-        return seq_sum(e * e)
+        return seq_sum(hb * (e * e))
 
     m = reround(mag, alpha, dq)
     m[~live] = 0
@@ -120,8 +125,8 @@ def quantize(w_bits: np.ndarray, max_iters=15, early_stop_rel=1e-3, n_dq=2, n_be
     for t_it in range(max_iters):
         m = reround(mag, alpha, dq)
         m[~live] = 0
-        A = seq_sum(mag64 * m)
-        B = seq_sum(m * m)
+        A = seq_sum((hb * mag64) * m)
+        B = seq_sum(hb * (m * m))
         num = math.fsum((A * vals[dd])[live])
         den = math.fsum((B * vals[dd] ** 2)[live])
         alpha_new = F32(num / den) if den > 0 else alpha  # Eq. 5

@@ -8,6 +8,12 @@
  * blocking, fusion or reuse: every candidate pair re-rounds the whole block and
  * sums its squared error term by term.
  *
+ * Optional column weights (Sec. 5, "Discussions and Future Works": the output
+ * distortion ||(W - What) X||^2, taken here in its diagonal form): with h_j >= 0
+ * per input column the objective is sum_ij h_j (W_ij - What_ij)^2, and every
+ * per-element term of Eq. 4-8 carries its column's h_j.  Without weights h_j = 1
+ * and the arithmetic is the unweighted one, operation for operation.
+ *
  * Arithmetic convention.  Every quantity that feeds a discrete decision (a
  * rounding to the E2M1 grid, a projection to E4M3) is a fixed sequence of IEEE
  * binary32 round-to-nearest operations, written out where it happens; every sum
@@ -21,7 +27,8 @@
  * Pins (see the CPU tests): E2M1 grid and E4M3 range from Sec. 3.1; rounding
  * against an independent library cast; Eq. 5/6 against brute-force minimisation;
  * the Eq. 8 argmin against a separate NumPy enumeration; grid-aligned tensors
- * against their closed-form result.  Parity unpinned: the early-stop trajectory
+ * against their closed-form result; the weighted form against weighted least
+ * squares, constant weights and zero-weight columns.  Parity unpinned: the early-stop trajectory
  * and the iteration-to-iteration path (the paper prints no numbers for them);
  * those rest on agreement between this file and the NumPy restatement.
  */
@@ -46,6 +53,7 @@
 #define REF_STATUS_ZERO_TENSOR 1
 #define REF_STATUS_NONFINITE 2
 #define REF_STATUS_RANGE 4
+#define REF_STATUS_BAD_WEIGHT 16   /* a column weight that is negative, not finite, or outside {0} u [2^-20, 2^20] */
 
 typedef struct soar_ref_cfg {
   int32_t max_iters;      /* T of Algorithm 1; 0 = max-based NVFP4 only (Eq. 1-3) */
@@ -130,10 +138,12 @@ uint8_t soar_ref_e4m3_encode(float v) {
 /* Re-rounding of one block under scales (alpha, dq) (Eq. 2; Algorithm 1 "Compute
  * FP4 assignment"): s = fl32(alpha*dq), r = fl32(1/s), x_j = fl32(|W_j|*r),
  * m_j = E2M1 rounding of x_j.  Writes magnitudes m[16]; returns through A, B the
- * binary64 sums  A = sum |W_j| m_j,  B = sum m_j^2  (the block's terms of Eq. 5/6;
- * W_j and Q_j share a sign, so W_j Q_j = |W_j| m_j). */
-void soar_ref_round_block(const uint16_t* w, float alpha, float dq, double* m,
-                          double* A, double* B) {
+ * binary64 sums  A = sum h_j |W_j| m_j,  B = sum h_j m_j^2  (the block's terms of Eq. 5/6;
+ * W_j and Q_j share a sign, so W_j Q_j = |W_j| m_j).  h points at the block's 16 column
+ * weights, or is NULL for h_j = 1.  Each product is exact in binary64 (24 + 8 + 2 and
+ * 24 + 4 significant bits); the sums run in element order. */
+void soar_ref_round_block_w(const uint16_t* w, const float* h, float alpha, float dq, double* m,
+                            double* A, double* B) {
   float s = alpha * dq;
   float r = 1.0f / s;
   double a = 0.0, b = 0.0;
@@ -141,25 +151,38 @@ void soar_ref_round_block(const uint16_t* w, float alpha, float dq, double* m,
     float mag = fabsf(soar_ref_bf16_to_f32(w[j]));
     float x = mag * r;
     double mj = soar_ref_e2m1_round((double)x);
+    double hj = h ? (double)h[j] : 1.0;
     m[j] = mj;
-    a += (double)mag * mj;
-    b += mj * mj;
+    a += (hj * (double)mag) * mj;
+    b += hj * (mj * mj);
   }
   *A = a;
   *B = b;
 }
 
+void soar_ref_round_block(const uint16_t* w, float alpha, float dq, double* m,
+                          double* A, double* B) {
+  soar_ref_round_block_w(w, NULL, alpha, dq, m, A, B);
+}
+
 /* Block reconstruction error of Eq. 8 for magnitudes m and dequantization scale
- * code d under global scale alpha:  sum_j (|W_j| - m_j * alpha*value(d))^2. */
-double soar_ref_block_error(const uint16_t* w, const double* m, float alpha, uint8_t d) {
+ * code d under global scale alpha:  sum_j h_j (|W_j| - m_j * alpha*value(d))^2
+ * (h == NULL: h_j = 1). */
+double soar_ref_block_error_w(const uint16_t* w, const float* h, const double* m, float alpha,
+                              uint8_t d) {
   double s = (double)alpha * (double)soar_ref_e4m3_decode(d);
   double L = 0.0;
   for (int j = 0; j < REF_BLOCK; ++j) {
     double mag = fabs((double)soar_ref_bf16_to_f32(w[j]));
+    double hj = h ? (double)h[j] : 1.0;
     double e = mag - m[j] * s;
-    L += e * e;
+    L += hj * (e * e);
   }
   return L;
+}
+
+double soar_ref_block_error(const uint16_t* w, const double* m, float alpha, uint8_t d) {
+  return soar_ref_block_error_w(w, NULL, m, alpha, d);
 }
 
 /* Eq. 6 / Algorithm 1 "Update block-wise scale": A/(alpha*B) as binary32 steps.
@@ -208,7 +231,8 @@ float soar_ref_beta(int k, int n_beta, int step_pct) {
  * minimum wins.  Returns the winner through dq_out/d_out/L_out and, through
  * gap_rel, the relative gap to the best candidate whose outcome (16 magnitudes,
  * scale code) differs from the winner's (1e300 if there is none). */
-static void dss_block(const uint16_t* w, float alpha, float center, const soar_ref_cfg* cfg,
+static void dss_block(const uint16_t* w, const float* h, float alpha, float center,
+                      const soar_ref_cfg* cfg,
                       float* dq_out, uint8_t* d_out, double* L_out, double* A_out,
                       double* B_out, double* gap_rel) {
   uint8_t dc[REF_MAX_DQ];
@@ -228,8 +252,8 @@ static void dss_block(const uint16_t* w, float alpha, float center, const soar_r
     for (int d = 0; d < nd; ++d) {
       float dq = (coupled ? soar_ref_e4m3_decode(dc[d]) : center) * beta;
       dqk[k][d] = dq;
-      soar_ref_round_block(w, alpha, dq, mk[k][d], &Ak[k][d], &Bk[k][d]);
-      double L = soar_ref_block_error(w, mk[k][d], alpha, dc[d]);
+      soar_ref_round_block_w(w, h, alpha, dq, mk[k][d], &Ak[k][d], &Bk[k][d]);
+      double L = soar_ref_block_error_w(w, h, mk[k][d], alpha, dc[d]);
       Lk[k][d] = L;
       if (bk < 0 || L < best) { best = L; bk = k; bd = d; }
     }
@@ -264,14 +288,16 @@ static void dss_block(const uint16_t* w, float alpha, float center, const soar_r
  *   trace_sse   [max_iters+1]: error of the initial state, then after each executed iteration
  *   tie_flags   per block (may be NULL): 1 if in any executed iteration the best two
  *               distinct candidate outcomes were closer than tie_rel (relative)
- *   out_sumsq   sum of W^2 (may be NULL)
+ *   out_sumsq   sum of h_j W^2 (may be NULL)
+ *   h           cols column weights (Sec. 5 in diagonal form), or NULL for h_j = 1; the
+ *               initialization (Eq. 1) does not depend on them
  * Returns status bits; *iters_run = executed iterations.
  */
-int soar_ref_quantize(const uint16_t* W, int64_t rows, int64_t cols, int64_t ld,
-                      const soar_ref_cfg* cfg, uint8_t* out_packed, uint8_t* out_scales,
-                      float* out_alpha, int32_t* iters_run, double* trace_alpha,
-                      double* trace_sse, uint8_t* tie_flags, double tie_rel,
-                      double* out_sumsq) {
+int soar_ref_quantize_weighted(const uint16_t* W, int64_t rows, int64_t cols, int64_t ld,
+                               const float* h, const soar_ref_cfg* cfg, uint8_t* out_packed,
+                               uint8_t* out_scales, float* out_alpha, int32_t* iters_run,
+                               double* trace_alpha, double* trace_sse, uint8_t* tie_flags,
+                               double tie_rel, double* out_sumsq) {
   const int64_t nbc = cols / REF_BLOCK;
   const int64_t nblk = rows * nbc;
   int status = 0;
@@ -285,11 +311,16 @@ int soar_ref_quantize(const uint16_t* W, int64_t rows, int64_t cols, int64_t ld,
       float v = fabsf(soar_ref_bf16_to_f32(W[r * ld + c]));
       if (!(v <= 3.4e38f)) status |= REF_STATUS_NONFINITE;
       if (v > amax) amax = v;
-      sumsq += (double)v * (double)v;
+      sumsq += (h ? (double)h[c] : 1.0) * ((double)v * (double)v);
+    }
+  if (h)
+    for (int64_t c = 0; c < cols; ++c) {
+      float hv = h[c];
+      if (!(hv == 0.0f || (hv >= 0x1p-20f && hv <= 0x1p20f))) status |= REF_STATUS_BAD_WEIGHT;
     }
   if (out_sumsq) *out_sumsq = sumsq;
   if (tie_flags) memset(tie_flags, 0, (size_t)nblk);
-  if (status & REF_STATUS_NONFINITE) return status;
+  if (status & (REF_STATUS_NONFINITE | REF_STATUS_BAD_WEIGHT)) return status;
   if (amax == 0.0f) {
     /* all-zero tensor: alpha = 1, zero scales, codes carry only the input's sign bit */
     for (int64_t r = 0; r < rows; ++r)
@@ -335,8 +366,9 @@ int soar_ref_quantize(const uint16_t* W, int64_t rows, int64_t cols, int64_t ld,
       dd[i] = c;
       dq[i] = soar_ref_e4m3_decode(c);
       double m[REF_BLOCK], A, B;
-      soar_ref_round_block(w, alpha, dq[i], m, &A, &B);
-      sL += soar_ref_block_error(w, m, alpha, c);
+      const float* hb = h ? h + b * REF_BLOCK : NULL;
+      soar_ref_round_block_w(w, hb, alpha, dq[i], m, &A, &B);
+      sL += soar_ref_block_error_w(w, hb, m, alpha, c);
     }
     rowL[r] = sL;
   }
@@ -356,7 +388,8 @@ int soar_ref_quantize(const uint16_t* W, int64_t rows, int64_t cols, int64_t ld,
         int64_t i = r * nbc + b;
         if (dd[i] == 0) continue;
         double m[REF_BLOCK], A, B;
-        soar_ref_round_block(W + r * ld + b * REF_BLOCK, alpha, dq[i], m, &A, &B);
+        soar_ref_round_block_w(W + r * ld + b * REF_BLOCK, h ? h + b * REF_BLOCK : NULL, alpha,
+                               dq[i], m, &A, &B);
         double v = (double)soar_ref_e4m3_decode(dd[i]);
         sA += A * v;
         sB += B * v * v;
@@ -379,15 +412,16 @@ int soar_ref_quantize(const uint16_t* W, int64_t rows, int64_t cols, int64_t ld,
         int64_t i = r * nbc + b;
         if (dd[i] == 0) continue;
         const uint16_t* w = W + r * ld + b * REF_BLOCK;
+        const float* hb = h ? h + b * REF_BLOCK : NULL;
         double m[REF_BLOCK], A, B;
-        soar_ref_round_block(w, alpha, dq[i], m, &A, &B);
+        soar_ref_round_block_w(w, hb, alpha, dq[i], m, &A, &B);
         float center = (cfg->flags & REF_FLAG_KEEP_BLOCK_SCALE)
                            ? soar_ref_e4m3_decode(dd[i])                  /* Sec. 3.3 alone: around the stored scale */
                            : soar_ref_block_scale(A, B, alpha_new, dd[i]);
         float ndq;
         uint8_t nd;
         double L, wA, wB, gap;
-        dss_block(w, alpha_new, center, cfg, &ndq, &nd, &L, &wA, &wB, &gap);
+        dss_block(w, hb, alpha_new, center, cfg, &ndq, &nd, &L, &wA, &wB, &gap);
         dq[i] = ndq;
         dd[i] = nd;
         sL += L;
@@ -433,11 +467,21 @@ int soar_ref_quantize(const uint16_t* W, int64_t rows, int64_t cols, int64_t ld,
   return status;
 }
 
-/* Eq. 3 + Eq. 4 on stored outputs: sum (W - Q*alpha*value(d))^2 and sum W^2,
- * element by element in binary64. */
-void soar_ref_dequant_error(const uint16_t* W, int64_t rows, int64_t cols, int64_t ld,
-                            const uint8_t* packed, const uint8_t* scales, float alpha,
-                            double* out_sse, double* out_sumsq) {
+/* Algorithm 1 as the paper states it: every h_j = 1. */
+int soar_ref_quantize(const uint16_t* W, int64_t rows, int64_t cols, int64_t ld,
+                      const soar_ref_cfg* cfg, uint8_t* out_packed, uint8_t* out_scales,
+                      float* out_alpha, int32_t* iters_run, double* trace_alpha,
+                      double* trace_sse, uint8_t* tie_flags, double tie_rel,
+                      double* out_sumsq) {
+  return soar_ref_quantize_weighted(W, rows, cols, ld, NULL, cfg, out_packed, out_scales, out_alpha,
+                                    iters_run, trace_alpha, trace_sse, tie_flags, tie_rel, out_sumsq);
+}
+
+/* Eq. 3 + Eq. 4 on stored outputs: sum h_j (W - Q*alpha*value(d))^2 and sum h_j W^2,
+ * element by element in binary64 (h == NULL: h_j = 1). */
+void soar_ref_dequant_error_weighted(const uint16_t* W, int64_t rows, int64_t cols, int64_t ld,
+                                     const float* h, const uint8_t* packed, const uint8_t* scales,
+                                     float alpha, double* out_sse, double* out_sumsq) {
   static const double grid[8] = {0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0};
   const int64_t nbc = cols / REF_BLOCK;
   double sse = 0.0, ss = 0.0;
@@ -448,12 +492,19 @@ void soar_ref_dequant_error(const uint16_t* W, int64_t rows, int64_t cols, int64
       int code = (c & 1) ? (byte >> 4) : (byte & 0xF);
       double q = grid[code & 7] * ((code & 8) ? -1.0 : 1.0);
       double s = (double)alpha * (double)soar_ref_e4m3_decode(scales[r * nbc + c / REF_BLOCK]);
+      double hj = h ? (double)h[c] : 1.0;
       double e = w - q * s;
-      sse += e * e;
-      ss += w * w;
+      sse += hj * (e * e);
+      ss += hj * (w * w);
     }
   *out_sse = sse;
   *out_sumsq = ss;
+}
+
+void soar_ref_dequant_error(const uint16_t* W, int64_t rows, int64_t cols, int64_t ld,
+                            const uint8_t* packed, const uint8_t* scales, float alpha,
+                            double* out_sse, double* out_sumsq) {
+  soar_ref_dequant_error_weighted(W, rows, cols, ld, NULL, packed, scales, alpha, out_sse, out_sumsq);
 }
 
 int soar_ref_num_threads(void) {

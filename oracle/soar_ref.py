@@ -22,6 +22,7 @@ _LIB = os.path.join(_HERE, "libsoar_ref.so")
 STATUS_ZERO_TENSOR = 1
 STATUS_NONFINITE = 2
 STATUS_RANGE = 4
+STATUS_BAD_WEIGHT = 16
 
 FLAG_COUPLED_SCALE, FLAG_KEEP_ALPHA, FLAG_KEEP_BLOCK_SCALE = 1, 2, 4
 
@@ -100,6 +101,11 @@ def lib() -> C.CDLL:
         L.soar_ref_round_block.argtypes = [u16p, C.c_float, C.c_float, dp, dp, dp]
         L.soar_ref_block_error.restype = C.c_double
         L.soar_ref_block_error.argtypes = [u16p, dp, C.c_float, C.c_uint8]
+        fp = C.POINTER(C.c_float)
+        L.soar_ref_round_block_w.restype = None
+        L.soar_ref_round_block_w.argtypes = [u16p, fp, C.c_float, C.c_float, dp, dp, dp]
+        L.soar_ref_block_error_w.restype = C.c_double
+        L.soar_ref_block_error_w.argtypes = [u16p, fp, dp, C.c_float, C.c_uint8]
         L.soar_ref_block_scale.restype = C.c_float
         L.soar_ref_block_scale.argtypes = [C.c_double, C.c_double, C.c_float, C.c_uint8]
         L.soar_ref_dq_candidates.restype = C.c_int
@@ -114,6 +120,15 @@ def lib() -> C.CDLL:
         L.soar_ref_dequant_error.restype = None
         L.soar_ref_dequant_error.argtypes = [
             u16p, C.c_int64, C.c_int64, C.c_int64, u8p, u8p, C.c_float, dp, dp,
+        ]
+        L.soar_ref_quantize_weighted.restype = C.c_int
+        L.soar_ref_quantize_weighted.argtypes = [
+            u16p, C.c_int64, C.c_int64, C.c_int64, fp, C.POINTER(_Cfg), u8p, u8p,
+            C.POINTER(C.c_float), C.POINTER(C.c_int32), dp, dp, u8p, C.c_double, dp,
+        ]
+        L.soar_ref_dequant_error_weighted.restype = None
+        L.soar_ref_dequant_error_weighted.argtypes = [
+            u16p, C.c_int64, C.c_int64, C.c_int64, fp, u8p, u8p, C.c_float, dp, dp,
         ]
         L.soar_ref_num_threads.restype = C.c_int
         _lib = L
@@ -132,11 +147,27 @@ def num_threads() -> int:
     return int(lib().soar_ref_num_threads())
 
 
-def quantize(w_bits: np.ndarray, cfg: RefCfg, tie_rel: float = 1e-6) -> RefResult:
-    """Run Algorithm 1 on a 2-D uint16 array of bf16 bit patterns (row stride = shape[1])."""
+def _f32(a: np.ndarray):
+    return a.ctypes.data_as(C.POINTER(C.c_float))
+
+
+def _weights(h, cols: int):
+    """Column weights as a contiguous float32 array of ``cols`` entries (None stays None)."""
+    if h is None:
+        return None
+    h = np.ascontiguousarray(h, dtype=np.float32)
+    assert h.shape == (cols,)
+    return h
+
+
+def quantize(w_bits: np.ndarray, cfg: RefCfg, tie_rel: float = 1e-6, h=None) -> RefResult:
+    """Run Algorithm 1 on a 2-D uint16 array of bf16 bit patterns (row stride = shape[1]).
+
+    ``h``: optional float32 column weights of the objective (Sec. 5, diagonal form)."""
     assert w_bits.dtype == np.uint16 and w_bits.ndim == 2
     rows, cols = w_bits.shape
     assert cols % 16 == 0
+    h = _weights(h, cols)
     w = np.ascontiguousarray(w_bits)
     packed = np.zeros((rows, cols // 2), np.uint8)
     scales = np.zeros((rows, cols // 16), np.uint8)
@@ -147,25 +178,32 @@ def quantize(w_bits: np.ndarray, cfg: RefCfg, tie_rel: float = 1e-6) -> RefResul
     iters = C.c_int32(0)
     sumsq = C.c_double(0.0)
     c = cfg.c()
-    st = lib().soar_ref_quantize(
-        _u16(w), rows, cols, cols, C.byref(c), _u8(packed), _u8(scales), C.byref(alpha),
-        C.byref(iters), ta.ctypes.data_as(C.POINTER(C.c_double)),
-        ts.ctypes.data_as(C.POINTER(C.c_double)), _u8(ties), tie_rel, C.byref(sumsq),
-    )
+    tail = (C.byref(c), _u8(packed), _u8(scales), C.byref(alpha), C.byref(iters),
+            ta.ctypes.data_as(C.POINTER(C.c_double)), ts.ctypes.data_as(C.POINTER(C.c_double)),
+            _u8(ties), tie_rel, C.byref(sumsq))
+    if h is None:
+        st = lib().soar_ref_quantize(_u16(w), rows, cols, cols, *tail)
+    else:
+        st = lib().soar_ref_quantize_weighted(_u16(w), rows, cols, cols, _f32(h), *tail)
     n = iters.value + 1
     return RefResult(packed, scales, float(alpha.value), int(iters.value), ta[:n].copy(),
                      ts[:n].copy(), ties, float(sumsq.value), int(st))
 
 
-def dequant_error(w_bits: np.ndarray, packed: np.ndarray, scales: np.ndarray, alpha: float):
-    """Sum of squared reconstruction error (Eq. 3-4) and sum of squares of W."""
+def dequant_error(w_bits: np.ndarray, packed: np.ndarray, scales: np.ndarray, alpha: float, h=None):
+    """Sum of (column-weighted) squared reconstruction error (Eq. 3-4) and sum of squares of W."""
     rows, cols = w_bits.shape
     w = np.ascontiguousarray(w_bits)
     p = np.ascontiguousarray(packed, dtype=np.uint8)
     s = np.ascontiguousarray(scales, dtype=np.uint8)
+    h = _weights(h, cols)
     sse, ss = C.c_double(0.0), C.c_double(0.0)
-    lib().soar_ref_dequant_error(_u16(w), rows, cols, cols, _u8(p), _u8(s), C.c_float(alpha),
-                                 C.byref(sse), C.byref(ss))
+    if h is None:
+        lib().soar_ref_dequant_error(_u16(w), rows, cols, cols, _u8(p), _u8(s), C.c_float(alpha),
+                                     C.byref(sse), C.byref(ss))
+    else:
+        lib().soar_ref_dequant_error_weighted(_u16(w), rows, cols, cols, _f32(h), _u8(p), _u8(s),
+                                              C.c_float(alpha), C.byref(sse), C.byref(ss))
     return float(sse.value), float(ss.value)
 
 
@@ -187,22 +225,30 @@ def e4m3_encode(v: float) -> int:
     return int(lib().soar_ref_e4m3_encode(C.c_float(v)))
 
 
-def round_block(w16: np.ndarray, alpha: float, dq: float):
-    """Returns (m[16], A, B) for one block of bf16 bit patterns."""
+def round_block(w16: np.ndarray, alpha: float, dq: float, h=None):
+    """Returns (m[16], A, B) for one block of bf16 bit patterns (``h``: its 16 column weights)."""
     w = np.ascontiguousarray(w16, dtype=np.uint16)
     assert w.size == 16
     m = np.zeros(16, np.float64)
     A, B = C.c_double(0.0), C.c_double(0.0)
-    lib().soar_ref_round_block(_u16(w), C.c_float(alpha), C.c_float(dq),
-                               m.ctypes.data_as(C.POINTER(C.c_double)), C.byref(A), C.byref(B))
+    mp = m.ctypes.data_as(C.POINTER(C.c_double))
+    if h is None:
+        lib().soar_ref_round_block(_u16(w), C.c_float(alpha), C.c_float(dq), mp, C.byref(A), C.byref(B))
+    else:
+        hh = _weights(h, 16)
+        lib().soar_ref_round_block_w(_u16(w), _f32(hh), C.c_float(alpha), C.c_float(dq), mp,
+                                     C.byref(A), C.byref(B))
     return m, float(A.value), float(B.value)
 
 
-def block_error(w16: np.ndarray, m: np.ndarray, alpha: float, d: int) -> float:
+def block_error(w16: np.ndarray, m: np.ndarray, alpha: float, d: int, h=None) -> float:
     w = np.ascontiguousarray(w16, dtype=np.uint16)
     mm = np.ascontiguousarray(m, dtype=np.float64)
-    return float(lib().soar_ref_block_error(_u16(w), mm.ctypes.data_as(C.POINTER(C.c_double)),
-                                            C.c_float(alpha), C.c_uint8(d)))
+    mp = mm.ctypes.data_as(C.POINTER(C.c_double))
+    if h is None:
+        return float(lib().soar_ref_block_error(_u16(w), mp, C.c_float(alpha), C.c_uint8(d)))
+    hh = _weights(h, 16)
+    return float(lib().soar_ref_block_error_w(_u16(w), _f32(hh), mp, C.c_float(alpha), C.c_uint8(d)))
 
 
 def block_scale(A: float, B: float, alpha: float, d_cur: int) -> float:

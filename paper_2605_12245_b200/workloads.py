@@ -170,3 +170,25 @@ def small_case(rows: int, cols: int, seed: int, dist: str = "student_t4",
     wl = Workload(f"small_{rows}x{cols}", seed, dist, (TensorSpec("w", rows, cols),),
                   outlier_cols_frac, outlier_entry_frac, outlier_scale)
     return generate(wl, 0, workers=1)
+
+
+def column_weights(cols: int, seed: int, samples: int = 128, outlier_frac: float = 0.005,
+                   zero_frac: float = 0.0) -> np.ndarray:
+    """Synthetic per-column weights for the weighted objective: float32 [cols].
+
+    Stand-in for the diagonal of X X^T / n of a calibration batch: channel ``c`` has standard
+    deviation ``sigma_c`` (log-normal, with a fraction ``outlier_frac`` of channels 10-30 times
+    larger, as LLM activations show), and ``h_c = sigma_c^2 * chi2(samples) / samples``.  The
+    result is scaled to mean 1, clipped to [2^-20, 2^20]; a fraction ``zero_frac`` of the
+    columns is then set to zero (channels that never fire)."""
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, cols, 0x5EED])))
+    sigma = np.exp(0.5 * rng.standard_normal(cols))
+    n_out = int(round(outlier_frac * cols))
+    if n_out > 0:
+        idx = rng.choice(cols, size=n_out, replace=False)
+        sigma[idx] *= rng.uniform(10.0, 30.0, size=n_out)
+    h = sigma ** 2 * rng.chisquare(samples, size=cols) / samples
+    h = np.clip(h / h.mean(), 2.0 ** -20, 2.0 ** 20)
+    if zero_frac > 0.0:
+        h[rng.random(cols) < zero_frac] = 0.0
+    return h.astype(np.float32)
