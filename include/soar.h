@@ -40,6 +40,8 @@ extern "C" {
 #define SOAR_STATUS_NONFINITE 2        /* NaN or Inf in the input: outputs unspecified      */
 #define SOAR_STATUS_RANGE 4            /* max |W| outside [2^-100, 2^100]: outputs unspecified */
 #define SOAR_STATUS_INTERNAL 8         /* a bounded wait inside a kernel gave up: outputs unspecified */
+#define SOAR_STATUS_BAD_WEIGHT 16      /* a column weight negative, not finite, or non-zero outside
+                                          [2^-20, 2^20] (soar_quantize_weighted): outputs unspecified */
 
 /* scale_layout bits */
 #define SOAR_SCALES_LINEAR 1           /* row-major [rows][cols/16] bytes                   */
@@ -205,6 +207,46 @@ int soar_dequant_error(const void* W_bf16, int64_t rows, int64_t cols, int64_t l
                        const void* fp4_packed, const void* e4m3_scales, int scale_layout,
                        const float* global_fp32, double* out_sse, double* out_sumsq,
                        void* stream);
+
+/*
+ * SOAR with a column-weighted objective: sum_ij h_j (W_ij - What_ij)^2, h = col_weight.
+ * This is the diagonal form of the output-distortion objective ||(W - What) X||^2 that the
+ * paper's Sec. 5 ("Discussions and Future Works") proposes for CJSO and DSS: h_j stands for the
+ * second moment of input channel j over calibration data.  Algorithm 1 runs unchanged except
+ * that every per-element term carries its column's weight: the block sums of Eq. 5 and Eq. 6
+ * become A = sum h_j W_j Q_j and B = sum h_j Q_j^2, the error of Eq. 8 and of the early stop
+ * (Sec. 4.1) is the weighted one, and the report's sse, sse_init and sumsq are weighted.  The
+ * initialization (Eq. 1) does not depend on h; with every h_j = 1 the outputs are those of
+ * soar_quantize.
+ *
+ *   col_weight  device, `cols` floats, 16-byte aligned, read-only.  Each must be zero or lie in
+ *               [2^-20, 2^20]; anything else (negative, NaN, Inf, out of range) is reported as
+ *               SOAR_STATUS_BAD_WEIGHT in out_result->status and the outputs are unspecified.
+ *               Only ratios between weights matter to the minimiser.
+ *   workspace   device, 256-byte aligned, >= soar_weighted_workspace_bytes(rows, cols, cfg):
+ *               2 KB of accumulators plus, when max_iters > 0, 17 bytes per block (A and B in
+ *               binary64 and the stored scale code), plus rows*cols/16 bytes when the row-major
+ *               scale layout is not requested.
+ * Every other argument, the stream semantics, ownership and the error codes are those of
+ * soar_quantize.  One matrix per call; the block sums are accumulated in binary64 in element
+ * order, so the pass is bound by arithmetic, not by HBM, even with one candidate.
+ */
+size_t soar_weighted_workspace_bytes(int64_t rows, int64_t cols, const soar_cfg* cfg);
+int soar_quantize_weighted(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld,
+                           const float* col_weight, const soar_cfg* cfg, void* out_fp4_packed,
+                           void* out_e4m3_scales, void* out_e4m3_scales_sw, float* out_global_fp32,
+                           void* workspace, size_t workspace_bytes, soar_result* out_result,
+                           void* stream);
+
+/*
+ * soar_dequant_error under the same column weights: *out_sse = sum h_j (W - code value *
+ * alpha * scale)^2 and *out_sumsq = sum h_j W^2 (binary64).  col_weight as above (not
+ * validated here: a NaN weight gives NaN sums); the other arguments as soar_dequant_error.
+ */
+int soar_dequant_error_weighted(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld,
+                                const float* col_weight, const void* fp4_packed,
+                                const void* e4m3_scales, int scale_layout, const float* global_fp32,
+                                double* out_sse, double* out_sumsq, void* stream);
 
 /*
  * soar_quantize without a workspace argument, for callers that must not allocate device

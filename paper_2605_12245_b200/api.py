@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(HERE, "libsoar.so")
 
 SOAR_OK = 0
 STATUS_ZERO_TENSOR, STATUS_NONFINITE, STATUS_RANGE, STATUS_INTERNAL = 1, 2, 4, 8
+STATUS_BAD_WEIGHT = 16
 SCALES_LINEAR, SCALES_SWIZZLED = 1, 2
 PRESET_PAPER, PRESET_SINGLE_PASS, PRESET_RTN, PRESET_CJSO_ONLY, PRESET_DSS_ONLY, PRESET_COUPLED_PAIR = 0, 1, 2, 3, 4, 5
 FLAG_COUPLED_SCALE, FLAG_KEEP_ALPHA, FLAG_KEEP_BLOCK_SCALE = 1, 2, 4
@@ -28,6 +29,7 @@ EXPORTS = (
     "soar_dequant_error", "soar_quantize_launches", "soar_status_string", "soar_quantize_host",
     "soar_trace_begin", "soar_trace_end", "soar_quantize_static", "soar_selftest_reciprocal",
     "soar_batch_workspace_bytes", "soar_quantize_batch",
+    "soar_weighted_workspace_bytes", "soar_quantize_weighted", "soar_dequant_error_weighted",
 )
 
 
@@ -115,6 +117,13 @@ def lib() -> C.CDLL:
         L.soar_batch_workspace_bytes.argtypes = [C.POINTER(SoarTensorDesc), C.c_int, C.POINTER(SoarCfg)]
         L.soar_quantize_batch.restype = C.c_int
         L.soar_quantize_batch.argtypes = [C.POINTER(SoarTensorDesc), C.c_int, C.POINTER(SoarCfg), vp, C.c_size_t, vp]
+        L.soar_weighted_workspace_bytes.restype = C.c_size_t
+        L.soar_weighted_workspace_bytes.argtypes = [i64, i64, C.POINTER(SoarCfg)]
+        L.soar_quantize_weighted.restype = C.c_int
+        L.soar_quantize_weighted.argtypes = [vp, i64, i64, i64, vp, C.POINTER(SoarCfg), vp, vp, vp, vp, vp,
+                                             C.c_size_t, vp, vp]
+        L.soar_dequant_error_weighted.restype = C.c_int
+        L.soar_dequant_error_weighted.argtypes = [vp, i64, i64, i64, vp, vp, vp, C.c_int, vp, vp, vp, vp]
         L.soar_selftest_reciprocal.restype = C.c_int
         L.soar_selftest_reciprocal.argtypes = [C.c_int, C.c_int, vp, vp]
         L.soar_trace_begin.restype = C.c_int
@@ -186,12 +195,17 @@ class QuantBuffers:
         return SoarResult.from_buffer_copy(raw)
 
 
-def alloc_buffers(rows: int, cols: int, cfg: SoarCfg, device="cuda") -> QuantBuffers:
+def soar_weighted_workspace_bytes(rows: int, cols: int, cfg: SoarCfg) -> int:
+    return int(lib().soar_weighted_workspace_bytes(rows, cols, C.byref(cfg)))
+
+
+def alloc_buffers(rows: int, cols: int, cfg: SoarCfg, device="cuda", weighted: bool = False) -> QuantBuffers:
+    """Output buffers and workspace for one matrix (``weighted``: sized for soar_quantize_weighted)."""
     u8 = dict(dtype=torch.uint8, device=device)
     lin = torch.empty((rows, cols // 16), **u8) if cfg.scale_layout & SCALES_LINEAR else None
     sw = (torch.empty(soar_swizzled_scale_bytes(rows, cols), **u8)
           if cfg.scale_layout & SCALES_SWIZZLED else None)
-    ws_bytes = soar_workspace_bytes(rows, cols, cfg)
+    ws_bytes = (soar_weighted_workspace_bytes if weighted else soar_workspace_bytes)(rows, cols, cfg)
     if ws_bytes == 0:
         raise SoarError("soar_workspace_bytes rejected the shape or cfg")
     return QuantBuffers(
@@ -218,6 +232,26 @@ def soar_quantize(W: torch.Tensor, cfg: SoarCfg, out: QuantBuffers | None = None
         _ptr(out.scales_sw), _ptr(out.alpha), _ptr(out.workspace), out.workspace.numel(),
         _ptr(out.result), _stream_ptr(stream))
     _check(rc, "soar_quantize")
+    return out
+
+
+def soar_quantize_weighted(W: torch.Tensor, col_weight: torch.Tensor, cfg: SoarCfg,
+                           out: QuantBuffers | None = None, stream=None) -> QuantBuffers:
+    """Enqueue ``soar_quantize_weighted``: ``col_weight`` is a float32 CUDA vector of W.shape[1] entries."""
+    _require_cuda(W, col_weight)
+    if W.dtype != torch.bfloat16 or W.dim() != 2 or W.stride(1) != 1:
+        raise SoarError("W must be a 2-D bf16 tensor with unit column stride")
+    rows, cols = W.shape
+    if col_weight.dtype != torch.float32 or col_weight.shape != (cols,) or not col_weight.is_contiguous():
+        raise SoarError("col_weight must be a contiguous float32 vector with one entry per column")
+    if out is None:
+        out = alloc_buffers(rows, cols, cfg, W.device, weighted=True)
+    _require_cuda(out.packed, out.scales, out.scales_sw, out.alpha, out.result, out.workspace)
+    rc = lib().soar_quantize_weighted(
+        _ptr(W), rows, cols, W.stride(0), _ptr(col_weight), C.byref(cfg), _ptr(out.packed), _ptr(out.scales),
+        _ptr(out.scales_sw), _ptr(out.alpha), _ptr(out.workspace), out.workspace.numel(),
+        _ptr(out.result), _stream_ptr(stream))
+    _check(rc, "soar_quantize_weighted")
     return out
 
 
@@ -284,6 +318,21 @@ def soar_dequant_error(W: torch.Tensor, packed: torch.Tensor, scales: torch.Tens
         _ptr(W), rows, cols, W.stride(0), _ptr(packed), _ptr(scales), scale_layout, _ptr(alpha),
         C.c_void_p(out.data_ptr()), C.c_void_p(out.data_ptr() + 8), _stream_ptr(stream))
     _check(rc, "soar_dequant_error")
+    return out
+
+
+def soar_dequant_error_weighted(W: torch.Tensor, col_weight: torch.Tensor, packed: torch.Tensor,
+                                scales: torch.Tensor, alpha: torch.Tensor, scale_layout: int = SCALES_LINEAR,
+                                stream=None, out: torch.Tensor | None = None) -> torch.Tensor:
+    """Enqueue ``soar_dequant_error_weighted``; returns a float64 CUDA tensor [sse, sumsq]."""
+    _require_cuda(W, col_weight, packed, scales, alpha)
+    rows, cols = W.shape
+    if out is None:
+        out = torch.empty(2, dtype=torch.float64, device=W.device)
+    rc = lib().soar_dequant_error_weighted(
+        _ptr(W), rows, cols, W.stride(0), _ptr(col_weight), _ptr(packed), _ptr(scales), scale_layout,
+        _ptr(alpha), C.c_void_p(out.data_ptr()), C.c_void_p(out.data_ptr() + 8), _stream_ptr(stream))
+    _check(rc, "soar_dequant_error_weighted")
     return out
 
 

@@ -52,7 +52,7 @@ constexpr unsigned int kWaitLimit = 1u << 22;  // mbarrier polls before a wait g
 
 struct Ws {
   unsigned int amax_bits;            // max over the tensor of the bf16 magnitude bit pattern
-  unsigned int error;                // non-zero when a bounded wait gave up
+  unsigned int error;                // kErr* bits; non-zero stops the remaining passes
   unsigned long long zero_blocks;
   unsigned long long wide;
   double sumsq;                      // sum W^2
@@ -61,6 +61,8 @@ struct Ws {
   double gsum[SOAR_MAX_ITERS + 1];   // stage s: sum of block errors minus sum W^2 (Eq. 4)
 };
 static_assert(sizeof(Ws) <= kWsFixedBytes, "workspace header too large");
+constexpr unsigned int kErrWait = 1u;     // a bounded wait gave up
+constexpr unsigned int kErrWeight = 2u;   // a column weight outside the accepted set
 
 struct Params {
   const uint16_t* W;
@@ -292,7 +294,7 @@ __device__ __forceinline__ bool is_producer_warp() { return threadIdx.x >= kTile
 
 __device__ __forceinline__ void record_failure(const Batch& bt) {
   for (int i = 0; i < bt.n; ++i)
-    if (bt.t[i].ws != nullptr) atomicOr(&bt.t[i].ws->error, 1u);
+    if (bt.t[i].ws != nullptr) atomicOr(&bt.t[i].ws->error, kErrWait);
 }
 
 // Producer (one thread): walks the CTA's share of the tile sequence (positions blockIdx.x,
@@ -519,6 +521,19 @@ __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
   return v;
+}
+
+// The sixteen column weights of block column cb, widened to binary64 (exact).
+__device__ __forceinline__ void load_weights(const float* h, unsigned int cb, double (&hd)[16]) {
+  const float4* src = reinterpret_cast<const float4*>(h) + static_cast<size_t>(cb) * 4;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const float4 v = __ldg(src + q);
+    hd[4 * q] = static_cast<double>(v.x);
+    hd[4 * q + 1] = static_cast<double>(v.y);
+    hd[4 * q + 2] = static_cast<double>(v.z);
+    hd[4 * q + 3] = static_cast<double>(v.w);
+  }
 }
 
 // Per-tensor partial sums of a CTA, in shared memory.  Each consumer warp adds its sums for a
@@ -770,14 +785,9 @@ __device__ __forceinline__ void iteration_head(const Params& p, int t, float& al
   run_out = run;
 }
 
-// Eq. 6 with the new alpha from the previous winner's sums (all codes zero keeps the stored
-// scale), and App. B.3's E4M3 codes around it: d_lo .. d_hi before clipping.
-__device__ __forceinline__ float block_center(const uint2 st, float alpha, int n_dq, bool keep, int& d_lo,
-                                              int& d_hi) {
-  const int d_cur = static_cast<int>(st.y >> 16);
-  const float B0 = 0.25f * static_cast<float>(st.y & 0xFFFFu);
-  const float center = (B0 > 0.0f && !keep) ? __fdiv_rn(__uint_as_float(st.x), __fmul_rn(alpha, B0))
-                                             : e4m3_value(d_cur);
+// App. B.3's E4M3 codes around a block's analytic scale: d_lo .. d_hi before clipping (the
+// nearest code alone for n_dq == 1, else n_dq codes bracketing the scale).
+__device__ __forceinline__ void candidate_window(float center, int n_dq, int& d_lo, int& d_hi) {
   const int cn = e4m3_encode(center);
   if (n_dq <= 1) {
     d_lo = d_hi = cn;
@@ -786,6 +796,17 @@ __device__ __forceinline__ float block_center(const uint2 st, float alpha, int n
     d_lo = cf - (n_dq / 2 - 1);
     d_hi = cf + n_dq / 2;
   }
+}
+
+// Eq. 6 with the new alpha from the previous winner's sums (all codes zero keeps the stored
+// scale), and the candidate codes around it.
+__device__ __forceinline__ float block_center(const uint2 st, float alpha, int n_dq, bool keep, int& d_lo,
+                                              int& d_hi) {
+  const int d_cur = static_cast<int>(st.y >> 16);
+  const float B0 = 0.25f * static_cast<float>(st.y & 0xFFFFu);
+  const float center = (B0 > 0.0f && !keep) ? __fdiv_rn(__uint_as_float(st.x), __fmul_rn(alpha, B0))
+                                             : e4m3_value(d_cur);
+  candidate_window(center, n_dq, d_lo, d_hi);
   return center;
 }
 
@@ -1035,7 +1056,8 @@ __global__ void __launch_bounds__(128) finalize_kernel(const __grid_constant__ B
     s_iters = iters;
     *out_alpha = alpha;
     if (res != nullptr) {
-      res->status = st | (ws->error ? SOAR_STATUS_INTERNAL : 0);
+      res->status = st | ((ws->error & kErrWait) ? SOAR_STATUS_INTERNAL : 0) |
+                    ((ws->error & kErrWeight) ? SOAR_STATUS_BAD_WEIGHT : 0);
       res->iters_run = iters;
       res->alpha = alpha;
       res->amax = bits_to_mag(amax_bits);
@@ -1084,11 +1106,13 @@ __global__ void __launch_bounds__(256) swizzle_kernel(const uint8_t* lin, uint8_
 // Eq. 3-4 on stored outputs: sum (w - q s)^2 and sum w^2, one binary64 fma per term, with the
 // bf16 values widened by bit placement (scaled by 2^-128, undone at the end) and the signed
 // E2M1 values read from a 16-entry table in shared memory.  A wait that gave up turns the
-// results into NaN.
+// results into NaN.  kWeighted multiplies every term by its column's weight h_j.
+template <bool kWeighted>
 __global__ void __launch_bounds__(kThreads) dequant_error_kernel(const __grid_constant__ Batch bt,
                                                                  const uint8_t* scales, int swizzled,
                                                                  unsigned int col_tiles, const float* alpha_ptr,
-                                                                 double* out_sse, double* out_sumsq) {
+                                                                 const float* h, double* out_sse,
+                                                                 double* out_sumsq) {
   __shared__ Ring ring;
   __shared__ Slots<2> slots;
   __shared__ double s_q[16];
@@ -1122,6 +1146,8 @@ __global__ void __launch_bounds__(kThreads) dequant_error_kernel(const __grid_co
     }
     const double s = alpha_scaled * static_cast<double>(e4m3_value(dc & 0x7F));
     const unsigned int u[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+    double hd[16];
+    if (kWeighted) load_weights(h, b % p.nbc, hd);
     double e0 = 0.0, e1 = 0.0, q0 = 0.0, q1 = 0.0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -1135,10 +1161,17 @@ __global__ void __launch_bounds__(kThreads) dequant_error_kernel(const __grid_co
       const unsigned int word = (i < 4) ? cw.x : cw.y;
       const double ql = s_q[(word >> (8 * (i & 3))) & 0xFu], qh = s_q[(word >> (8 * (i & 3) + 4)) & 0xFu];
       const double dl = fma(-ql, s, wl), dh = fma(-qh, s, wh);
-      e0 = fma(dl, dl, e0);
-      e1 = fma(dh, dh, e1);
-      q0 = fma(wl, wl, q0);
-      q1 = fma(wh, wh, q1);
+      if (kWeighted) {
+        e0 = fma(hd[2 * i], dl * dl, e0);
+        e1 = fma(hd[2 * i + 1], dh * dh, e1);
+        q0 = fma(hd[2 * i], wl * wl, q0);
+        q1 = fma(hd[2 * i + 1], wh * wh, q1);
+      } else {
+        e0 = fma(dl, dl, e0);
+        e1 = fma(dh, dh, e1);
+        q0 = fma(wl, wl, q0);
+        q1 = fma(wh, wh, q1);
+      }
     }
     acc[0] += e0 + e1;
     acc[1] += q0 + q1;
@@ -1147,6 +1180,267 @@ __global__ void __launch_bounds__(kThreads) dequant_error_kernel(const __grid_co
   acc[0] = failed ? __longlong_as_double(0x7FF8000000000000ll) : acc[0] * 0x1p256;
   acc[1] = failed ? __longlong_as_double(0x7FF8000000000000ll) : acc[1] * 0x1p256;
   double* const dst[2] = {out_sse, out_sumsq};
+  slots_add(slots, 0, acc, dst);
+}
+
+// ------------------------------------------------------------------ column-weighted objective
+//
+// Sec. 5 proposes to minimise the output distortion ||(W - What) X||^2 in CJSO and DSS; its
+// diagonal form is sum_ij h_j (W_ij - What_ij)^2 with h_j the second moment of input channel j.
+// Algorithm 1 is unchanged except that the block sums carry the weights,
+//   A = sum h_j |w_j| m_j,   B = sum h_j m_j^2,
+// in Eq. 5, Eq. 6 and the error of Eq. 8.  The weights are arbitrary binary32 numbers, so the
+// integer dot products of the unweighted kernels do not apply: the sums are binary64, taken in
+// element order (each product is exact: 24 + 8 + 2 and 24 + 4 significant bits), and the state
+// kept between iterations is {A, B} in binary64 plus the scale code.  One tensor per launch.
+
+struct Weighted {
+  const float* h;    // cols weights
+  double2* sums;     // per block {A, B} of the current codes; null when T == 0
+  uint8_t* code;     // per block stored scale code (0: all-zero block); null when T == 0
+};
+
+// A and B of a code vector (sign bits ignored) for hw[j] = h_j |w_j| and hd[j] = h_j.
+__device__ __forceinline__ void weighted_sums(const double (&hw)[16], const double (&hd)[16], unsigned int c0,
+                                              unsigned int c1, double& A, double& B) {
+  const unsigned int m0 = c0 & 0x77777777u, m1 = c1 & 0x77777777u;
+  const unsigned int t[4] = {twice_magnitude_x4(m0), twice_magnitude_x4(m0 >> 16), twice_magnitude_x4(m1),
+                             twice_magnitude_x4(m1 >> 16)};
+  double a = 0.0, b = 0.0;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const double dm = uint_to_double((t[j >> 2] >> (8 * (j & 3))) & 0xFFu);   // 2 m_j
+    a = fma(hw[j], dm, a);
+    b = fma(hd[j], dm * dm, b);
+  }
+  // halving every term halves every partial sum exactly
+  A = 0.5 * a;
+  B = 0.25 * b;
+}
+
+__device__ __forceinline__ bool weight_ok(float h) {
+  return h == 0.0f || (h >= 0x1p-20f && h <= 0x1p20f);
+}
+
+// Eq. 1's tensor maximum, sum h_j W^2 for the error report, and the check of the weights.
+__global__ void __launch_bounds__(kThreads, 2) weighted_amax_kernel(const __grid_constant__ Batch bt, const float* h) {
+  __shared__ Ring ring;
+  __shared__ Slots<1> slots;
+  slots_clear(slots);
+  ring_init(ring);
+  if (is_producer_warp()) {
+    if (threadIdx.x == kTile) ring_produce(ring, bt, 0, 1u);
+    return;
+  }
+  const Params& p = bt.t[0];
+  unsigned int mx = 0;
+  bool bad = false;
+  double sq[1] = {0.0};
+  for (unsigned int n = 0;; ++n) {
+    uint4 v0, v1;
+    int ti;
+    unsigned int tile;
+    if (ring_consume(ring, bt, n, v0, v1, ti, tile) != 0) break;
+    const unsigned int b = tile * kTile + threadIdx.x;
+    if (b >= p.nblk) continue;
+    const unsigned int u[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+    double hd[16];
+    load_weights(h, b % p.nbc, hd);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      // magnitude bit patterns order like the magnitudes; NaN patterns lie above infinity's
+      mx = max(mx, max(u[i] & 0x7FFFu, (u[i] >> 16) & 0x7FFFu));
+      const double wl = static_cast<double>(__uint_as_float(u[i] << 16));
+      const double wh = static_cast<double>(__uint_as_float(u[i] & 0xFFFF0000u));
+      sq[0] = fma(hd[2 * i], wl * wl, sq[0]);
+      sq[0] = fma(hd[2 * i + 1], wh * wh, sq[0]);
+      bad = bad || !weight_ok(static_cast<float>(hd[2 * i])) || !weight_ok(static_cast<float>(hd[2 * i + 1]));
+    }
+  }
+  mx = __reduce_max_sync(0xFFFFFFFFu, mx);
+  const bool any_bad = __any_sync(0xFFFFFFFFu, bad);
+  if ((threadIdx.x & 31) == 0) {
+    if (mx) atomicMax(&p.ws->amax_bits, mx);
+    if (any_bad) atomicOr(&p.ws->error, kErrWeight);
+  }
+  double* const dst[1] = {&p.ws->sumsq};
+  slots_add(slots, 0, sq, dst);
+}
+
+// Algorithm 1 "Initialization" (Eq. 1; the weights play no part in it), the first codes, and
+// the weighted stage-0 sums of Eq. 5 and of the starting error.
+__global__ void __launch_bounds__(kThreads, 2)
+weighted_init_kernel(const __grid_constant__ Batch bt, const Weighted wq, int reverse, int final) {
+  __shared__ Ring ring;
+  __shared__ Slots<3> slots;
+  slots_clear(slots);
+  ring_init(ring);
+  const Params& p = bt.t[0];
+  if (is_producer_warp()) {
+    if (threadIdx.x == kTile) {
+      const bool run = !(status_from_amax(p.ws->amax_bits) & (SOAR_STATUS_NONFINITE | SOAR_STATUS_RANGE)) &&
+                       p.ws->error == 0;
+      ring_produce(ring, bt, reverse, run ? 1u : 0u);
+    }
+    return;
+  }
+  const unsigned int amax_bits = p.ws->amax_bits;
+  const float alpha = amax_bits == 0 ? 1.0f : __fdiv_rn(bits_to_mag(amax_bits), 2688.0f);
+  const float six_alpha = __fmul_rn(alpha, 6.0f);
+  const double alpha_d = static_cast<double>(alpha);
+  double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum
+  unsigned int zeros = 0, unused_wide = 0;
+  for (unsigned int n = 0;; ++n) {
+    uint4 v0, v1;
+    int ti;
+    unsigned int tile;
+    if (ring_consume(ring, bt, n, v0, v1, ti, tile) != 0) break;
+    const unsigned int b = tile * kTile + threadIdx.x;
+    if (b >= p.nblk) continue;
+    Block blk;
+    unpack_block(v0, v1, blk);
+    uint2 codes;
+    if (blk.bmax == 0.0f) {
+      round_block(blk, 1.0f, codes.x, codes.y);
+      reinterpret_cast<uint2*>(p.packed)[b] = codes;
+      p.scales[b] = 0;
+      if (wq.code != nullptr) wq.code[b] = 0;
+      ++zeros;
+      continue;
+    }
+    int c = e4m3_encode(__fdiv_rn(blk.bmax, six_alpha));
+    c = max(c, 1);
+    const float v = e4m3_value(c);
+    round_block(blk, recip_scale(alpha, v), codes.x, codes.y);
+    double hd[16], hw[16];
+    load_weights(wq.h, b % p.nbc, hd);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) hw[j] = hd[j] * static_cast<double>(fabsf(blk.w[j]));
+    double A, B;
+    weighted_sums(hw, hd, codes.x, codes.y, A, B);
+    if (final) {
+      reinterpret_cast<uint2*>(p.packed)[b] = codes;
+      p.scales[b] = static_cast<uint8_t>(c);
+    }
+    if (wq.sums != nullptr) {
+      wq.sums[b] = make_double2(A, B);
+      wq.code[b] = static_cast<uint8_t>(c);
+    }
+    const double vd = static_cast<double>(v);
+    const double sd = alpha_d * vd;
+    acc[0] = fma(A, vd, acc[0]);
+    acc[1] = fma(B * vd, vd, acc[1]);
+    acc[2] += sd * fma(sd, B, -2.0 * A);
+  }
+  double* const dst[3] = {&p.ws->num[0], &p.ws->den[0], &p.ws->gsum[0]};
+  slots_add(slots, 0, acc, dst);
+  add_counters(p.ws, zeros, unused_wide);
+}
+
+// One iteration t of Algorithm 1 under the weighted objective: Eq. 5 from the stage-t sums,
+// Eq. 6 per block from its stored {A, B}, App. B.3's candidates, Eq. 8 with the weighted
+// error written as  sum h w^2 + sd^2 B - 2 sd A  (sd = alpha * candidate scale value), first
+// minimum in (beta, code) order.  All of cfg's shapes and arms run through this one loop.
+__global__ void __launch_bounds__(kThreads, 2)
+weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int t, int reverse, int emit,
+                        int keep) {
+  __shared__ Ring ring;
+  __shared__ Slots<3> slots;
+  __shared__ float s_beta[SOAR_MAX_BETA];
+  __shared__ float s_alpha;
+  __shared__ int s_run;
+  const Params& p = bt.t[0];
+  if (threadIdx.x == 0) {
+    float a;
+    int run;
+    iteration_head(p, t, a, run);
+    s_alpha = a;
+    s_run = run;
+  }
+  const int n_dq = p.n_dq, n_beta = p.n_beta;
+  for (int k = threadIdx.x; k < n_beta; k += kThreads)
+    s_beta[k] = static_cast<float>((100.0 + static_cast<double>((k - n_beta / 2) * p.beta_step_pct)) / 100.0);
+  slots_clear(slots);
+  __syncthreads();
+  if (s_run == 0) return;   // stopped earlier (Sec. 4.1), or the input was rejected
+  ring_init(ring);
+  if (is_producer_warp()) {
+    if (threadIdx.x == kTile) ring_produce(ring, bt, reverse, 1u);
+    return;
+  }
+  const float alpha = s_alpha;
+  const double alpha_d = static_cast<double>(alpha);
+  const bool coupled = (p.flags & SOAR_FLAG_COUPLED_SCALE) != 0;
+  const bool keep_scale = (p.flags & SOAR_FLAG_KEEP_BLOCK_SCALE) != 0;
+  double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum of stage t+1
+  for (unsigned int n = 0;; ++n) {
+    uint4 v0, v1;
+    int ti;
+    unsigned int tile;
+    if (ring_consume(ring, bt, n, v0, v1, ti, tile) != 0) break;
+    const unsigned int b = tile * kTile + threadIdx.x;
+    if (b >= p.nblk) continue;
+    const int d_cur = wq.code[b];
+    if (d_cur == 0) continue;   // all-zero block
+    const double2 ab = wq.sums[b];
+    Block blk;
+    unpack_block(v0, v1, blk);
+    Block mags;                 // the block's magnitudes: the candidate loop only ranks
+    double hd[16], hw[16];
+    load_weights(wq.h, b % p.nbc, hd);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      mags.w[j] = fabsf(blk.w[j]);
+      hw[j] = hd[j] * static_cast<double>(mags.w[j]);
+    }
+    // Eq. 6 (binary32 steps); a block whose weighted codes are all zero keeps its stored scale
+    const float center = (ab.y > 0.0 && !keep_scale)
+                             ? __fdiv_rn(static_cast<float>(ab.x), __fmul_rn(alpha, static_cast<float>(ab.y)))
+                             : e4m3_value(d_cur);
+    int d_lo, d_hi;
+    candidate_window(center, n_dq, d_lo, d_hi);
+    const int nd = d_hi - d_lo + 1;
+    double best = __longlong_as_double(0x7FF0000000000000ll);
+    int best_key = 0;
+    for (int k = 0; k < n_beta; ++k) {
+      unsigned int c0, c1;
+      double A = 0.0, B = 0.0;
+      if (!coupled) {
+        round_block(mags, recip_scale(alpha, __fmul_rn(center, s_beta[k])), c0, c1);
+        weighted_sums(hw, hd, c0, c1, A, B);
+      }
+      for (int d = 0; d < nd; ++d) {
+        const float dv = e4m3_value(clip_code(d_lo + d));
+        if (coupled) {
+          round_block(mags, recip_scale(alpha, __fmul_rn(dv, s_beta[k])), c0, c1);
+          weighted_sums(hw, hd, c0, c1, A, B);
+        }
+        const double sd = alpha_d * static_cast<double>(dv);
+        const double g = sd * fma(sd, B, -2.0 * A);
+        if (g < best) { best = g; best_key = nd * k + d; }
+      }
+    }
+    // the winner, made again from its index, now with the signs
+    const int bk = best_key / nd;
+    const int best_d = clip_code(d_lo + (best_key - bk * nd));
+    unsigned int best0, best1;
+    double bestA, bestB;
+    round_block(blk, recip_scale(alpha, __fmul_rn(coupled ? e4m3_value(best_d) : center, s_beta[bk])), best0, best1);
+    weighted_sums(hw, hd, best0, best1, bestA, bestB);
+    if (emit) {
+      reinterpret_cast<uint2*>(p.packed)[b] = make_uint2(best0, best1);
+      p.scales[b] = static_cast<uint8_t>(best_d);
+    }
+    if (keep) {
+      wq.sums[b] = make_double2(bestA, bestB);
+      wq.code[b] = static_cast<uint8_t>(best_d);
+    }
+    const double vd = static_cast<double>(e4m3_value(best_d));
+    acc[0] = fma(bestA, vd, acc[0]);
+    acc[1] = fma(bestB * vd, vd, acc[1]);
+    acc[2] += best;
+  }
+  double* const dst[3] = {&p.ws->num[t + 1], &p.ws->den[t + 1], &p.ws->gsum[t + 1]};
   slots_add(slots, 0, acc, dst);
 }
 
@@ -1167,9 +1461,13 @@ __global__ void selftest_reciprocal_kernel(unsigned int lo_exp, unsigned int hi_
 
 // Optional launch tracing for benchmarks: while enabled, every kernel this library launches
 // is bracketed by two CUDA events on the launching stream.
-enum KernelId { K_AMAX = 0, K_INIT, K_ITERATE, K_FINALIZE, K_SWIZZLE, K_DEQUANT_ERROR, K_COUNT };
-const char* const kKernelNames[K_COUNT] = {"amax_kernel",     "init_kernel",    "iterate_kernel",
-                                           "finalize_kernel", "swizzle_kernel", "dequant_error_kernel"};
+enum KernelId {
+  K_AMAX = 0, K_INIT, K_ITERATE, K_FINALIZE, K_SWIZZLE, K_DEQUANT_ERROR,
+  K_WEIGHTED_AMAX, K_WEIGHTED_INIT, K_WEIGHTED_ITERATE, K_COUNT
+};
+const char* const kKernelNames[K_COUNT] = {"amax_kernel",          "init_kernel",          "iterate_kernel",
+                                           "finalize_kernel",      "swizzle_kernel",       "dequant_error_kernel",
+                                           "weighted_amax_kernel", "weighted_init_kernel", "weighted_iterate_kernel"};
 struct TraceRec {
   int id;
   cudaEvent_t e0, e1;
@@ -1500,9 +1798,10 @@ int soar_quantize_static(const void* W_bf16, int64_t rows, int64_t cols, int64_t
                        out_global_fp32, scratch, SOAR_STATIC_SCRATCH_BYTES, out_result, stream);
 }
 
-int soar_dequant_error(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, const void* fp4_packed,
-                       const void* e4m3_scales, int scale_layout, const float* global_fp32,
-                       double* out_sse, double* out_sumsq, void* stream) {
+namespace {
+int dequant_error_impl(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, const float* h,
+                       const void* fp4_packed, const void* e4m3_scales, int scale_layout,
+                       const float* global_fp32, double* out_sse, double* out_sumsq, void* stream) {
   const int rc = check_shape(W_bf16, rows, cols, ld);
   if (rc != SOAR_OK) return rc;
   if (fp4_packed == nullptr || e4m3_scales == nullptr || global_fp32 == nullptr || out_sse == nullptr ||
@@ -1530,9 +1829,135 @@ int soar_dequant_error(const void* W_bf16, int64_t rows, int64_t cols, int64_t l
     bt.t[0] = p;
     bt.total_tiles = p.ntiles;
     for (int j = 0; j < kMaxBatch; ++j) bt.tile_end[j] = j == 0 ? p.ntiles : 0xFFFFFFFFu;
-    dequant_error_kernel<<<persistent_grid(dequant_error_kernel, p.ntiles, kThreads), kThreads, 0, st>>>(
-        bt, static_cast<const uint8_t*>(e4m3_scales), scale_layout == SOAR_SCALES_SWIZZLED ? 1 : 0,
-        (p.nbc + 3) / 4, global_fp32, out_sse, out_sumsq);
+    const uint8_t* sc = static_cast<const uint8_t*>(e4m3_scales);
+    const int sw = scale_layout == SOAR_SCALES_SWIZZLED ? 1 : 0;
+    if (h == nullptr)
+      dequant_error_kernel<false><<<persistent_grid(dequant_error_kernel<false>, p.ntiles, kThreads), kThreads, 0,
+                                    st>>>(bt, sc, sw, (p.nbc + 3) / 4, global_fp32, nullptr, out_sse, out_sumsq);
+    else
+      dequant_error_kernel<true><<<persistent_grid(dequant_error_kernel<true>, p.ntiles, kThreads), kThreads, 0,
+                                   st>>>(bt, sc, sw, (p.nbc + 3) / 4, global_fp32, h, out_sse, out_sumsq);
+  }
+  return cudaGetLastError() == cudaSuccess ? SOAR_OK : SOAR_ERR_CUDA;
+}
+}  // namespace
+
+int soar_dequant_error(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, const void* fp4_packed,
+                       const void* e4m3_scales, int scale_layout, const float* global_fp32,
+                       double* out_sse, double* out_sumsq, void* stream) {
+  return dequant_error_impl(W_bf16, rows, cols, ld, nullptr, fp4_packed, e4m3_scales, scale_layout, global_fp32,
+                            out_sse, out_sumsq, stream);
+}
+
+int soar_dequant_error_weighted(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld,
+                                const float* col_weight, const void* fp4_packed, const void* e4m3_scales,
+                                int scale_layout, const float* global_fp32, double* out_sse,
+                                double* out_sumsq, void* stream) {
+  if (col_weight == nullptr) return SOAR_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(col_weight) % 16 != 0) return SOAR_ERR_UNSUPPORTED;
+  return dequant_error_impl(W_bf16, rows, cols, ld, col_weight, fp4_packed, e4m3_scales, scale_layout,
+                            global_fp32, out_sse, out_sumsq, stream);
+}
+
+size_t soar_weighted_workspace_bytes(int64_t rows, int64_t cols, const soar_cfg* cfg) {
+  if (check_cfg(cfg) != SOAR_OK || rows <= 0 || cols <= 0 || cols % 16 != 0) return 0;
+  const size_t nblk = static_cast<size_t>(rows) * static_cast<size_t>(cols / 16);
+  size_t n = kWsFixedBytes;
+  if (cfg->max_iters > 0) n += round256(nblk * sizeof(double2)) + round256(nblk);
+  if (!(cfg->scale_layout & SOAR_SCALES_LINEAR)) n += round256(nblk);
+  return n;
+}
+
+int soar_quantize_weighted(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, const float* col_weight,
+                           const soar_cfg* cfg, void* out_fp4_packed, void* out_e4m3_scales,
+                           void* out_e4m3_scales_sw, float* out_global_fp32, void* workspace,
+                           size_t workspace_bytes, soar_result* out_result, void* stream) {
+  int rc = check_cfg(cfg);
+  if (rc != SOAR_OK) return rc;
+  rc = check_shape(W_bf16, rows, cols, ld);
+  if (rc != SOAR_OK) return rc;
+  const bool want_lin = (cfg->scale_layout & SOAR_SCALES_LINEAR) != 0;
+  const bool want_sw = (cfg->scale_layout & SOAR_SCALES_SWIZZLED) != 0;
+  if (col_weight == nullptr || out_fp4_packed == nullptr || out_global_fp32 == nullptr) return SOAR_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(col_weight) % 16 != 0 || reinterpret_cast<uintptr_t>(out_fp4_packed) % 16 != 0)
+    return SOAR_ERR_UNSUPPORTED;
+  if (want_lin && out_e4m3_scales == nullptr) return SOAR_ERR_INVALID_ARG;
+  if (want_sw && out_e4m3_scales_sw == nullptr) return SOAR_ERR_INVALID_ARG;
+  const size_t need = soar_weighted_workspace_bytes(rows, cols, cfg);
+  if (workspace == nullptr || need == 0 || workspace_bytes < need) return SOAR_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return SOAR_ERR_UNSUPPORTED;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* next = static_cast<uint8_t*>(workspace);
+  if (cudaMemsetAsync(next, 0, kWsFixedBytes, st) != cudaSuccess) return SOAR_ERR_CUDA;
+  Batch bt;
+  Reports rp;
+  memset(&bt, 0, sizeof(bt));
+  memset(&rp, 0, sizeof(rp));
+  Params& p = bt.t[0];
+  p.W = static_cast<const uint16_t*>(W_bf16);
+  p.packed = static_cast<uint8_t*>(out_fp4_packed);
+  p.ws = reinterpret_cast<Ws*>(next);
+  next += kWsFixedBytes;
+  p.ld = ld;
+  p.nbc = static_cast<unsigned int>(cols / 16);
+  p.nblk = static_cast<unsigned int>(rows * (cols / 16));
+  p.ntiles = (p.nblk + kTile - 1) / kTile;
+  p.contiguous = (ld == cols) ? 1 : 0;
+  Weighted wq;
+  wq.h = col_weight;
+  wq.sums = nullptr;
+  wq.code = nullptr;
+  if (cfg->max_iters > 0) {
+    wq.sums = reinterpret_cast<double2*>(next);
+    next += round256(static_cast<size_t>(p.nblk) * sizeof(double2));
+    wq.code = next;
+    next += round256(p.nblk);
+  }
+  p.scales = want_lin ? static_cast<uint8_t*>(out_e4m3_scales) : next;
+  p.max_iters = cfg->max_iters;
+  p.early_stop_rel = cfg->early_stop_rel;
+  p.n_dq = cfg->n_dq;
+  p.n_beta = cfg->n_beta;
+  p.beta_step_pct = cfg->beta_step_pct;
+  p.flags = cfg->flags;
+  bt.n = 1;
+  bt.total_tiles = p.ntiles;
+  for (int j = 0; j < kMaxBatch; ++j) bt.tile_end[j] = j == 0 ? p.ntiles : 0xFFFFFFFFu;
+  rp.alpha[0] = out_global_fp32;
+  rp.result[0] = out_result;
+
+  const unsigned int tiles = p.ntiles;
+  int reverse = 1;   // the first pass runs forward; each later one starts where the last ended
+  {
+    ScopedLaunch sl(K_WEIGHTED_AMAX, st);
+    weighted_amax_kernel<<<persistent_grid(weighted_amax_kernel, tiles, kThreads), kThreads, 0, st>>>(bt, col_weight);
+  }
+  {
+    ScopedLaunch sl(K_WEIGHTED_INIT, st);
+    weighted_init_kernel<<<persistent_grid(weighted_init_kernel, tiles, kThreads), kThreads, 0, st>>>(
+        bt, wq, reverse, cfg->max_iters == 0 ? 1 : 0);
+  }
+  const bool may_stop = cfg->early_stop_rel > 0.0f;
+  const unsigned int g_it = persistent_grid(weighted_iterate_kernel, tiles, kThreads);
+  for (int t = 0; t < cfg->max_iters; ++t) {
+    reverse ^= 1;
+    const int last = (t == cfg->max_iters - 1) ? 1 : 0;
+    ScopedLaunch sl(K_WEIGHTED_ITERATE, st);
+    weighted_iterate_kernel<<<g_it, kThreads, 0, st>>>(bt, wq, t, reverse, (may_stop || last) ? 1 : 0, !last);
+  }
+  {
+    ScopedLaunch sl(K_FINALIZE, st);
+    finalize_kernel<<<1, 128, 0, st>>>(bt, rp);
+  }
+  if (want_sw) {
+    const unsigned int rt = static_cast<unsigned int>((rows + 127) / 128);
+    const unsigned int ct = (p.nbc + 3) / 4;
+    const size_t blocks = (static_cast<size_t>(rt) * ct * 512 + 255) / 256;
+    const unsigned int grid = static_cast<unsigned int>(blocks < 65535u * 16u ? blocks : 65535u * 16u);
+    ScopedLaunch sl(K_SWIZZLE, st);
+    swizzle_kernel<<<grid, 256, 0, st>>>(p.scales, static_cast<uint8_t*>(out_e4m3_scales_sw),
+                                         static_cast<unsigned int>(rows), p.nbc, rt, ct);
   }
   return cudaGetLastError() == cudaSuccess ? SOAR_OK : SOAR_ERR_CUDA;
 }
