@@ -214,11 +214,12 @@ def run_reference(args):
     rows = min(spec.rows, max(1, args.ref_rows))
     rows = max(1, rows // WL._chunk_rows(spec.cols)) * WL._chunk_rows(spec.cols)
     w = wl.generate(0, 0, rows)
+    h = WL.column_weights(spec.cols, 1000) if args.objective == "weighted" else None
     for _ in range(args.warmup):
-        R.quantize(w[: max(1, rows // 8)], rcfg)
+        R.quantize(w[: max(1, rows // 8)], rcfg, h=h)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        R.quantize(w, rcfg)
+        R.quantize(w, rcfg, h=h)
     dt = (time.perf_counter() - t0) / args.steps
     value = 2.0 * w.size / dt / 1e9
     sample = f"{rows} rows x {spec.cols} cols of tensor '{spec.name}' of {wl.name} per step"
@@ -227,7 +228,8 @@ def run_reference(args):
         n_gpus=args.gpus, steps=args.steps, warmup=args.warmup, ms_per_step=dt * 1e3,
         higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32", data="synthetic",
         config=dict(workload=wl.name, preset=args.preset, max_iters=cfg.max_iters, n_beta=cfg.n_beta,
-                    n_dq=cfg.n_dq, early_stop_rel=cfg.early_stop_rel, sample=sample),
+                    n_dq=cfg.n_dq, early_stop_rel=cfg.early_stop_rel, sample=sample,
+                    **({"objective": "column-weighted"} if h is not None else {})),
         cpu_baseline=dict(value=value, unit="GB/s", cores=R.num_threads(), kind="oracle", sample=sample),
         e2e=dict(value=value, unit="GB/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0),
         elements_per_s=w.size / dt, gpu_launches=0,
@@ -484,6 +486,188 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# Column-weighted objective: per candidate and element the scale multiply, the rounding and two binary64
+# accumulations (A and B carry arbitrary weights, so they cannot be integer dot products); a binary64
+# fused multiply-add issues at half the FP32 rate and counts as two lane-operations.
+WEIGHTED_OPS_PER_ELEMENT_EVAL = 6
+WEIGHTED_STATE_BYTES = 17.0 / 16    # {A, B} in binary64 and the scale code per 16-element block
+
+
+def weighted_kernel_bytes_per_elem(name: str, cfg, t: int = 0) -> float:
+    if name == "weighted_amax_kernel":
+        return 2.0
+    if name == "weighted_init_kernel":
+        return 2.0 + (WEIGHTED_STATE_BYTES if cfg.max_iters > 0 else OUT_BYTES)
+    if name == "weighted_iterate_kernel":
+        last = t == cfg.max_iters - 1
+        emits = last or cfg.early_stop_rel > 0
+        return 2.0 + WEIGHTED_STATE_BYTES + (0.0 if last else WEIGHTED_STATE_BYTES) + (OUT_BYTES if emits else 0.0)
+    return 0.0
+
+
+def run_weighted(args):
+    """The same step under the column-weighted objective: one soar_quantize_weighted call per tensor,
+    W and the column weights resident in HBM."""
+    import torch
+
+    from paper_2605_12245_b200 import api
+    from paper_2605_12245_b200 import sharding as SH
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    api.lib()
+    peaks = load_peaks()
+    wl = pick_workload(args.workload, rank)
+    cfg = preset_cfg(api, args.preset, args)
+    host_w, host_h, dev_w, dev_h, outs = [], [], [], [], []
+    for i, spec in enumerate(wl.tensors):
+        bits = wl.generate(i)
+        hw = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+        hh = torch.from_numpy(WL.column_weights(spec.cols, 1000 * (rank + 1) + i))
+        host_w.append(hw)
+        host_h.append(hh)
+        dev_w.append(hw.cuda())
+        dev_h.append(hh.cuda())
+        outs.append(api.alloc_buffers(spec.rows, spec.cols, cfg, weighted=True))
+    elements = wl.elements
+    stream = torch.cuda.current_stream()
+
+    def step():
+        for W, h, o in zip(dev_w, dev_h, outs):
+            api.soar_quantize_weighted(W, h, cfg, o, stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup, trace):
+        for _ in range(warmup):
+            fn()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if trace:
+            api.soar_trace_begin()
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        tr = api.soar_trace_end() if trace else {}
+        barrier()
+        return SH.max_over_ranks(e0.elapsed_time(e1) / steps, "cuda"), tr
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms, _ = timed(step, args.steps, args.warmup, False)
+    traced_ms, trace = timed(step, args.steps, 0, True)
+    clocks = sampler.stop()
+    results = [o.read_result() for o in outs]
+    iters = [r.iters_run for r in results]
+    value = world * 2.0 * elements / (ms * 1e-3) / 1e9
+    launches = sum(v[0] for v in trace.values())
+    dom = max(trace, key=lambda k: trace[k][1])
+    n_launch, tot_ms = trace[dom]
+    ops_per_block = cfg.n_beta * (16 * WEIGHTED_OPS_PER_ELEMENT_EVAL + cfg.n_dq * OPS_PER_PAIR_SCORE)
+    it_bytes = sum(s.rows * s.cols * weighted_kernel_bytes_per_elem("weighted_iterate_kernel", cfg, t)
+                   for s, it in zip(wl.tensors, iters) for t in range(it)) * args.steps
+    if dom == "weighted_iterate_kernel":
+        blocks_iters = sum((s.rows * s.cols // 16) * it for s, it in zip(wl.tensors, iters)) * args.steps
+        achieved = blocks_iters * ops_per_block / (tot_ms * 1e-3) / 1e12
+        peak = SM_COUNT * FP32_LANES_PER_SM * peaks["sm_max_mhz"] * 1e6 / 1e12
+        roofline = dict(bound="alu", kernel=dom, achieved=achieved, peak=peak, unit="Tlane-op/s", frac=achieved / peak,
+                        traffic=None, launches=n_launch, active_launches=sum(iters) * args.steps,
+                        kernel_ms_per_step=tot_ms / args.steps,
+                        peak_source="148 SMs x 128 FP32 lanes x clocks.max.sm",
+                        hbm_gbs_for_context=it_bytes / (tot_ms * 1e-3) / 1e9)
+    else:
+        byts = elements * args.steps * weighted_kernel_bytes_per_elem(dom, cfg)
+        achieved = byts / (tot_ms * 1e-3) / 1e9
+        roofline = dict(bound="hbm", kernel=dom, achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
+                        frac=achieved / peaks["hbm_gbs"], traffic=None, launches=n_launch,
+                        kernel_ms_per_step=tot_ms / args.steps, peak_source=peaks["source"])
+    kernels = {k: dict(launches=v[0], ms_per_step=v[1] / args.steps, share=v[1] / sum(x[1] for x in trace.values()))
+               for k, v in trace.items()}
+
+    # what the weights buy: weighted error of this run against the weighted error of the unweighted method's output
+    gain = None
+    if rank == 0:
+        plain = api.soar_quantize(dev_w[0], cfg)
+        e = api.soar_dequant_error_weighted(dev_w[0], dev_h[0], plain.packed, plain.scales, plain.alpha).cpu().numpy()
+        gain = dict(tensor=wl.tensors[0].name, weighted_rel_error=results[0].sse / results[0].sumsq,
+                    weighted_rel_error_of_unweighted_run=float(e[0] / e[1]),
+                    weighted_rel_error_of_max_based_start=results[0].sse_init / results[0].sumsq)
+        del plain
+
+    # ---- end to end: pinned host buffers in and out, copies inside the timed region (one stream)
+    e2e = None
+    if not args.no_e2e and args.workload != "config3":
+        pin = lambda t: torch.empty_like(t, device="cpu").pin_memory()  # noqa: E731
+        hin = [pin(h) for h in host_w]
+        for a, b in zip(hin, host_w):
+            a.copy_(b)
+        hout = [(pin(o.packed), pin(o.scales), pin(o.alpha), pin(o.result)) for o in outs]
+
+        def e2e_step():
+            for W, hsrc, h, o, ho in zip(dev_w, hin, dev_h, outs, hout):
+                W.copy_(hsrc, non_blocking=True)
+                api.soar_quantize_weighted(W, h, cfg, o, stream)
+                for dst, src in zip(ho, (o.packed, o.scales, o.alpha, o.result)):
+                    dst.copy_(src, non_blocking=True)
+
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            e2e_step()
+        torch.cuda.synchronize()
+        dt = SH.max_over_ranks((time.perf_counter() - t0) / args.steps, "cuda")
+        import ctypes
+        e2e = dict(value=world * 2.0 * elements / dt / 1e9, unit="GB/s", ms_per_step=dt * 1e3,
+                   h2d_bytes_per_step=2 * elements,
+                   d2h_bytes_per_step=elements // 2 + elements // 16 + len(wl.tensors) * (4 + ctypes.sizeof(api.SoarResult)),
+                   api="pinned host buffers; copy-in, soar_quantize_weighted and copy-out in order on one stream "
+                       "(the column weights stay on the device)")
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        from oracle import soar_ref as R
+        spec = wl.tensors[0]
+        rows = max(1, min(spec.rows, args.cpu_rows) // WL._chunk_rows(spec.cols)) * WL._chunk_rows(spec.cols)
+        w = host_w[0][:rows].view(torch.int16).numpy().view(np.uint16)
+        t0 = time.perf_counter()
+        ref = R.quantize(w, ref_cfg_of(R, cfg), h=host_h[0].numpy())
+        dt = time.perf_counter() - t0
+        cpu = dict(value=2.0 * w.size / dt / 1e9, unit="GB/s", cores=R.num_threads(), kind="oracle",
+                   sample=f"first {rows} rows x {spec.cols} cols of tensor '{spec.name}', {ref.iters_run} iterations, {dt:.1f} s",
+                   elements_per_s=w.size / dt)
+
+    if rank == 0:
+        line = dict(
+            metric="soar_quantize_bf16_input_throughput", value=value, unit="GB/s", n_gpus=world,
+            steps=args.steps, warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak",
+            vs_baseline=None, dtype="f64", data="synthetic",
+            config=dict(workload=wl.name, objective="column-weighted", preset=args.preset, max_iters=cfg.max_iters,
+                        n_beta=cfg.n_beta, n_dq=cfg.n_dq, early_stop_rel=cfg.early_stop_rel, tensors=len(wl.tensors),
+                        elements=elements, iters_run=iters,
+                        l2="inputs (%.2f GB per step) exceed the 126 MB L2" % (2 * elements / 1e9),
+                        parallelism=f"{world} rank(s), one layer of these shapes each, no collective"),
+            elements_per_s=world * elements / (ms * 1e-3), traced_ms_per_step=traced_ms, roofline=roofline,
+            kernels=kernels, cpu_baseline=cpu, e2e=e2e, gpu_launches=launches, clocks=clocks, weighting_gain=gain)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -497,6 +681,8 @@ def main():
     ap.add_argument("--pairs", type=int, default=0, help="candidate pairs per block (overrides the preset's grid)")
     ap.add_argument("--iters", type=int, default=None, help="iterations T, early stop off (overrides the preset)")
     ap.add_argument("--sweep", default="", help="comma-separated candidate-pair counts to time, one iteration each")
+    ap.add_argument("--objective", default="plain", choices=["plain", "weighted"],
+                    help="weighted: the column-weighted objective through soar_quantize_weighted")
     ap.add_argument("--no-batch", action="store_true", help="one soar_quantize call per tensor instead of soar_quantize_batch")
     ap.add_argument("--graph", action="store_true", help="replay each step from a CUDA graph (no per-kernel trace)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -506,6 +692,8 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.objective == "weighted":
+        run_weighted(args)
     else:
         run_ours(args)
 

@@ -1218,6 +1218,24 @@ __device__ __forceinline__ void weighted_sums(const double (&hw)[16], const doub
   B = 0.25 * b;
 }
 
+// The same sums for ranking candidates: two interleaved partial chains per sum instead of one
+// sixteen-long chain of dependent additions.  The result may differ from weighted_sums in the
+// last bit, which only a tie between candidates could feel.
+__device__ __forceinline__ void weighted_sums_split(const double (&hw)[16], const double (&hd)[16], unsigned int c0,
+                                                    unsigned int c1, double& A, double& B) {
+  const unsigned int t[4] = {twice_magnitude_x4(c0), twice_magnitude_x4(c0 >> 16), twice_magnitude_x4(c1),
+                             twice_magnitude_x4(c1 >> 16)};
+  double a[2] = {0.0, 0.0}, b[2] = {0.0, 0.0};
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const double dm = uint_to_double((t[j >> 2] >> (8 * (j & 3))) & 0xFFu);
+    a[j & 1] = fma(hw[j], dm, a[j & 1]);
+    b[j & 1] = fma(hd[j], dm * dm, b[j & 1]);
+  }
+  A = 0.5 * (a[0] + a[1]);
+  B = 0.25 * (b[0] + b[1]);
+}
+
 __device__ __forceinline__ bool weight_ok(float h) {
   return h == 0.0f || (h >= 0x1p-20f && h <= 0x1p20f);
 }
@@ -1402,18 +1420,22 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
     const int nd = d_hi - d_lo + 1;
     double best = __longlong_as_double(0x7FF0000000000000ll);
     int best_key = 0;
+    // the products alpha * center * beta are monotone in beta: the end points bound them all
+    const bool fast_rcp = !coupled && recip_fast_ok(__fmul_rn(alpha, __fmul_rn(center, s_beta[0]))) &&
+                          recip_fast_ok(__fmul_rn(alpha, __fmul_rn(center, s_beta[n_beta - 1])));
     for (int k = 0; k < n_beta; ++k) {
       unsigned int c0, c1;
       double A = 0.0, B = 0.0;
       if (!coupled) {
-        round_block(mags, recip_scale(alpha, __fmul_rn(center, s_beta[k])), c0, c1);
-        weighted_sums(hw, hd, c0, c1, A, B);
+        const float s = __fmul_rn(alpha, __fmul_rn(center, s_beta[k]));
+        round_block(mags, fast_rcp ? recip_fast(s) : __frcp_rn(s), c0, c1);
+        weighted_sums_split(hw, hd, c0, c1, A, B);
       }
       for (int d = 0; d < nd; ++d) {
         const float dv = e4m3_value(clip_code(d_lo + d));
         if (coupled) {
           round_block(mags, recip_scale(alpha, __fmul_rn(dv, s_beta[k])), c0, c1);
-          weighted_sums(hw, hd, c0, c1, A, B);
+          weighted_sums_split(hw, hd, c0, c1, A, B);
         }
         const double sd = alpha_d * static_cast<double>(dv);
         const double g = sd * fma(sd, B, -2.0 * A);
@@ -1436,9 +1458,10 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
       wq.code[b] = static_cast<uint8_t>(best_d);
     }
     const double vd = static_cast<double>(e4m3_value(best_d));
+    const double sd = alpha_d * vd;
     acc[0] = fma(bestA, vd, acc[0]);
     acc[1] = fma(bestB * vd, vd, acc[1]);
-    acc[2] += best;
+    acc[2] += sd * fma(sd, bestB, -2.0 * bestA);
   }
   double* const dst[3] = {&p.ws->num[t + 1], &p.ws->den[t + 1], &p.ws->gsum[t + 1]};
   slots_add(slots, 0, acc, dst);

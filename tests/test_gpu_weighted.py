@@ -140,3 +140,20 @@ def test_argument_errors_of_the_weighted_entry():
     # the plain workspace is smaller than the weighted one: it must be refused
     small = api.alloc_buffers(16, 64, cfg)
     assert L.soar_quantize_weighted(*args(ws=small.workspace.data_ptr(), wsb=small.workspace.numel())) == -3
+
+
+@pytest.mark.parametrize("tensor", [1, 0])          # k (1024 x 8192), q (8192 x 8192) of the Llama-3-70B layer
+def test_full_size_tensors_under_the_weighted_objective(tensor):
+    """Whole tensors of the benchmark's workload in the launch configuration bench.py times
+    (--objective weighted), element by element against the oracle."""
+    wl = WL.config4()
+    w = WL.generate(wl, tensor)
+    h = WL.column_weights(wl.tensors[tensor].cols, 1000 + tensor)
+    cfg, ref_cfg = P.cfg_pair()
+    gpu, W, hw = run_weighted(w, h, cfg)
+    ref = R.quantize(w, ref_cfg, h=h)
+    rep = P.assert_parity(gpu, ref)
+    print(wl.tensors[tensor].name, "weighted:", rep)
+    assert gpu.result.sumsq == pytest.approx(ref.sumsq, rel=1e-9)
+    e = api.soar_dequant_error_weighted(W, hw, gpu.buffers.packed, gpu.buffers.scales, gpu.buffers.alpha).cpu().numpy()
+    assert e[0] == pytest.approx(gpu.result.sse, rel=1e-9)
