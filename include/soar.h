@@ -98,7 +98,9 @@ typedef struct soar_result {
   double sumsq;                             /* sum W^2                                       */
   int64_t zero_blocks;                      /* blocks whose 16 elements are all zero         */
   int64_t wide_candidates;                  /* candidate evaluations that took the binary64
-                                               accumulation path (scale far below block max) */
+                                               accumulation path (scale far below block max);
+                                               soar_quantize_weighted: blocks (summed over the
+                                               iterations) ranked by the exact loop            */
   double trace_alpha[SOAR_MAX_ITERS + 1];   /* alpha^(0), then alpha of each executed iteration */
   double trace_sse[SOAR_MAX_ITERS + 1];     /* error of the start, then after each iteration */
 } soar_result;

@@ -1236,6 +1236,77 @@ __device__ __forceinline__ void weighted_sums_split(const double (&hw)[16], cons
   B = 0.25 * (b[0] + b[1]);
 }
 
+// Fixed-point images of sixteen non-negative binary64 values below 2^(e+1), `bits` (33..48) wide:
+// F_j = rn(v_j * 2^(bits - 1 - e)) <= 2^bits, cut into three 16-bit limbs and packed two elements
+// per word, the operand layout of the 16-bit x 8-bit dot-product instruction.
+struct Limbs {
+  unsigned int hi[8], mid[8], lo[8];
+};
+
+__device__ __forceinline__ int exponent_of(double v) {
+  return ((__double2hiint(v) >> 20) & 0x7FF) - 1023;
+}
+
+__device__ __forceinline__ double two_to(int e) { return __hiloint2double((1023 + e) << 20, 0); }
+
+__device__ __forceinline__ void make_limbs(const double (&v)[16], int e, int bits, Limbs& L) {
+  const double scale = two_to(bits - 1 - e);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const unsigned long long f0 = __double2ull_rn(v[2 * i] * scale), f1 = __double2ull_rn(v[2 * i + 1] * scale);
+    const unsigned int a0 = static_cast<unsigned int>(f0), a1 = static_cast<unsigned int>(f1);
+    L.hi[i] = (static_cast<unsigned int>(f0 >> 32) & 0xFFFFu) | (static_cast<unsigned int>(f1 >> 32) << 16);
+    L.mid[i] = __byte_perm(a0, a1, 0x7632);
+    L.lo[i] = __byte_perm(a0, a1, 0x5410);
+  }
+}
+
+// Widths of the images of h_j |w_j| and of h_j: sum F_j 2m_j <= 192 * 2^45 and
+// sum G_j (2m_j)^2 <= 2304 * 2^41 both stay below 2^53.
+constexpr int kImageBitsA = 45, kImageBitsB = 41;
+
+// Four magnitude codes to four bytes holding (2m)^2: 0,1,4,9,16,36,64,144.
+__device__ __forceinline__ unsigned int twice_magnitude_squared_x4(unsigned int codes) {
+  unsigned int out;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(0x09040100u), "r"(0x90402410u), "r"(codes));
+  return out;
+}
+
+// Integer images of the weighted sums of a magnitude code vector:
+// At = sum F_j (2 m_j) and Bt = sum G_j (2 m_j)^2, exact, as binary64.
+__device__ __forceinline__ void limb_sums(const Limbs& F, const Limbs& G, unsigned int c0, unsigned int c1, double& At,
+                                          double& Bt) {
+  const unsigned int c[4] = {c0, c0 >> 16, c1, c1 >> 16};
+  unsigned int ah = 0, am = 0, al = 0, bh = 0, bm = 0, bl = 0;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const unsigned int t = twice_magnitude_x4(c[q]), u = twice_magnitude_squared_x4(c[q]);
+    ah = __dp2a_lo(F.hi[2 * q], t, ah);
+    ah = __dp2a_hi(F.hi[2 * q + 1], t, ah);
+    am = __dp2a_lo(F.mid[2 * q], t, am);
+    am = __dp2a_hi(F.mid[2 * q + 1], t, am);
+    al = __dp2a_lo(F.lo[2 * q], t, al);
+    al = __dp2a_hi(F.lo[2 * q + 1], t, al);
+    bh = __dp2a_lo(G.hi[2 * q], u, bh);
+    bh = __dp2a_hi(G.hi[2 * q + 1], u, bh);
+    bm = __dp2a_lo(G.mid[2 * q], u, bm);
+    bm = __dp2a_hi(G.mid[2 * q + 1], u, bm);
+    bl = __dp2a_lo(G.lo[2 * q], u, bl);
+    bl = __dp2a_hi(G.lo[2 * q + 1], u, bl);
+  }
+  // every limb sum is below 2^28 and, for kImageBitsA/B wide images, the whole below 2^53: exact
+  At = fma(fma(uint_to_double(ah), 65536.0, uint_to_double(am)), 65536.0, uint_to_double(al));
+  Bt = fma(fma(uint_to_double(bh), 65536.0, uint_to_double(bm)), 65536.0, uint_to_double(bl));
+}
+
+// hd[j] = h_j and hw[j] = h_j |w_j| of a block, binary64 (both exact).
+__device__ __forceinline__ void block_weights(const float* h, unsigned int cb, const Block& mags, double (&hd)[16],
+                                              double (&hw)[16]) {
+  load_weights(h, cb, hd);
+#pragma unroll
+  for (int j = 0; j < 16; ++j) hw[j] = hd[j] * static_cast<double>(mags.w[j]);
+}
+
 __device__ __forceinline__ bool weight_ok(float h) {
   return h == 0.0f || (h >= 0x1p-20f && h <= 0x1p20f);
 }
@@ -1391,6 +1462,7 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
   const bool coupled = (p.flags & SOAR_FLAG_COUPLED_SCALE) != 0;
   const bool keep_scale = (p.flags & SOAR_FLAG_KEEP_BLOCK_SCALE) != 0;
   double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum of stage t+1
+  unsigned int exact_blocks = 0, unused_zeros = 0;
   for (unsigned int n = 0;; ++n) {
     uint4 v0, v1;
     int ti;
@@ -1404,13 +1476,9 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
     Block blk;
     unpack_block(v0, v1, blk);
     Block mags;                 // the block's magnitudes: the candidate loop only ranks
-    double hd[16], hw[16];
-    load_weights(wq.h, b % p.nbc, hd);
+    const unsigned int cb = b % p.nbc;
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      mags.w[j] = fabsf(blk.w[j]);
-      hw[j] = hd[j] * static_cast<double>(mags.w[j]);
-    }
+    for (int j = 0; j < 16; ++j) mags.w[j] = fabsf(blk.w[j]);
     // Eq. 6 (binary32 steps); a block whose weighted codes are all zero keeps its stored scale
     const float center = (ab.y > 0.0 && !keep_scale)
                              ? __fdiv_rn(static_cast<float>(ab.x), __fmul_rn(alpha, static_cast<float>(ab.y)))
@@ -1418,37 +1486,111 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
     int d_lo, d_hi;
     candidate_window(center, n_dq, d_lo, d_hi);
     const int nd = d_hi - d_lo + 1;
-    double best = __longlong_as_double(0x7FF0000000000000ll);
     int best_key = 0;
     // the products alpha * center * beta are monotone in beta: the end points bound them all
     const bool fast_rcp = !coupled && recip_fast_ok(__fmul_rn(alpha, __fmul_rn(center, s_beta[0]))) &&
                           recip_fast_ok(__fmul_rn(alpha, __fmul_rn(center, s_beta[n_beta - 1])));
-    for (int k = 0; k < n_beta; ++k) {
-      unsigned int c0, c1;
-      double A = 0.0, B = 0.0;
-      if (!coupled) {
-        const float s = __fmul_rn(alpha, __fmul_rn(center, s_beta[k]));
-        round_block(mags, fast_rcp ? recip_fast(s) : __frcp_rn(s), c0, c1);
-        weighted_sums_split(hw, hd, c0, c1, A, B);
-      }
-      for (int d = 0; d < nd; ++d) {
-        const float dv = e4m3_value(clip_code(d_lo + d));
-        if (coupled) {
-          round_block(mags, recip_scale(alpha, __fmul_rn(dv, s_beta[k])), c0, c1);
-          weighted_sums_split(hw, hd, c0, c1, A, B);
+
+    // Fast ranking.  The weighted error minus sum h w^2 is  g = sd^2 B - 2 sd A.  With 45- and 41-bit fixed-point
+    // images F_j of h_j |w_j| and G_j of h_j (relative to the block's largest), the integer sums
+    // At = sum F_j 2m_j and Bt = sum G_j (2m_j)^2 are exact and cost one dot-product instruction per
+    // two elements and limb; A = cA At and B = cB Bt up to the rounding of the images, at most 96 cA and
+    // 1152 cB.  The loop keeps, per E4M3 code, the best and the second-best distinct value; when the
+    // overall runner-up is further from the winner than those roundings could account for, the
+    // winner is the exact loop's winner.  Otherwise (rarely) the exact loop below decides.
+    bool decided = false;
+    if (!coupled && nd <= 2 && fast_rcp) {
+      double hmax = 0.0, hwmax = 0.0;
+      Limbs F, G;
+      {
+        double hd[16], hw[16];
+        block_weights(wq.h, cb, mags, hd, hw);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          hmax = fmax(hmax, hd[j]);
+          hwmax = fmax(hwmax, hw[j]);
         }
-        const double sd = alpha_d * static_cast<double>(dv);
-        const double g = sd * fma(sd, B, -2.0 * A);
-        if (g < best) { best = g; best_key = nd * k + d; }
+        if (hwmax > 0.0) {
+          make_limbs(hw, exponent_of(hwmax), kImageBitsA, F);
+          make_limbs(hd, exponent_of(hmax), kImageBitsB, G);
+        }
+      }
+      if (hwmax > 0.0) {
+        const int ea = exponent_of(hwmax), eb = exponent_of(hmax);
+        const double cA = two_to(ea - kImageBitsA), cB = two_to(eb - kImageBitsB - 1);   // A = cA At, B = cB Bt
+        const double sd0 = alpha_d * static_cast<double>(e4m3_value(clip_code(d_lo)));
+        const double sd1 = alpha_d * static_cast<double>(e4m3_value(clip_code(d_lo + 1)));
+        // g = 2 sd cA (rho Bt - At)  with  rho = sd cB / (2 cA)
+        const double ratio = two_to(eb - ea + kImageBitsA - kImageBitsB - 2);   // cB / (2 cA)
+        const double rho0 = sd0 * ratio, rho1 = sd1 * ratio;
+        const double inf = __longlong_as_double(0x7FF0000000000000ll);
+        double h0 = inf, s0 = inf, h1 = inf, s1 = inf;
+        int k0 = 0, k1 = 0;
+        uint2 w0 = make_uint2(0u, 0u), w1 = w0;   // code vectors of the two current winners
+        for (int k = 0; k < n_beta; ++k) {
+          unsigned int c0, c1;
+          round_block(mags, recip_fast(__fmul_rn(alpha, __fmul_rn(center, s_beta[k]))), c0, c1);
+          double At, Bt;
+          limb_sums(F, G, c0, c1, At, Bt);
+          // an equal value from the same codes is the same outcome again (a neighbouring beta); from other
+          // codes it is a tie that the images cannot resolve, and counts as a runner-up
+          const double e0 = fma(rho0, Bt, -At);
+          if (e0 < h0) { s0 = h0; h0 = e0; k0 = k; w0 = make_uint2(c0, c1); }
+          else if (e0 < s0 && (e0 > h0 || c0 != w0.x || c1 != w0.y)) s0 = e0;
+          if (nd == 2) {
+            const double e1 = fma(rho1, Bt, -At);
+            if (e1 < h1) { s1 = h1; h1 = e1; k1 = k; w1 = make_uint2(c0, c1); }
+            else if (e1 < s1 && (e1 > h1 || c0 != w1.x || c1 != w1.y)) s1 = e1;
+          }
+        }
+        const double q0 = 2.0 * sd0 * cA, q1 = 2.0 * sd1 * cA;
+        const double g0 = q0 * h0, g1 = (nd == 2) ? q1 * h1 : inf;
+        const bool second = g1 < g0;
+        const double win = second ? g1 : g0;
+        const double runner = fmin(second ? g0 : g1, second ? q1 * s1 : q0 * s0);
+        const double sdm = fmax(sd0, sd1);
+        const double margin = 2.02 * sdm * fma(sdm, 1152.0 * cB, 192.0 * cA);
+        decided = runner - win > margin;
+        best_key = second ? nd * k1 + 1 : nd * k0;
       }
     }
-    // the winner, made again from its index, now with the signs
+    if (!decided) {
+      // exact loop: binary64 sums for every candidate; also the coupled arm and wider code windows
+      double hd[16], hw[16];
+      block_weights(wq.h, cb, mags, hd, hw);
+      double best = __longlong_as_double(0x7FF0000000000000ll);
+      for (int k = 0; k < n_beta; ++k) {
+        unsigned int c0, c1;
+        double A = 0.0, B = 0.0;
+        if (!coupled) {
+          const float s = __fmul_rn(alpha, __fmul_rn(center, s_beta[k]));
+          round_block(mags, fast_rcp ? recip_fast(s) : __frcp_rn(s), c0, c1);
+          weighted_sums_split(hw, hd, c0, c1, A, B);
+        }
+        for (int d = 0; d < nd; ++d) {
+          const float dv = e4m3_value(clip_code(d_lo + d));
+          if (coupled) {
+            round_block(mags, recip_scale(alpha, __fmul_rn(dv, s_beta[k])), c0, c1);
+            weighted_sums_split(hw, hd, c0, c1, A, B);
+          }
+          const double sd = alpha_d * static_cast<double>(dv);
+          const double g = sd * fma(sd, B, -2.0 * A);
+          if (g < best) { best = g; best_key = nd * k + d; }
+        }
+      }
+      ++exact_blocks;
+    }
+    // the winner, made again from its index, now with the signs and the sums in element order
     const int bk = best_key / nd;
     const int best_d = clip_code(d_lo + (best_key - bk * nd));
     unsigned int best0, best1;
     double bestA, bestB;
     round_block(blk, recip_scale(alpha, __fmul_rn(coupled ? e4m3_value(best_d) : center, s_beta[bk])), best0, best1);
-    weighted_sums(hw, hd, best0, best1, bestA, bestB);
+    {
+      double hd[16], hw[16];
+      block_weights(wq.h, cb, mags, hd, hw);
+      weighted_sums(hw, hd, best0, best1, bestA, bestB);
+    }
     if (emit) {
       reinterpret_cast<uint2*>(p.packed)[b] = make_uint2(best0, best1);
       p.scales[b] = static_cast<uint8_t>(best_d);
@@ -1465,6 +1607,7 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
   }
   double* const dst[3] = {&p.ws->num[t + 1], &p.ws->den[t + 1], &p.ws->gsum[t + 1]};
   slots_add(slots, 0, acc, dst);
+  add_counters(p.ws, unused_zeros, exact_blocks);   // reported as soar_result.wide_candidates
 }
 
 // Counts the binary32 inputs with biased exponent lo_exp..hi_exp (all 2^23 significands each)
