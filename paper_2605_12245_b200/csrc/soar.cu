@@ -1526,21 +1526,21 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
         const double inf = __longlong_as_double(0x7FF0000000000000ll);
         double h0 = inf, s0 = inf, h1 = inf, s1 = inf;
         int k0 = 0, k1 = 0;
-        uint2 w0 = make_uint2(0u, 0u), w1 = w0;   // code vectors of the two current winners
         for (int k = 0; k < n_beta; ++k) {
           unsigned int c0, c1;
           round_block(mags, recip_fast(__fmul_rn(alpha, __fmul_rn(center, s_beta[k]))), c0, c1);
           double At, Bt;
           limb_sums(F, G, c0, c1, At, Bt);
-          // an equal value from the same codes is the same outcome again (a neighbouring beta); from other
-          // codes it is a tie that the images cannot resolve, and counts as a runner-up
+          // An equal value is the same outcome again (a neighbouring beta with the same codes) and is
+          // passed over, as the exact loop's strict comparison passes it over.  (Different codes with
+          // equal images differ in exact error by less than the margin below: a tie either way.)
           const double e0 = fma(rho0, Bt, -At);
-          if (e0 < h0) { s0 = h0; h0 = e0; k0 = k; w0 = make_uint2(c0, c1); }
-          else if (e0 < s0 && (e0 > h0 || c0 != w0.x || c1 != w0.y)) s0 = e0;
+          if (e0 < h0) { s0 = h0; h0 = e0; k0 = k; }
+          else if (e0 > h0 && e0 < s0) s0 = e0;
           if (nd == 2) {
             const double e1 = fma(rho1, Bt, -At);
-            if (e1 < h1) { s1 = h1; h1 = e1; k1 = k; w1 = make_uint2(c0, c1); }
-            else if (e1 < s1 && (e1 > h1 || c0 != w1.x || c1 != w1.y)) s1 = e1;
+            if (e1 < h1) { s1 = h1; h1 = e1; k1 = k; }
+            else if (e1 > h1 && e1 < s1) s1 = e1;
           }
         }
         const double q0 = 2.0 * sd0 * cA, q1 = 2.0 * sd1 * cA;
