@@ -1426,6 +1426,40 @@ weighted_init_kernel(const __grid_constant__ Batch bt, const Weighted wq, int re
   add_counters(p.ws, zeros, unused_wide);
 }
 
+// Eq. 8 for one block with binary64 sums for every candidate: index nd * k + d of the first minimum
+// in (beta, code) order.  Serves the coupled arm, code windows wider than two, and the blocks the
+// fixed-point ranking cannot decide; kept out of line so that its registers do not weigh on
+// that ranking's loop.
+__device__ __noinline__ int weighted_exact_argmin(const float* h, unsigned int cb, const Block& mags, float alpha,
+                                                  float center, const float* s_beta, int n_beta, int d_lo, int nd,
+                                                  bool coupled, bool fast_rcp) {
+  double hd[16], hw[16];
+  block_weights(h, cb, mags, hd, hw);
+  const double alpha_d = static_cast<double>(alpha);
+  double best = __longlong_as_double(0x7FF0000000000000ll);
+  int best_key = 0;
+  for (int k = 0; k < n_beta; ++k) {
+    unsigned int c0, c1;
+    double A = 0.0, B = 0.0;
+    if (!coupled) {
+      const float s = __fmul_rn(alpha, __fmul_rn(center, s_beta[k]));
+      round_block(mags, fast_rcp ? recip_fast(s) : __frcp_rn(s), c0, c1);
+      weighted_sums_split(hw, hd, c0, c1, A, B);
+    }
+    for (int d = 0; d < nd; ++d) {
+      const float dv = e4m3_value(clip_code(d_lo + d));
+      if (coupled) {
+        round_block(mags, recip_scale(alpha, __fmul_rn(dv, s_beta[k])), c0, c1);
+        weighted_sums_split(hw, hd, c0, c1, A, B);
+      }
+      const double sd = alpha_d * static_cast<double>(dv);
+      const double g = sd * fma(sd, B, -2.0 * A);
+      if (g < best) { best = g; best_key = nd * k + d; }
+    }
+  }
+  return best_key;
+}
+
 // One iteration t of Algorithm 1 under the weighted objective: Eq. 5 from the stage-t sums,
 // Eq. 6 per block from its stored {A, B}, App. B.3's candidates, Eq. 8 with the weighted
 // error written as  sum h w^2 + sd^2 B - 2 sd A  (sd = alpha * candidate scale value), first
@@ -1555,29 +1589,7 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
       }
     }
     if (!decided) {
-      // exact loop: binary64 sums for every candidate; also the coupled arm and wider code windows
-      double hd[16], hw[16];
-      block_weights(wq.h, cb, mags, hd, hw);
-      double best = __longlong_as_double(0x7FF0000000000000ll);
-      for (int k = 0; k < n_beta; ++k) {
-        unsigned int c0, c1;
-        double A = 0.0, B = 0.0;
-        if (!coupled) {
-          const float s = __fmul_rn(alpha, __fmul_rn(center, s_beta[k]));
-          round_block(mags, fast_rcp ? recip_fast(s) : __frcp_rn(s), c0, c1);
-          weighted_sums_split(hw, hd, c0, c1, A, B);
-        }
-        for (int d = 0; d < nd; ++d) {
-          const float dv = e4m3_value(clip_code(d_lo + d));
-          if (coupled) {
-            round_block(mags, recip_scale(alpha, __fmul_rn(dv, s_beta[k])), c0, c1);
-            weighted_sums_split(hw, hd, c0, c1, A, B);
-          }
-          const double sd = alpha_d * static_cast<double>(dv);
-          const double g = sd * fma(sd, B, -2.0 * A);
-          if (g < best) { best = g; best_key = nd * k + d; }
-        }
-      }
+      best_key = weighted_exact_argmin(wq.h, cb, mags, alpha, center, s_beta, n_beta, d_lo, nd, coupled, fast_rcp);
       ++exact_blocks;
     }
     // the winner, made again from its index, now with the signs and the sums in element order
