@@ -121,13 +121,14 @@ def kernel_bytes_per_elem(name: str, cfg, t: int = 0) -> float:
 
 
 # DRAM bytes per element (dram__bytes_read.sum + dram__bytes_write.sum of one launch, ncu, config 5:
-# profiles/single_pass_kernels_config5.md and profiles/iterate_kernel_paper_config5.md).  Traffic grows in
+# profiles/single_pass_kernels_config5.md, profiles/iterate_kernel_paper_config5.md and
+# profiles/weighted_iterate_kernel_config5.md).  Traffic grows in
 # proportion to the elements, so a launch's traffic is this figure times its elements.  The figures
 # belong to one version of the kernels: they are dropped when the kernel source no longer matches.
 NCU_TRAFFIC = {
-    "kernel_source_sha256_16": "0b131d2c2d88c2d3",
+    "kernel_source_sha256_16": "b180723d44702aee",
     "bytes_per_elem": {"amax_kernel": 2.02, "init_kernel": 2.43, "iterate_kernel/single": 3.00,
-                       "iterate_kernel/grid": 3.45},
+                       "iterate_kernel/grid": 3.44, "weighted_iterate_kernel": 4.59},
 }
 
 
@@ -583,8 +584,11 @@ def run_weighted(args):
         blocks_iters = sum((s.rows * s.cols // 16) * it for s, it in zip(wl.tensors, iters)) * args.steps
         achieved = blocks_iters * ops_per_block / (tot_ms * 1e-3) / 1e12
         peak = SM_COUNT * FP32_LANES_PER_SM * peaks["sm_max_mhz"] * 1e6 / 1e12
+        tpe = ncu_traffic_per_elem(dom, cfg)
+        work_elems = sum(s.rows * s.cols * it for s, it in zip(wl.tensors, iters))
         roofline = dict(bound="alu", kernel=dom, achieved=achieved, peak=peak, unit="Tlane-op/s", frac=achieved / peak,
-                        traffic=None, launches=n_launch, active_launches=sum(iters) * args.steps,
+                        traffic=None if tpe is None or sum(iters) == 0 else tpe * work_elems / sum(iters),
+                        launches=n_launch, active_launches=sum(iters) * args.steps,
                         kernel_ms_per_step=tot_ms / args.steps,
                         peak_source="148 SMs x 128 FP32 lanes x clocks.max.sm",
                         hbm_gbs_for_context=it_bytes / (tot_ms * 1e-3) / 1e9)
