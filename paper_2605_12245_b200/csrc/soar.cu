@@ -32,6 +32,13 @@
 // 16-bit fixed-point magnitudes and the codes' byte values (dp2a / dp4a), exact whenever
 // the block maximum times the reciprocal scale is at most 32; otherwise a binary64 path is
 // taken.  Tensor sums and candidate comparisons are binary64.
+//
+// Column-weighted objective (Sec. 5 in diagonal form; soar_quantize_weighted): the same passes as
+// weighted_amax_kernel, weighted_init_kernel and weighted_iterate_kernel, one matrix per launch.
+// Block sums carry a binary32 weight per column, so they are binary64 sums in element order
+// (17 bytes of state per block); the candidate loop ranks on exact integer sums over
+// fixed-point images of the weighted magnitudes and falls back to binary64 sums only for
+// blocks where the images' rounding could change the winner.
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <string.h>
