@@ -597,22 +597,14 @@ __device__ __forceinline__ bool stops_after(double prev, double cur, float eps) 
 
 // ------------------------------------------------------------------ kernels
 
-// Sum of squares of a block's sixteen bf16 values, binary64, scaled by 2^-256: a bf16
-// magnitude h (8 exponent bits e, 7 fraction bits) placed at bits 27..13 of a binary64 high
-// word and OR-ed with exponent 768 is the value times 2^-128, with no carry to handle.
-// Exact for normal bf16 values; kExact also maps zeros and bf16 subnormals (below 1.2e-38)
-// to zero, which the plain form would count as 2^-127 each.
-template <bool kExact>
+// Sum of squares of a block's sixteen bf16 values in binary64 (every square is exact).  The
+// widening is the float-to-double conversion instruction, which issues beside the integer pipe
+// that carries the rest of the pass.
 __device__ __forceinline__ void sumsq_block(const unsigned int (&u)[8], double& s0, double& s1) {
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    unsigned int lo = ((u[i] << 13) & 0x0FFFE000u) | 0x30000000u;
-    unsigned int hi = ((u[i] >> 3) & 0x0FFFE000u) | 0x30000000u;
-    if (kExact) {
-      if ((u[i] & 0x00007F80u) == 0) lo = 0;
-      if ((u[i] & 0x7F800000u) == 0) hi = 0;
-    }
-    const double dl = __hiloint2double(static_cast<int>(lo), 0), dh = __hiloint2double(static_cast<int>(hi), 0);
+    const double dl = static_cast<double>(__uint_as_float(u[i] << 16));
+    const double dh = static_cast<double>(__uint_as_float(u[i] & 0xFFFF0000u));
     s0 = fma(dl, dl, s0);
     s1 = fma(dh, dh, s1);
   }
@@ -641,7 +633,7 @@ __global__ void __launch_bounds__(kThreads, 6) amax_kernel(const __grid_constant
         mx = max(mx & 0xFFFFu, mx >> 16);
         mx = __reduce_max_sync(0xFFFFFFFFu, mx);
         if ((threadIdx.x & 31) == 0 && mx) atomicMax(&bt.t[cur].ws->amax_bits, mx);
-        double acc[1] = {(sq[0] + sq[1]) * 0x1p256};   // undo the 2^-128 scaling of the values
+        double acc[1] = {sq[0] + sq[1]};
         double* const dst[1] = {&bt.t[cur].ws->sumsq};
         slots_add(slots, cur, acc, dst);
         mx = 0;
@@ -653,21 +645,18 @@ __global__ void __launch_bounds__(kThreads, 6) amax_kernel(const __grid_constant
     }
     if (tile * kTile + threadIdx.x >= nblk) continue;
     const unsigned int u[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-    // largest and smallest magnitude of the block with packed bf16 min/max (a NaN input comes out
-    // of the maximum as NaN, whose bits are above the infinity pattern)
-    unsigned int bmx = 0, bmn = 0x7F7F7F7Fu;
+    // largest magnitude of the block with packed bf16 max (a NaN input comes out of the maximum
+    // as NaN, whose bits are above the infinity pattern)
+    unsigned int bmx = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       unsigned int m;
       asm("abs.bf16x2 %0, %1;" : "=r"(m) : "r"(u[i]));
       asm("max.NaN.bf16x2 %0, %0, %1;" : "+r"(bmx) : "r"(m));
-      asm("min.bf16x2 %0, %0, %1;" : "+r"(bmn) : "r"(m));
     }
     bmx &= 0x7FFF7FFFu;
     mx = __vmaxu2(mx, bmx);
-    // a magnitude below 0x0080 has a zero exponent field: zero or subnormal
-    if (min(bmn & 0xFFFFu, bmn >> 16) >= 0x80u) sumsq_block<false>(u, sq[0], sq[1]);
-    else sumsq_block<true>(u, sq[0], sq[1]);
+    sumsq_block(u, sq[0], sq[1]);
   }
 }
 
@@ -1111,9 +1100,10 @@ __global__ void __launch_bounds__(256) swizzle_kernel(const uint8_t* lin, uint8_
 }
 
 // Eq. 3-4 on stored outputs: sum (w - q s)^2 and sum w^2, one binary64 fma per term, with the
-// bf16 values widened by bit placement (scaled by 2^-128, undone at the end) and the signed
-// E2M1 values read from a 16-entry table in shared memory.  A wait that gave up turns the
-// results into NaN.  kWeighted multiplies every term by its column's weight h_j.
+// bf16 values widened by the conversion instruction (which runs beside the integer and
+// binary64 pipes) and the signed E2M1 values read from a 16-entry table in shared memory.
+// A wait that gave up turns the results into NaN.  kWeighted multiplies every term by its
+// column's weight h_j.
 template <bool kWeighted>
 __global__ void __launch_bounds__(kThreads) dequant_error_kernel(const __grid_constant__ Batch bt,
                                                                  const uint8_t* scales, int swizzled,
@@ -1134,7 +1124,7 @@ __global__ void __launch_bounds__(kThreads) dequant_error_kernel(const __grid_co
     if (threadIdx.x == kTile) ring_produce(ring, bt, 0, 1u);
     return;
   }
-  const double alpha_scaled = static_cast<double>(*alpha_ptr) * 0x1p-128;
+  const double alpha_d = static_cast<double>(*alpha_ptr);
   double acc[2] = {0.0, 0.0};
   for (unsigned int n = 0;; ++n) {
     uint4 v0, v1;
@@ -1151,20 +1141,15 @@ __global__ void __launch_bounds__(kThreads) dequant_error_kernel(const __grid_co
     } else {
       dc = scales[b];
     }
-    const double s = alpha_scaled * static_cast<double>(e4m3_value(dc & 0x7F));
+    const double s = alpha_d * static_cast<double>(e4m3_value(dc & 0x7F));
     const unsigned int u[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
     double hd[16];
     if (kWeighted) load_weights(h, b % p.nbc, hd);
     double e0 = 0.0, e1 = 0.0, q0 = 0.0, q1 = 0.0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      // magnitude at bits 27..13 with exponent offset 768 (value * 2^-128), sign at bit 31;
-      // zeros and bf16 subnormals become zero
-      unsigned int lo = ((u[i] << 13) & 0x0FFFE000u) | 0x30000000u | ((u[i] << 16) & 0x80000000u);
-      unsigned int hi = ((u[i] >> 3) & 0x0FFFE000u) | 0x30000000u | (u[i] & 0x80000000u);
-      if ((u[i] & 0x00007F80u) == 0) lo = 0;
-      if ((u[i] & 0x7F800000u) == 0) hi = 0;
-      const double wl = __hiloint2double(static_cast<int>(lo), 0), wh = __hiloint2double(static_cast<int>(hi), 0);
+      const double wl = static_cast<double>(__uint_as_float(u[i] << 16));
+      const double wh = static_cast<double>(__uint_as_float(u[i] & 0xFFFF0000u));
       const unsigned int word = (i < 4) ? cw.x : cw.y;
       const double ql = s_q[(word >> (8 * (i & 3))) & 0xFu], qh = s_q[(word >> (8 * (i & 3) + 4)) & 0xFu];
       const double dl = fma(-ql, s, wl), dh = fma(-qh, s, wh);
@@ -1184,8 +1169,7 @@ __global__ void __launch_bounds__(kThreads) dequant_error_kernel(const __grid_co
     acc[1] += q0 + q1;
   }
   const bool failed = *static_cast<volatile int*>(&ring.fail) != 0;
-  acc[0] = failed ? __longlong_as_double(0x7FF8000000000000ll) : acc[0] * 0x1p256;
-  acc[1] = failed ? __longlong_as_double(0x7FF8000000000000ll) : acc[1] * 0x1p256;
+  if (failed) acc[0] = acc[1] = __longlong_as_double(0x7FF8000000000000ll);
   double* const dst[2] = {out_sse, out_sumsq};
   slots_add(slots, 0, acc, dst);
 }
