@@ -173,6 +173,48 @@ size_t soar_batch_workspace_bytes(const soar_tensor_desc* tensors, int n, const 
 int soar_quantize_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void* workspace,
                         size_t workspace_bytes, void* stream);
 
+/*
+ * The accumulators at the head of a workspace.  Matrix i of a batch owns the
+ * SOAR_WORKSPACE_HEADER_BYTES bytes at byte i * SOAR_WORKSPACE_HEADER_BYTES of `workspace`
+ * (soar_quantize: i = 0), laid out as below.  They are all that couples the blocks of a tensor
+ * (Algorithm 1: the maximum of Eq. 1, the two sums of Eq. 5, the error of Sec. 4.1's stop), and
+ * they are public for one purpose: a caller that splits a tensor's rows over several GPUs runs
+ * soar_quantize_stage on each part and, between stages, combines these fields over the parts.
+ */
+#define SOAR_WORKSPACE_HEADER_BYTES 2048
+typedef struct soar_workspace_header {
+  uint32_t amax_bits;               /* bf16 bit pattern of max |W|: combine with max           */
+  uint32_t error;                   /* non-zero stops the remaining stages: combine with OR/max */
+  uint64_t zero_blocks;             /* counters for the report: sum                            */
+  uint64_t wide;
+  double sumsq;                     /* sum W^2: sum                                            */
+  double num[SOAR_MAX_ITERS + 1];   /* stage s: sum A_b * scale_b      (numerator of Eq. 5): sum   */
+  double den[SOAR_MAX_ITERS + 1];   /* stage s: sum B_b * scale_b^2    (denominator of Eq. 5): sum */
+  double gsum[SOAR_MAX_ITERS + 1];  /* stage s: error minus sum W^2    (Eq. 4): sum            */
+} soar_workspace_header;
+
+/*
+ * soar_quantize_batch one stage at a time, for tensors whose rows are split over several
+ * GPUs (or several calls).  The stages, in order: SOAR_STAGE_AMAX (clears the headers; writes
+ * amax_bits, sumsq), SOAR_STAGE_INIT (stage-0 entries of num, den, gsum; zero_blocks),
+ * iteration t = 0 .. max_iters-1 passed as `stage` = t (entries t+1 of num, den, gsum; wide),
+ * SOAR_STAGE_FINALIZE (alpha, report, swizzled scales).  Each stage reads the header entries the
+ * earlier stages wrote, so a caller that has split a tensor combines, after every stage, the
+ * fields that stage wrote over all parts (sum or max as marked above, e.g. with an all-reduce
+ * on the same stream) and every part then continues with the whole tensor's values: alpha, the
+ * early stop and the report come out as for the unsplit tensor, up to the order of the
+ * binary64 additions.  Run over one part with nothing combined, the stages in order are
+ * exactly soar_quantize_batch.  Arguments, checks and error codes as soar_quantize_batch; an
+ * unknown stage returns SOAR_ERR_INVALID_ARG.  The swizzled scale layout is tiled by 128 rows,
+ * so a part's rows must be a multiple of 128 for its swizzled output to be a slice of the
+ * whole tensor's.
+ */
+#define SOAR_STAGE_AMAX (-3)
+#define SOAR_STAGE_INIT (-2)
+#define SOAR_STAGE_FINALIZE (-1)
+int soar_quantize_stage(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void* workspace,
+                        size_t workspace_bytes, int stage, void* stream);
+
 /* Device staging buffers for soar_quantize_host (all device memory, caller-owned, same sizes
  * and alignment as the matching soar_quantize arguments; W holds rows*ld bf16 elements). */
 typedef struct soar_staging {

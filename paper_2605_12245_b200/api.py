@@ -30,6 +30,7 @@ EXPORTS = (
     "soar_trace_begin", "soar_trace_end", "soar_quantize_static", "soar_selftest_reciprocal",
     "soar_batch_workspace_bytes", "soar_quantize_batch",
     "soar_weighted_workspace_bytes", "soar_quantize_weighted", "soar_dequant_error_weighted",
+    "soar_quantize_stage",
 )
 
 
@@ -124,6 +125,9 @@ def lib() -> C.CDLL:
                                              C.c_size_t, vp, vp]
         L.soar_dequant_error_weighted.restype = C.c_int
         L.soar_dequant_error_weighted.argtypes = [vp, i64, i64, i64, vp, vp, vp, C.c_int, vp, vp, vp, vp]
+        L.soar_quantize_stage.restype = C.c_int
+        L.soar_quantize_stage.argtypes = [C.POINTER(SoarTensorDesc), C.c_int, C.POINTER(SoarCfg), vp, C.c_size_t,
+                                          C.c_int, vp]
         L.soar_selftest_reciprocal.restype = C.c_int
         L.soar_selftest_reciprocal.argtypes = [C.c_int, C.c_int, vp, vp]
         L.soar_trace_begin.restype = C.c_int
@@ -289,6 +293,30 @@ def soar_quantize_batch(Ws, cfg: SoarCfg, outs, workspace: torch.Tensor | None =
 
 
 STATIC_MAX_ELEMENTS = 1 << 24
+
+
+STAGE_AMAX, STAGE_INIT, STAGE_FINALIZE = -3, -2, -1
+WORKSPACE_HEADER_BYTES = 2048
+
+
+class SoarWorkspaceHeader(C.Structure):
+    """Mirror of ``soar_workspace_header`` (used for field offsets only)."""
+
+    _fields_ = [
+        ("amax_bits", C.c_uint32), ("error", C.c_uint32), ("zero_blocks", C.c_uint64), ("wide", C.c_uint64),
+        ("sumsq", C.c_double), ("num", C.c_double * (MAX_ITERS + 1)), ("den", C.c_double * (MAX_ITERS + 1)),
+        ("gsum", C.c_double * (MAX_ITERS + 1)),
+    ]
+
+
+def soar_quantize_stage(Ws, cfg: SoarCfg, outs, workspace: torch.Tensor, stage: int, stream=None) -> None:
+    """Enqueue one stage of ``soar_quantize_batch`` (``STAGE_AMAX``, ``STAGE_INIT``, iteration ``t >= 0``,
+    ``STAGE_FINALIZE``) for the matrices ``Ws`` with output buffers ``outs`` and a shared ``workspace``."""
+    d = _descs(Ws, outs)
+    _require_cuda(workspace)
+    rc = lib().soar_quantize_stage(d, len(Ws), C.byref(cfg), _ptr(workspace), workspace.numel(), int(stage),
+                                   _stream_ptr(stream))
+    _check(rc, "soar_quantize_stage")
 
 
 def soar_quantize_static(W: torch.Tensor, cfg: SoarCfg, out: QuantBuffers, stream=None) -> QuantBuffers:

@@ -40,6 +40,7 @@
 // fixed-point images of the weighted magnitudes and falls back to binary64 sums only for
 // blocks where the images' rounding could change the winner.
 #include <cuda_runtime.h>
+#include <stddef.h>
 #include <stdint.h>
 #include <string.h>
 
@@ -68,6 +69,17 @@ struct Ws {
   double gsum[SOAR_MAX_ITERS + 1];   // stage s: sum of block errors minus sum W^2 (Eq. 4)
 };
 static_assert(sizeof(Ws) <= kWsFixedBytes, "workspace header too large");
+// the same layout is published as soar_workspace_header
+static_assert(kWsFixedBytes == SOAR_WORKSPACE_HEADER_BYTES && sizeof(Ws) == sizeof(soar_workspace_header) &&
+                  offsetof(Ws, amax_bits) == offsetof(soar_workspace_header, amax_bits) &&
+                  offsetof(Ws, error) == offsetof(soar_workspace_header, error) &&
+                  offsetof(Ws, zero_blocks) == offsetof(soar_workspace_header, zero_blocks) &&
+                  offsetof(Ws, wide) == offsetof(soar_workspace_header, wide) &&
+                  offsetof(Ws, sumsq) == offsetof(soar_workspace_header, sumsq) &&
+                  offsetof(Ws, num) == offsetof(soar_workspace_header, num) &&
+                  offsetof(Ws, den) == offsetof(soar_workspace_header, den) &&
+                  offsetof(Ws, gsum) == offsetof(soar_workspace_header, gsum),
+              "Ws and soar_workspace_header differ");
 constexpr unsigned int kErrWait = 1u;     // a bounded wait gave up
 constexpr unsigned int kErrWeight = 2u;   // a column weight outside the accepted set
 
@@ -1792,8 +1804,16 @@ size_t soar_batch_workspace_bytes(const soar_tensor_desc* tensors, int n, const 
   return total;
 }
 
-int soar_quantize_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void* workspace,
-                        size_t workspace_bytes, void* stream) {
+}  // extern "C"
+
+namespace {
+
+// Which launches a call makes: all of them (soar_quantize_batch), or one stage
+// (soar_quantize_stage; iterations t_lo <= t < t_hi for kStageIterate).
+enum : int { kStageAmax = 1, kStageInit = 2, kStageIterate = 4, kStageFinalize = 8, kStageAll = 15 };
+
+int run_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void* workspace, size_t workspace_bytes,
+              void* stream, int stages, int t_lo, int t_hi) {
   int rc = check_cfg(cfg);
   if (rc != SOAR_OK) return rc;
   if (tensors == nullptr || n <= 0) return SOAR_ERR_INVALID_ARG;
@@ -1816,7 +1836,9 @@ int soar_quantize_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* 
   // workspace: the n headers first (one memset clears them all), then each tensor's arrays
   uint8_t* const headers = static_cast<uint8_t*>(workspace);
   uint8_t* next = headers + static_cast<size_t>(n) * kWsFixedBytes;
-  if (cudaMemsetAsync(headers, 0, static_cast<size_t>(n) * kWsFixedBytes, st) != cudaSuccess) return SOAR_ERR_CUDA;
+  if ((stages & kStageAmax) &&
+      cudaMemsetAsync(headers, 0, static_cast<size_t>(n) * kWsFixedBytes, st) != cudaSuccess)
+    return SOAR_ERR_CUDA;
 
   const bool single = cfg->n_beta == 1 && cfg->n_dq <= 2;
   const bool may_stop = cfg->early_stop_rel > 0.0f;
@@ -1863,33 +1885,34 @@ int soar_quantize_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* 
     for (int j = bt.n; j < kMaxBatch; ++j) bt.tile_end[j] = 0xFFFFFFFFu;   // never reached by a tile index
     bt.total_tiles = tiles;
 
-    // Passes alternate direction over the tiles: each starts where the previous one ended,
-    // on data still in L2.
-    int reverse = 0;
-    {
+    // Passes alternate direction over the tiles (amax forward, init backward, iteration t forward
+    // for even t): each starts where the previous one ended, on data still in L2.
+    if (stages & kStageAmax) {
       ScopedLaunch sl(K_AMAX, st);
-      amax_kernel<<<persistent_grid(amax_kernel, tiles, kThreads), kThreads, 0, st>>>(bt, reverse);
+      amax_kernel<<<persistent_grid(amax_kernel, tiles, kThreads), kThreads, 0, st>>>(bt, 0);
     }
-    reverse ^= 1;
-    {
+    if (stages & kStageInit) {
       ScopedLaunch sl(K_INIT, st);
-      init_kernel<<<persistent_grid(init_kernel, tiles, kThreads), kThreads, 0, st>>>(bt, reverse,
+      init_kernel<<<persistent_grid(init_kernel, tiles, kThreads), kThreads, 0, st>>>(bt, 1,
                                                                                       cfg->max_iters == 0 ? 1 : 0);
     }
-    const int mode = !single ? 0 : ((cfg->flags & SOAR_FLAG_COUPLED_SCALE) ? 2 : 1);
-    const unsigned int g_it = mode == 0   ? persistent_grid(iterate_kernel<0>, tiles, kThreads)
-                              : mode == 1 ? persistent_grid(iterate_kernel<1>, tiles, kThreads)
-                                          : persistent_grid(iterate_kernel<2>, tiles, kThreads);
-    for (int t = 0; t < cfg->max_iters; ++t) {
-      reverse ^= 1;
-      // with the early stop on, any iteration may turn out to be the last one
-      const int last = (t == cfg->max_iters - 1) ? 1 : 0;
-      const int emit = (may_stop || last) ? 1 : 0;
-      ScopedLaunch sl(K_ITERATE, st);
-      if (mode == 0) iterate_kernel<0><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
-      else if (mode == 1) iterate_kernel<1><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
-      else iterate_kernel<2><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
+    if (stages & kStageIterate) {
+      const int mode = !single ? 0 : ((cfg->flags & SOAR_FLAG_COUPLED_SCALE) ? 2 : 1);
+      const unsigned int g_it = mode == 0   ? persistent_grid(iterate_kernel<0>, tiles, kThreads)
+                                : mode == 1 ? persistent_grid(iterate_kernel<1>, tiles, kThreads)
+                                            : persistent_grid(iterate_kernel<2>, tiles, kThreads);
+      for (int t = t_lo; t < t_hi; ++t) {
+        const int reverse = t & 1;
+        // with the early stop on, any iteration may turn out to be the last one
+        const int last = (t == cfg->max_iters - 1) ? 1 : 0;
+        const int emit = (may_stop || last) ? 1 : 0;
+        ScopedLaunch sl(K_ITERATE, st);
+        if (mode == 0) iterate_kernel<0><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
+        else if (mode == 1) iterate_kernel<1><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
+        else iterate_kernel<2><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
+      }
     }
+    if (!(stages & kStageFinalize)) continue;
     {
       ScopedLaunch sl(K_FINALIZE, st);
       finalize_kernel<<<bt.n, 128, 0, st>>>(bt, rp);
@@ -1910,6 +1933,29 @@ int soar_quantize_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* 
     }
   }
   return cudaGetLastError() == cudaSuccess ? SOAR_OK : SOAR_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+int soar_quantize_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+  const int rc = check_cfg(cfg);
+  if (rc != SOAR_OK) return rc;
+  return run_batch(tensors, n, cfg, workspace, workspace_bytes, stream, kStageAll, 0, cfg->max_iters);
+}
+
+int soar_quantize_stage(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void* workspace,
+                        size_t workspace_bytes, int stage, void* stream) {
+  const int rc = check_cfg(cfg);
+  if (rc != SOAR_OK) return rc;
+  if (stage == SOAR_STAGE_AMAX) return run_batch(tensors, n, cfg, workspace, workspace_bytes, stream, kStageAmax, 0, 0);
+  if (stage == SOAR_STAGE_INIT) return run_batch(tensors, n, cfg, workspace, workspace_bytes, stream, kStageInit, 0, 0);
+  if (stage == SOAR_STAGE_FINALIZE)
+    return run_batch(tensors, n, cfg, workspace, workspace_bytes, stream, kStageFinalize, 0, 0);
+  if (stage < 0 || stage >= cfg->max_iters) return SOAR_ERR_INVALID_ARG;
+  return run_batch(tensors, n, cfg, workspace, workspace_bytes, stream, kStageIterate, stage, stage + 1);
 }
 
 int soar_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, const soar_cfg* cfg,

@@ -57,3 +57,64 @@ def test_single_process_helpers_need_no_process_group():
     assert S.whole_job_throughput(10.0, 2.0) == 5.0
     with pytest.raises(ValueError):
         S.assign_tensors(5, 2, 2)
+
+
+# ---- one tensor split by rows: the header plumbing between stages (no kernels run here)
+
+def _header_worker(rank, world, port, out_dir):
+    import ctypes as C
+
+    from paper_2605_12245_b200 import api
+    from paper_2605_12245_b200 import row_sharded as RS
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        T = 3
+        h = api.SoarWorkspaceHeader()
+        h.amax_bits = 0x3C00 + 7 * rank                 # the larger one must win
+        h.error = rank                                  # an error on any part stops all
+        h.zero_blocks = 10 + rank
+        h.wide = 100 * (rank + 1)
+        h.sumsq = 1.5 + rank
+        for i in range(T + 1):
+            h.num[i], h.den[i], h.gsum[i] = 1.0 + i + 10 * rank, 2.0 + i + 20 * rank, -(3.0 + i) - rank
+        raw = bytearray(api.WORKSPACE_HEADER_BYTES)
+        raw[:C.sizeof(h)] = bytes(h)
+        header = torch.frombuffer(raw, dtype=torch.uint8)
+        snaps = []
+        for stage in RS.stages(T):
+            RS.combine_header(header, stage, T, RS.dist_all_reduce())
+            snaps.append(bytes(raw[:C.sizeof(h)]))
+        np.save(os.path.join(out_dir, f"h{rank}.npy"), np.frombuffer(b"".join(snaps), dtype=np.uint8))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_row_sharded_header_fields_are_combined_stage_by_stage(tmp_path):
+    import ctypes as C
+
+    from paper_2605_12245_b200 import api
+    from paper_2605_12245_b200 import row_sharded as RS
+    world, port, T = 2, _free_port(), 3
+    mp.spawn(_header_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    size = C.sizeof(api.SoarWorkspaceHeader)
+    per_rank = [np.load(tmp_path / f"h{r}.npy").reshape(-1, size) for r in range(world)]
+    stage_list = RS.stages(T)
+    assert stage_list == [api.STAGE_AMAX, api.STAGE_INIT, 0, 1, 2, api.STAGE_FINALIZE]
+    for r in range(world):
+        snaps = [api.SoarWorkspaceHeader.from_buffer_copy(per_rank[r][i].tobytes()) for i in range(len(stage_list))]
+        a = snaps[0]                                   # after the amax stage
+        assert a.amax_bits == 0x3C07 and a.error == 1 and a.sumsq == 1.5 + 2.5
+        assert a.num[0] == 1.0 + 10 * r and a.zero_blocks == 10 + r          # not yet combined
+        b = snaps[1]                                   # after init: stage-0 sums and the zero-block count
+        assert (b.num[0], b.den[0], b.gsum[0]) == (1.0 + 11.0, 2.0 + 22.0, -3.0 - 4.0)
+        assert b.zero_blocks == 21 and b.sumsq == 4.0                        # sumsq is not added twice
+        assert b.num[1] == 2.0 + 10 * r and b.wide == 100 * (r + 1)
+        for t in range(T):                             # after iteration t: entries t+1
+            c = snaps[2 + t]
+            assert (c.num[t + 1], c.den[t + 1], c.gsum[t + 1]) == (2 * (2.0 + t) + 10, 2 * (3.0 + t) + 20, -2 * (4.0 + t) - 1)
+            if t + 2 <= T:
+                assert c.num[t + 2] == 3.0 + t + 10 * r                      # later entries untouched
+        # the counter that grows in every stage is combined once, after the last iteration
+        assert snaps[2].wide == snaps[3].wide == 100 * (r + 1) and snaps[4].wide == 300
+        assert bytes(snaps[-1]) == bytes(snaps[-2])    # nothing is combined after the report stage
