@@ -672,6 +672,100 @@ def run_weighted(args):
         dist.destroy_process_group()
 
 
+def run_row_sharded(args):
+    """One tensor (the workload's largest) split by rows over the ranks: strong scaling.  Each rank runs the
+    stages on its rows and the ranks all-reduce the workspace-header fields between stages."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2605_12245_b200 import api
+    from paper_2605_12245_b200 import row_sharded as RS
+    from paper_2605_12245_b200 import sharding as SH
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    api.lib()
+    peaks = load_peaks()
+    wl = pick_workload(args.workload)
+    ti = max(range(len(wl.tensors)), key=lambda i: wl.tensors[i].rows * wl.tensors[i].cols)
+    spec = wl.tensors[ti]
+    cr = WL._chunk_rows(spec.cols)                       # parts start on the generator's chunk boundaries
+    per = ((spec.rows + world - 1) // world + cr - 1) // cr * cr
+    r0, r1 = min(spec.rows, rank * per), min(spec.rows, (rank + 1) * per)
+    cfg = preset_cfg(api, args.preset, args)
+    W = torch.from_numpy(wl.generate(ti, r0, r1).view(np.int16)).view(torch.bfloat16).cuda()
+    out = api.alloc_buffers(r1 - r0, spec.cols, cfg)
+    stream = torch.cuda.current_stream()
+    elements = spec.rows * spec.cols
+
+    if world == 1:      # no process group: the combine step still runs, over one part
+        def reduce(buf, how):
+            return None
+    else:
+        reduce = RS.dist_all_reduce()
+    header = out.workspace[:api.WORKSPACE_HEADER_BYTES]
+
+    def step():
+        for stage in RS.stages(cfg.max_iters):
+            api.soar_quantize_stage([W], cfg, [out], out.workspace, stage)
+            RS.combine_header(header, stage, cfg.max_iters, reduce)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    api.soar_trace_begin()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    trace = api.soar_trace_end()
+    barrier()
+    clocks = sampler.stop()
+    ms = SH.max_over_ranks(e0.elapsed_time(e1) / args.steps, "cuda")
+    res = out.read_result()
+    dom = max(trace, key=lambda k: trace[k][1])
+    n_launch, tot_ms = trace[dom]
+    local_blocks = (r1 - r0) * spec.cols // 16
+    ops = local_blocks * res.iters_run * iterate_ops_per_block(cfg) * args.steps
+    peak = SM_COUNT * FP32_LANES_PER_SM * peaks["sm_max_mhz"] * 1e6 / 1e12
+    achieved = ops / (tot_ms * 1e-3) / 1e12
+    if rank == 0:
+        line = dict(
+            metric="soar_quantize_bf16_input_throughput", value=2.0 * elements / (ms * 1e-3) / 1e9, unit="GB/s",
+            n_gpus=world, steps=args.steps, warmup=args.warmup, ms_per_step=ms, higher_is_better=True,
+            scaling="strong", vs_baseline=None, dtype="f32", data="synthetic",
+            config=dict(workload=wl.name, tensor=spec.name, rows=spec.rows, cols=spec.cols, preset=args.preset,
+                        max_iters=cfg.max_iters, n_beta=cfg.n_beta, n_dq=cfg.n_dq, early_stop_rel=cfg.early_stop_rel,
+                        iters_run=res.iters_run, elements=elements,
+                        l2="inputs (%.2f GB per rank) exceed the 126 MB L2" % (2 * (r1 - r0) * spec.cols / 1e9),
+                        parallelism=f"{world} rank(s), rows split evenly, two small all-reduces per stage"),
+            elements_per_s=elements / (ms * 1e-3),
+            roofline=dict(bound="alu", kernel=dom, achieved=achieved, peak=peak, unit="Tlane-op/s",
+                          frac=achieved / peak, traffic=None, launches=n_launch, kernel_ms_per_step=tot_ms / args.steps,
+                          peak_source="148 SMs x 128 FP32 lanes x clocks.max.sm (rank 0's kernels and rows)"),
+            kernels={k: dict(launches=v[0], ms_per_step=v[1] / args.steps) for k, v in trace.items()},
+            cpu_baseline=None, e2e=None, gpu_launches=sum(v[0] for v in trace.values()), clocks=clocks)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -687,6 +781,8 @@ def main():
     ap.add_argument("--sweep", default="", help="comma-separated candidate-pair counts to time, one iteration each")
     ap.add_argument("--objective", default="plain", choices=["plain", "weighted"],
                     help="weighted: the column-weighted objective through soar_quantize_weighted")
+    ap.add_argument("--row-sharded", action="store_true",
+                    help="split the workload's largest tensor by rows over the ranks (strong scaling)")
     ap.add_argument("--no-batch", action="store_true", help="one soar_quantize call per tensor instead of soar_quantize_batch")
     ap.add_argument("--graph", action="store_true", help="replay each step from a CUDA graph (no per-kernel trace)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -696,6 +792,8 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.row_sharded:
+        run_row_sharded(args)
     elif args.objective == "weighted":
         run_weighted(args)
     else:
