@@ -126,7 +126,7 @@ def kernel_bytes_per_elem(name: str, cfg, t: int = 0) -> float:
 # proportion to the elements, so a launch's traffic is this figure times its elements.  The figures
 # belong to one version of the kernels: they are dropped when the kernel source no longer matches.
 NCU_TRAFFIC = {
-    "kernel_source_sha256_16": "f37eecb5c996b54d",
+    "kernel_source_sha256_16": "ebb21c61ca096541",
     "bytes_per_elem": {"amax_kernel": 2.02, "init_kernel": 2.43, "iterate_kernel/single": 3.00,
                        "iterate_kernel/grid": 3.44, "weighted_iterate_kernel": 4.59},
 }
