@@ -124,22 +124,34 @@ def kernel_bytes_per_elem(name: str, cfg, t: int = 0) -> float:
 # profiles/single_pass_kernels_config5.md, profiles/iterate_kernel_paper_config5.md and
 # profiles/weighted_iterate_kernel_config5.md).  Traffic grows in
 # proportion to the elements, so a launch's traffic is this figure times its elements.  The figures
-# belong to one version of the kernels: they are dropped when the kernel source no longer matches.
+# belong to one version of the kernels: they are dropped when the device part of the source (everything above
+# the host-side section of soar.cu) no longer matches.
 NCU_TRAFFIC = {
-    "kernel_source_sha256_16": "ebb21c61ca096541",
+    "kernel_source_sha256_16": "9eb1d56795922166",
     "bytes_per_elem": {"amax_kernel": 2.02, "init_kernel": 2.43, "iterate_kernel/single": 3.00,
                        "iterate_kernel/grid": 3.44, "weighted_iterate_kernel": 4.59},
 }
 
 
-def ncu_traffic_per_elem(name: str, cfg):
-    import hashlib
+HOST_MARKER = b"// ------------------------------------------------------------------ host side"
+
+
+def kernel_source_hash() -> str | None:
+    """sha256 (16 hex digits) of the device part of soar.cu: everything above the host-side section."""
     src = os.path.join(ROOT, "paper_2605_12245_b200", "csrc", "soar.cu")
+    import hashlib
     try:
         with open(src, "rb") as f:
-            if hashlib.sha256(f.read()).hexdigest()[:16] != NCU_TRAFFIC["kernel_source_sha256_16"]:
-                return None
+            text = f.read()
     except OSError:
+        return None
+    if HOST_MARKER not in text:
+        return None
+    return hashlib.sha256(text.split(HOST_MARKER)[0]).hexdigest()[:16]
+
+
+def ncu_traffic_per_elem(name: str, cfg):
+    if kernel_source_hash() != NCU_TRAFFIC["kernel_source_sha256_16"]:
         return None
     if name == "iterate_kernel":
         name += "/single" if (cfg.n_beta == 1 and cfg.n_dq <= 2) else "/grid"
