@@ -118,3 +118,28 @@ def test_row_sharded_header_fields_are_combined_stage_by_stage(tmp_path):
         # the counter that grows in every stage is combined once, after the last iteration
         assert snaps[2].wide == snaps[3].wide == 100 * (r + 1) and snaps[4].wide == 300
         assert bytes(snaps[-1]) == bytes(snaps[-2])    # nothing is combined after the report stage
+
+
+def test_row_sharded_schedule_combines_every_written_entry_exactly_once():
+    from paper_2605_12245_b200 import api
+    from paper_2605_12245_b200 import row_sharded as RS
+    for T in (0, 1, 4):
+        seen = []
+        for stage in RS.stages(T):
+            seen += [(n, i) for n, i, how in RS.fields_written(stage, T) if how == RS.SUM]
+        want = [("sumsq", 0), ("zero_blocks", 0), ("wide", 0)] + [(f, i) for f in ("num", "den", "gsum") for i in range(T + 1)]
+        assert sorted(seen) == sorted(want)                     # sums: once each, none missing
+        assert RS.fields_written(api.STAGE_FINALIZE, T) == []
+        # the counter that grows until the report is combined after the last stage before it
+        last = T - 1 if T > 0 else api.STAGE_INIT
+        assert ("wide", 0, RS.SUM) in RS.fields_written(last, T)
+    with pytest.raises(ValueError):
+        RS.fields_written(4, 4)
+    # views address the published layout
+    import ctypes as C
+    raw = bytearray(api.WORKSPACE_HEADER_BYTES)
+    header = torch.frombuffer(raw, dtype=torch.uint8)
+    RS.header_view(header, "den", 3).fill_(2.5)
+    RS.header_view(header, "amax_bits").fill_(0x3F80)
+    h = api.SoarWorkspaceHeader.from_buffer_copy(bytes(raw[:C.sizeof(api.SoarWorkspaceHeader)]))
+    assert h.den[3] == 2.5 and h.amax_bits == 0x3F80 and h.num[3] == 0.0
