@@ -47,3 +47,31 @@ def test_host_side_helpers():
     assert api.lib().soar_status_string(-3).decode().startswith("workspace")
     bad = api.soar_default_cfg(n_beta=0)
     assert api.soar_workspace_bytes(128, 256, bad) == 0
+
+
+def test_python_mirrors_of_the_public_structs_match_the_header(tmp_path):
+    """Compile the header with gcc and compare sizes and field offsets with the ctypes mirrors."""
+    import subprocess
+    structs = {"soar_cfg": api.SoarCfg, "soar_result": api.SoarResult, "soar_tensor_desc": api.SoarTensorDesc,
+               "soar_staging": api.SoarStaging, "soar_trace_entry": api.SoarTraceEntry,
+               "soar_workspace_header": api.SoarWorkspaceHeader}
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "soar.h"', "int main(void) {"]
+    for cname, py in structs.items():
+        lines.append(f'  printf("{cname} %zu\\n", sizeof({cname}));')
+        for fname, *_ in py._fields_:
+            lines.append(f'  printf("{cname}.{fname} %zu\\n", offsetof({cname}, {fname}));')
+    lines += ['  printf("HEADER_BYTES %d\\n", SOAR_WORKSPACE_HEADER_BYTES);',
+              '  printf("STAGES %d %d %d\\n", SOAR_STAGE_AMAX, SOAR_STAGE_INIT, SOAR_STAGE_FINALIZE);',
+              "  return 0;", "}"]
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.check_call(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
+    got = dict(l.rsplit(" ", 1) if not l.startswith("STAGES") else ("STAGES", l[7:])
+               for l in subprocess.check_output([str(exe)], text=True).splitlines())
+    for cname, py in structs.items():
+        assert int(got[cname]) == C.sizeof(py), cname
+        for fname, *_ in py._fields_:
+            assert int(got[f"{cname}.{fname}"]) == getattr(py, fname).offset, (cname, fname)
+    assert int(got["HEADER_BYTES"]) == api.WORKSPACE_HEADER_BYTES >= C.sizeof(api.SoarWorkspaceHeader)
+    assert [int(v) for v in got["STAGES"].split()] == [api.STAGE_AMAX, api.STAGE_INIT, api.STAGE_FINALIZE]
