@@ -82,13 +82,15 @@ def compare(gpu: GpuOut, ref: R.RefResult) -> Report:
                   float(alpha_rel), float(sse_rel))
 
 
-def assert_parity(gpu: GpuOut, ref: R.RefResult) -> Report:
+def assert_parity(gpu: GpuOut, ref: R.RefResult, mismatch_cap: int | None = None) -> Report:
+    """``mismatch_cap`` replaces the 0.01 % bound on mismatching blocks (all of which must lie in blocks the
+    oracle flagged as ties) for tensors so small that one block is already more than 0.01 %."""
     rep = compare(gpu, ref)
     assert gpu.result.status == ref.status
     assert gpu.result.iters_run == ref.iters_run, (gpu.result.iters_run, ref.iters_run)
     assert rep.alpha_rel <= ALPHA_RTOL, rep
     assert rep.mismatched_outside_ties == 0, rep
-    assert rep.mismatched <= MAX_MISMATCH_FRACTION * rep.blocks, rep
+    assert rep.mismatched <= (MAX_MISMATCH_FRACTION * rep.blocks if mismatch_cap is None else mismatch_cap), rep
     assert rep.sse_rel <= SSE_RTOL, rep
     n = ref.iters_run + 1
     ta = np.array(gpu.result.trace_alpha[:n])
