@@ -154,7 +154,7 @@ def ncu_traffic_per_elem(name: str, cfg):
     if kernel_source_hash() != NCU_TRAFFIC["kernel_source_sha256_16"]:
         return None
     if name == "iterate_kernel":
-        name += "/single" if (cfg.n_beta == 1 and cfg.n_dq <= 2) else "/grid"
+        name += "/single" if cfg.n_beta == 1 and not (cfg.n_dq > 2 and cfg.flags & 1) else "/grid"
     return NCU_TRAFFIC["bytes_per_elem"].get(name)
 
 
@@ -434,6 +434,16 @@ def run_ours(args):
                                  achieved_gbs=k_bytes / (k_ms * 1e-3) / 1e9,
                                  frac_of_measured_hbm=k_bytes / (k_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]))
         extra["sweep"] = rows_out
+    if args.sweep_dq:      # the other axis: one quantization scale (beta = 1), K E4M3 codes around it
+        rows_out = []
+        for K in [int(x) for x in args.sweep_dq.split(",")]:
+            c = api.soar_default_cfg(api.PRESET_SINGLE_PASS, n_dq=K, n_beta=1)
+            k_ms, _ = timed(lambda: step(c), max(args.steps, 5), 3, trace=False)
+            k_bytes = elements * call_bytes_per_elem(c, 1)
+            rows_out.append(dict(n_dq=K, n_beta=1, ms_per_step=k_ms, value=world * 2.0 * elements / (k_ms * 1e-3) / 1e9,
+                                 unit="GB/s", achieved_gbs=k_bytes / (k_ms * 1e-3) / 1e9,
+                                 frac_of_measured_hbm=k_bytes / (k_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]))
+        extra["sweep_dq"] = rows_out
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region
     import ctypes
@@ -795,6 +805,7 @@ def main():
                     help="weighted: the column-weighted objective through soar_quantize_weighted")
     ap.add_argument("--row-sharded", action="store_true",
                     help="split the workload's largest tensor by rows over the ranks (strong scaling)")
+    ap.add_argument("--sweep-dq", default="", help="comma-separated counts of E4M3 codes per block to time with beta = 1")
     ap.add_argument("--no-batch", action="store_true", help="one soar_quantize call per tensor instead of soar_quantize_batch")
     ap.add_argument("--graph", action="store_true", help="replay each step from a CUDA graph (no per-kernel trace)")
     ap.add_argument("--no-e2e", action="store_true")

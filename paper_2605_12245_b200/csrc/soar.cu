@@ -924,9 +924,15 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
       block_sums(blk, fx, r, best0, best1, bestA, bestB, wide);
       const double A2 = -2.0 * bestA;
       best = sd0 * fma(sd0, bestB, A2);               // block error minus sum W^2
-      if (n_dq == 2) {
+      if (n_dq >= 2) {
         const double g1 = sd1 * fma(sd1, bestB, A2);
         if (g1 < best) { best = g1; best_d = dc1; }
+      }
+      for (int d = d_lo + 2; d <= d_hi; ++d) {        // wider code windows (App. B.3 with more than two codes)
+        const int dc = clip_code(d);
+        const double sd = alpha_d * static_cast<double>(e4m3_value(dc));
+        const double g = sd * fma(sd, bestB, A2);
+        if (g < best) { best = g; best_d = dc; }
       }
     } else {
       // Eq. 8 over beta ascending, then scale code ascending; strict '<' keeps the first
@@ -1840,7 +1846,9 @@ int run_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void*
       cudaMemsetAsync(headers, 0, static_cast<size_t>(n) * kWsFixedBytes, st) != cudaSuccess)
     return SOAR_ERR_CUDA;
 
-  const bool single = cfg->n_beta == 1 && cfg->n_dq <= 2;
+  // one quantization scale per block: the codes are made once (any number of E4M3 codes scored on them;
+  // the coupled arm, where every code rounds the block anew, only with at most two)
+  const bool single = cfg->n_beta == 1 && (cfg->n_dq <= 2 || !(cfg->flags & SOAR_FLAG_COUPLED_SCALE));
   const bool may_stop = cfg->early_stop_rel > 0.0f;
   for (int first = 0; first < n; first += kMaxBatch) {
     Batch bt;
