@@ -826,8 +826,9 @@ __device__ __forceinline__ int clip_code(int d) { return max(1, min(0x7E, d)); }
 // be the one returned); the per-block sums are kept when `keep` is set (another iteration
 // may follow).  Modes 1 and 2 are the shapes with one quantization scale per E4M3 code and at most two
 // codes, whose passes are bound by HBM rather than by the candidate loop.
-template <int kMode>   // 0: candidate grid; 1: one candidate scale (beta = 1); 2: the same with the coupled scale
-__global__ void __launch_bounds__(kThreads, kMode == 1 ? 3 : 2)
+template <int kMode>   // 0: candidate grid; 1: one candidate scale (beta = 1), at most two codes; 2: the same with the
+                       // coupled scale; 3: one candidate scale, any number of codes
+__global__ void __launch_bounds__(kThreads, (kMode == 1 || kMode == 3) ? 3 : 2)
 iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, int keep) {
   constexpr bool kSingle = kMode != 0;
   __shared__ RingWithState ring;
@@ -928,11 +929,13 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
         const double g1 = sd1 * fma(sd1, bestB, A2);
         if (g1 < best) { best = g1; best_d = dc1; }
       }
-      for (int d = d_lo + 2; d <= d_hi; ++d) {        // wider code windows (App. B.3 with more than two codes)
-        const int dc = clip_code(d);
-        const double sd = alpha_d * static_cast<double>(e4m3_value(dc));
-        const double g = sd * fma(sd, bestB, A2);
-        if (g < best) { best = g; best_d = dc; }
+      if (kMode == 3) {
+        for (int d = d_lo + 2; d <= d_hi; ++d) {      // wider code windows (App. B.3 with more than two codes)
+          const int dc = clip_code(d);
+          const double sd = alpha_d * static_cast<double>(e4m3_value(dc));
+          const double g = sd * fma(sd, bestB, A2);
+          if (g < best) { best = g; best_d = dc; }
+        }
       }
     } else {
       // Eq. 8 over beta ascending, then scale code ascending; strict '<' keeps the first
@@ -1905,10 +1908,11 @@ int run_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void*
                                                                                       cfg->max_iters == 0 ? 1 : 0);
     }
     if (stages & kStageIterate) {
-      const int mode = !single ? 0 : ((cfg->flags & SOAR_FLAG_COUPLED_SCALE) ? 2 : 1);
+      const int mode = !single ? 0 : ((cfg->flags & SOAR_FLAG_COUPLED_SCALE) ? 2 : (cfg->n_dq <= 2 ? 1 : 3));
       const unsigned int g_it = mode == 0   ? persistent_grid(iterate_kernel<0>, tiles, kThreads)
                                 : mode == 1 ? persistent_grid(iterate_kernel<1>, tiles, kThreads)
-                                            : persistent_grid(iterate_kernel<2>, tiles, kThreads);
+                                : mode == 2 ? persistent_grid(iterate_kernel<2>, tiles, kThreads)
+                                            : persistent_grid(iterate_kernel<3>, tiles, kThreads);
       for (int t = t_lo; t < t_hi; ++t) {
         const int reverse = t & 1;
         // with the early stop on, any iteration may turn out to be the last one
@@ -1917,7 +1921,8 @@ int run_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void*
         ScopedLaunch sl(K_ITERATE, st);
         if (mode == 0) iterate_kernel<0><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
         else if (mode == 1) iterate_kernel<1><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
-        else iterate_kernel<2><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
+        else if (mode == 2) iterate_kernel<2><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
+        else iterate_kernel<3><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
       }
     }
     if (!(stages & kStageFinalize)) continue;
