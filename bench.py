@@ -450,7 +450,7 @@ def run_ours(args):
     ctypes_sizeof_result = ctypes.sizeof(api.SoarResult)
     e2e = None
     if not args.no_e2e and args.workload != "config3":      # config 3 would pin 18 GB of host memory
-        pipe = api.HostPipeline([(s.rows, s.cols) for s in wl.tensors], cfg, depth=4)
+        pipe = api.HostPipeline([(s.rows, s.cols) for s in wl.tensors], cfg, depth=6)
         hosts = []
         for h, spec in zip(host_w, wl.tensors):
             hb = api.alloc_host_buffers(spec.rows, spec.cols, cfg)
@@ -474,7 +474,7 @@ def run_ours(args):
         e2e = dict(value=world * 2.0 * elements / dt / 1e9, unit="GB/s", ms_per_step=dt * 1e3,
                    h2d_bytes_per_step=2 * elements,
                    d2h_bytes_per_step=elements // 2 + elements // 16 + len(wl.tensors) * (4 + ctypes_sizeof_result),
-                   api="HostPipeline: pinned host buffers, copy-in / soar_quantize / copy-out on three streams, 4 slots")
+                   api="HostPipeline: pinned host buffers, copy-in / soar_quantize / copy-out on three streams, 6 slots")
 
     # ---- the oracle on the host cores, bounded sample (rank 0, single GPU only)
     cpu = None

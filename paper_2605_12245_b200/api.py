@@ -428,12 +428,15 @@ class HostPipeline:
         self.h2d, self.compute, self.d2h = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
         for sl in self.slots:
             sl["stored"].record(self.d2h)
+        self._next = 0      # slots are taken in turn across calls, so a new list starts on the slot freed longest ago
 
     def run(self, hosts) -> None:
         """Enqueue the whole list (``HostBuffers`` each); results are in the host buffers once
-        ``synchronize()`` returns."""
-        for i, hb in enumerate(hosts):
-            sl = self.slots[i % len(self.slots)]
+        ``synchronize()`` returns.  Calls may follow one another without a synchronize in
+        between: the copies of the next list then overlap the work on the previous one."""
+        for hb in hosts:
+            sl = self.slots[self._next % len(self.slots)]
+            self._next += 1
             rows, cols = hb.W.shape
             n = rows * cols
             big = sl["out"]
