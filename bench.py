@@ -633,21 +633,18 @@ def run_weighted(args):
                     weighted_rel_error_of_max_based_start=results[0].sse_init / results[0].sumsq)
         del plain
 
-    # ---- end to end: pinned host buffers in and out, copies inside the timed region (one stream)
+    # ---- end to end: pinned host buffers in and out, copies inside the timed region
     e2e = None
     if not args.no_e2e and args.workload != "config3":
-        pin = lambda t: torch.empty_like(t, device="cpu").pin_memory()  # noqa: E731
-        hin = [pin(h) for h in host_w]
-        for a, b in zip(hin, host_w):
-            a.copy_(b)
-        hout = [(pin(o.packed), pin(o.scales), pin(o.alpha), pin(o.result)) for o in outs]
+        pipe = api.HostPipeline([(s.rows, s.cols) for s in wl.tensors], cfg, depth=6, weighted=True)
+        hosts = []
+        for hsrc, spec in zip(host_w, wl.tensors):
+            hb = api.alloc_host_buffers(spec.rows, spec.cols, cfg)
+            hb.W.copy_(hsrc)
+            hosts.append(hb)
 
         def e2e_step():
-            for W, hsrc, h, o, ho in zip(dev_w, hin, dev_h, outs, hout):
-                W.copy_(hsrc, non_blocking=True)
-                api.soar_quantize_weighted(W, h, cfg, o, stream)
-                for dst, src in zip(ho, (o.packed, o.scales, o.alpha, o.result)):
-                    dst.copy_(src, non_blocking=True)
+            pipe.run(hosts, dev_h)
 
         for _ in range(2):
             e2e_step()
@@ -661,8 +658,8 @@ def run_weighted(args):
         e2e = dict(value=world * 2.0 * elements / dt / 1e9, unit="GB/s", ms_per_step=dt * 1e3,
                    h2d_bytes_per_step=2 * elements,
                    d2h_bytes_per_step=elements // 2 + elements // 16 + len(wl.tensors) * (4 + ctypes.sizeof(api.SoarResult)),
-                   api="pinned host buffers; copy-in, soar_quantize_weighted and copy-out in order on one stream "
-                       "(the column weights stay on the device)")
+                   api="HostPipeline: pinned host buffers, copy-in / soar_quantize_weighted / copy-out on three streams, "
+                       "6 slots (the column weights stay on the device)")
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:

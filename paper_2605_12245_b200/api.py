@@ -414,27 +414,33 @@ class HostPipeline:
     """Quantizes matrices that live in pinned host memory with the three legs overlapped:
     host-to-device copies on one stream, ``soar_quantize`` on a second, device-to-host copies of
     the results on a third, chained by events over ``depth`` device staging slots sized for the
-    largest matrix.  Stream plumbing only; the work is ``soar_quantize``."""
+    largest matrix.  Stream plumbing only; the work is ``soar_quantize`` (``soar_quantize_weighted``
+    when column weights are given)."""
 
-    def __init__(self, shapes, cfg: SoarCfg, depth: int = 3, device="cuda"):
+    def __init__(self, shapes, cfg: SoarCfg, depth: int = 3, device="cuda", weighted: bool = False):
         self.cfg = cfg
+        self.weighted = weighted
         rows, cols = max(shapes, key=lambda rc: rc[0] * rc[1])
         self.slots = []
         for _ in range(depth):
             self.slots.append(dict(
                 W=torch.empty(rows * cols, dtype=torch.bfloat16, device=device),
-                out=alloc_buffers(rows, cols, cfg, device),
+                out=alloc_buffers(rows, cols, cfg, device, weighted=weighted),
                 loaded=torch.cuda.Event(), computed=torch.cuda.Event(), stored=torch.cuda.Event()))
         self.h2d, self.compute, self.d2h = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
         for sl in self.slots:
             sl["stored"].record(self.d2h)
         self._next = 0      # slots are taken in turn across calls, so a new list starts on the slot freed longest ago
 
-    def run(self, hosts) -> None:
+    def run(self, hosts, col_weights=None) -> None:
         """Enqueue the whole list (``HostBuffers`` each); results are in the host buffers once
         ``synchronize()`` returns.  Calls may follow one another without a synchronize in
-        between: the copies of the next list then overlap the work on the previous one."""
-        for hb in hosts:
+        between: the copies of the next list then overlap the work on the previous one.
+        ``col_weights``: one float32 CUDA vector per matrix for the weighted objective (the
+        pipeline must have been built with ``weighted=True``)."""
+        if col_weights is not None and not self.weighted:
+            raise SoarError("this pipeline's workspaces are not sized for the weighted objective")
+        for k, hb in enumerate(hosts):
             sl = self.slots[self._next % len(self.slots)]
             self._next += 1
             rows, cols = hb.W.shape
@@ -451,7 +457,10 @@ class HostPipeline:
                 W.copy_(hb.W, non_blocking=True)
                 sl["loaded"].record(self.h2d)
             self.compute.wait_event(sl["loaded"])
-            soar_quantize(W, self.cfg, view, self.compute)
+            if col_weights is None:
+                soar_quantize(W, self.cfg, view, self.compute)
+            else:
+                soar_quantize_weighted(W, col_weights[k], self.cfg, view, self.compute)
             sl["computed"].record(self.compute)
             self.d2h.wait_event(sl["computed"])
             with torch.cuda.stream(self.d2h):

@@ -157,3 +157,28 @@ def test_full_size_tensors_under_the_weighted_objective(tensor):
     assert gpu.result.sumsq == pytest.approx(ref.sumsq, rel=1e-9)
     e = api.soar_dequant_error_weighted(W, hw, gpu.buffers.packed, gpu.buffers.scales, gpu.buffers.alpha).cpu().numpy()
     assert e[0] == pytest.approx(gpu.result.sse, rel=1e-9)
+
+
+def test_host_pipeline_with_column_weights_returns_what_direct_calls_return():
+    cfg = api.soar_default_cfg(api.PRESET_PAPER, max_iters=2, n_beta=11)
+    shapes = [(64, 256), (130, 1040), (16, 64), (257, 512), (64, 256)]
+    ws = [WL.small_case(r, c, 40 + i) for i, (r, c) in enumerate(shapes)]
+    hs = [torch.from_numpy(WL.column_weights(c, 40 + i)).cuda() for i, (r, c) in enumerate(shapes)]
+    pipe = api.HostPipeline(shapes, cfg, depth=2, weighted=True)
+    hosts = []
+    for w, (r, c) in zip(ws, shapes):
+        hb = api.alloc_host_buffers(r, c, cfg)
+        hb.W.copy_(torch.from_numpy(w.view(np.int16)).view(torch.bfloat16))
+        hosts.append(hb)
+    pipe.run(hosts, hs)
+    pipe.run(hosts, hs)          # a second list right behind the first
+    pipe.synchronize()
+    for w, h, hb in zip(ws, hs, hosts):
+        direct = api.soar_quantize_weighted(P.to_device(w), h, cfg)
+        torch.cuda.synchronize()
+        assert np.array_equal(hb.packed.numpy(), direct.packed.cpu().numpy())
+        assert np.array_equal(hb.scales.numpy(), direct.scales.cpu().numpy())
+        assert float(hb.alpha[0]) == float(direct.alpha.cpu()[0])
+        assert hb.read_result().iters_run == direct.read_result().iters_run
+    with pytest.raises(api.SoarError):
+        api.HostPipeline(shapes, cfg, depth=2).run(hosts, hs)
