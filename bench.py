@@ -164,6 +164,26 @@ def call_bytes_per_elem(cfg, iters_run: int) -> float:
             + sum(kernel_bytes_per_elem("iterate_kernel", cfg, t) for t in range(iters_run)))
 
 
+def oracle_one_thread(R, w, rcfg, h=None):
+    """The oracle on one host thread (a per-core figure): the OpenMP runtime's own switch, called from
+    here; the oracle is run as it stands.  Returns None when the runtime cannot be reached."""
+    import ctypes
+    try:
+        gomp = ctypes.CDLL("libgomp.so.1")
+        before = R.num_threads()
+        gomp.omp_set_num_threads(1)
+    except (OSError, AttributeError):
+        return None
+    try:
+        t0 = time.perf_counter()
+        ref = R.quantize(w, rcfg, h=h)
+        dt = time.perf_counter() - t0
+    finally:
+        gomp.omp_set_num_threads(before)
+    return dict(value=2.0 * w.size / dt / 1e9, unit="GB/s", elements_per_s=w.size / dt,
+                sample=f"{w.shape[0]} rows x {w.shape[1]} cols, {ref.iters_run} iterations, {dt:.1f} s")
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
 
@@ -488,7 +508,8 @@ def run_ours(args):
         dt = time.perf_counter() - t0
         cpu = dict(value=2.0 * w.size / dt / 1e9, unit="GB/s", cores=R.num_threads(), kind="oracle",
                    sample=f"first {rows} rows x {spec.cols} cols of tensor '{spec.name}', {ref.iters_run} iterations, {dt:.1f} s",
-                   elements_per_s=w.size / dt)
+                   elements_per_s=w.size / dt,
+                   one_thread=oracle_one_thread(R, w[: max(1, rows // 16)], ref_cfg_of(R, cfg)))
 
     if rank == 0:
         line = dict(
