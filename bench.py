@@ -693,7 +693,8 @@ def run_weighted(args):
         dt = time.perf_counter() - t0
         cpu = dict(value=2.0 * w.size / dt / 1e9, unit="GB/s", cores=R.num_threads(), kind="oracle",
                    sample=f"first {rows} rows x {spec.cols} cols of tensor '{spec.name}', {ref.iters_run} iterations, {dt:.1f} s",
-                   elements_per_s=w.size / dt)
+                   elements_per_s=w.size / dt,
+                   one_thread=oracle_one_thread(R, w[: max(1, rows // 16)], ref_cfg_of(R, cfg), h=host_h[0].numpy()))
 
     if rank == 0:
         line = dict(
