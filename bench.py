@@ -349,16 +349,19 @@ def run_ours(args):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         if trace:
             api.soar_trace_begin()
+        t0 = time.perf_counter()
         e0.record(stream)
         for _ in range(steps):
             fn()
         e1.record(stream)
         torch.cuda.synchronize()
+        host_ms.append((time.perf_counter() - t0) * 1e3 / steps)      # host clock, final synchronize included
         tr = api.soar_trace_end() if trace else {}
         barrier()
         ms = SH.max_over_ranks(e0.elapsed_time(e1) / steps, "cuda")
         return ms, tr
 
+    host_ms = []
     sampler = ClockSampler(local)
     sampler.start()
     # headline: K steps with nothing between the kernels; then the same K steps again with an
@@ -521,7 +524,7 @@ def run_ours(args):
                         elements=elements, iters_run=iters,
                         l2="inputs (%.2f GB per step) exceed the 126 MB L2" % (2 * elements / 1e9),
                         parallelism=f"{world} rank(s), one layer of these shapes each, no collective"),
-            elements_per_s=world * elements / (ms * 1e-3),
+            elements_per_s=world * elements / (ms * 1e-3), host_clock_ms_per_step=host_ms[0],
             hbm_frac_end_to_end_of_measured=value / peaks["hbm_gbs"],
             traced_ms_per_step=traced_ms, cuda_graph=bool(args.graph), batched=not args.no_batch, roofline=roofline, kernels=kernels, cpu_baseline=cpu, e2e=e2e, gpu_launches=launches,
             clocks=clocks, **extra)
