@@ -182,3 +182,39 @@ def test_host_pipeline_with_column_weights_returns_what_direct_calls_return():
         assert hb.read_result().iters_run == direct.read_result().iters_run
     with pytest.raises(api.SoarError):
         api.HostPipeline(shapes, cfg, depth=2).run(hosts, hs)
+
+
+def test_the_weighted_call_and_the_staged_calls_replay_from_a_cuda_graph():
+    """Neither entry point synchronizes or allocates: both can be captured once and replayed."""
+    w = WL.small_case(128, 2048, 83, outlier_cols_frac=0.002, outlier_scale=20.0)
+    h = WL.column_weights(2048, 83)
+    cfg, ref_cfg = P.cfg_pair()
+    W = P.to_device(w)
+    hw = torch.from_numpy(h).cuda()
+    side = torch.cuda.Stream()
+    # weighted objective
+    out = api.alloc_buffers(*w.shape, cfg, weighted=True)
+    api.soar_quantize_weighted(W, hw, cfg, out, side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        api.soar_quantize_weighted(W, hw, cfg, out, side)
+    out.packed.zero_(); out.scales.zero_(); out.alpha.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    gpu = P.GpuOut(out.packed.cpu().numpy(), out.scales.cpu().numpy(), float(out.alpha.cpu()[0]),
+                   out.read_result(), out)
+    P.assert_parity(gpu, R.quantize(w, ref_cfg, h=h))
+    # the stages of the plain call, one by one
+    from paper_2605_12245_b200 import row_sharded as RS
+    out2 = api.alloc_buffers(*w.shape, cfg)
+    g2 = torch.cuda.CUDAGraph()
+    torch.cuda.synchronize()
+    with torch.cuda.graph(g2, stream=side):
+        for stage in RS.stages(cfg.max_iters):
+            api.soar_quantize_stage([W], cfg, [out2], out2.workspace, stage, side)
+    g2.replay()
+    torch.cuda.synchronize()
+    gpu2 = P.GpuOut(out2.packed.cpu().numpy(), out2.scales.cpu().numpy(), float(out2.alpha.cpu()[0]),
+                    out2.read_result(), out2)
+    P.assert_parity(gpu2, R.quantize(w, ref_cfg))
