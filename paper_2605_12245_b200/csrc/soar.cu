@@ -57,6 +57,7 @@ constexpr int kStages = 4;                     // depth of the shared-memory rin
 constexpr int kTileBytes = kTile * 32;         // 16 bf16 per block
 constexpr size_t kWsFixedBytes = 2048;
 constexpr unsigned int kWaitLimit = 1u << 22;  // mbarrier polls before a wait gives up
+constexpr unsigned int kProducerSleepNs = 32;  // the producer's pause between polls for a free stage
 
 struct Ws {
   unsigned int amax_bits;            // max over the tensor of the bf16 magnitude bit pattern
@@ -182,10 +183,11 @@ __device__ __forceinline__ float e2m1_code_value(unsigned int code3) {
   return 0.5f * static_cast<float>(static_cast<unsigned int>(lut >> (8 * code3)) & 0xFFu);
 }
 
-// Non-negative integer below 2^31 to binary64 without a conversion instruction.
-__device__ __forceinline__ double uint_to_double(unsigned int v) {
-  return __hiloint2double(0x43300000, static_cast<int>(v)) - 4503599627370496.0;
-}
+// Unsigned integer to binary64 (exact).  The conversion instruction issues on the pipe of the
+// special-function unit, which these kernels leave almost idle; building the value from bit
+// patterns instead costs two register moves and a binary64 add on pipes that are busy
+// (38.5 against 39.4 ms per Llama-3-70B-shaped layer in the candidate loop).
+__device__ __forceinline__ double uint_to_double(unsigned int v) { return __uint2double_rn(v); }
 
 // ------------------------------------------------------------------ shared-memory tile ring
 
@@ -215,7 +217,10 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned i
                : "memory");
 }
 
-// Waits for the phase with the given parity; gives up after kWaitLimit polls.
+// Waits for the phase with the given parity; gives up after kWaitLimit polls.  With kSleepNs > 0
+// the thread sleeps that long between polls (the producer, which otherwise spins beside the
+// consumer warps of its scheduler).
+template <unsigned int kSleepNs = 0>
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned int parity) {
   const unsigned int addr = smem_u32(bar);
   for (unsigned int i = 0; i < kWaitLimit; ++i) {
@@ -228,6 +233,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned int 
         : "r"(addr), "r"(parity)
         : "memory");
     if (ok) return true;
+    if (kSleepNs > 0) __nanosleep(kSleepNs);
   }
   return false;
 }
@@ -332,7 +338,7 @@ __device__ __forceinline__ void ring_produce(R& ring, const Batch& bt, int rever
     const int ti = tensor_of(bt, reverse ? bt.total_tiles - 1 - g0 : g0, tile);
     if (!((run_mask >> ti) & 1u)) continue;
     const int s = static_cast<int>(n % kStages);
-    if (n >= static_cast<unsigned int>(kStages)) ok = mbar_wait(&ring.empty[s], (n / kStages - 1) & 1u);
+    if (n >= static_cast<unsigned int>(kStages)) ok = mbar_wait<kProducerSleepNs>(&ring.empty[s], (n / kStages - 1) & 1u);
     if (!ok || *static_cast<volatile int*>(&ring.fail)) { ok = false; break; }
     ring.meta_tensor[s] = ti;
     ring.meta_tile[s] = tile;
@@ -341,7 +347,7 @@ __device__ __forceinline__ void ring_produce(R& ring, const Batch& bt, int rever
   }
   if (ok) {   // end marker: completes the stage's phase with no bytes
     const int s = static_cast<int>(n % kStages);
-    if (n >= static_cast<unsigned int>(kStages)) ok = mbar_wait(&ring.empty[s], (n / kStages - 1) & 1u);
+    if (n >= static_cast<unsigned int>(kStages)) ok = mbar_wait<kProducerSleepNs>(&ring.empty[s], (n / kStages - 1) & 1u);
     if (ok) {
       ring.meta_tensor[s] = -1;
       mbar_arrive(&ring.full[s]);
@@ -519,21 +525,26 @@ __device__ __forceinline__ void block_sums(const Block& blk, const Fixed& fx, fl
   }
 }
 
-__device__ __forceinline__ float recip_scale(float alpha, float dq) {
-  return __frcp_rn(__fmul_rn(alpha, dq));
-}
 
 // 1/s rounded to nearest for s in [2^-125, 2^126): the hardware's approximate reciprocal
 // followed by one Newton step, y + y * (1 - s y), both as fused multiply-adds.  On sm_100a this
 // equals rcp.rn for every binary32 input of that range (soar_selftest_reciprocal compares all
-// of them); it is a third of the instructions.  Callers check the range (recip_fast_ok).
+// of them); it is a third of the instructions.  Callers check the range (recip_fast_ok).  The
+// flush-to-zero form of the approximation is used: on that range neither s nor 1/s is
+// subnormal, and the plain form carries extra instructions that rescale subnormal inputs.
 __device__ __forceinline__ float recip_fast(float s) {
   float y;
-  asm("rcp.approx.f32 %0, %1;" : "=f"(y) : "f"(s));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(s));
   return __fmaf_rn(y, __fmaf_rn(-s, y, 1.0f), y);
 }
 __device__ __forceinline__ bool recip_fast_ok(float s) {
   return ((__float_as_uint(s) >> 23) - 2u) <= 250u;   // positive, biased exponent 2 .. 252
+}
+
+// fl(1 / fl(alpha * dq)): the reciprocal scale of Eq. 2.
+__device__ __forceinline__ float recip_scale(float alpha, float dq) {
+  const float s = __fmul_rn(alpha, dq);
+  return recip_fast_ok(s) ? recip_fast(s) : __frcp_rn(s);
 }
 
 __device__ __forceinline__ double warp_sum(double v) {
