@@ -189,6 +189,12 @@ __device__ __forceinline__ float e2m1_code_value(unsigned int code3) {
 // (38.5 against 39.4 ms per Llama-3-70B-shaped layer in the candidate loop).
 __device__ __forceinline__ double uint_to_double(unsigned int v) { return __uint2double_rn(v); }
 
+// The same from bit patterns (2^52 + v, minus 2^52), for the places that convert sixteen values
+// per block at once: there the conversion pipe would be the busy one.
+__device__ __forceinline__ double uint_to_double_bits(unsigned int v) {
+  return __hiloint2double(0x43300000, static_cast<int>(v)) - 4503599627370496.0;
+}
+
 // ------------------------------------------------------------------ shared-memory tile ring
 
 __device__ __forceinline__ unsigned int smem_u32(const void* p) {
@@ -1232,7 +1238,7 @@ __device__ __forceinline__ void weighted_sums(const double (&hw)[16], const doub
   double a = 0.0, b = 0.0;
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
-    const double dm = uint_to_double((t[j >> 2] >> (8 * (j & 3))) & 0xFFu);   // 2 m_j
+    const double dm = uint_to_double_bits((t[j >> 2] >> (8 * (j & 3))) & 0xFFu);   // 2 m_j
     a = fma(hw[j], dm, a);
     b = fma(hd[j], dm * dm, b);
   }
@@ -1251,7 +1257,7 @@ __device__ __forceinline__ void weighted_sums_split(const double (&hw)[16], cons
   double a[2] = {0.0, 0.0}, b[2] = {0.0, 0.0};
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
-    const double dm = uint_to_double((t[j >> 2] >> (8 * (j & 3))) & 0xFFu);
+    const double dm = uint_to_double_bits((t[j >> 2] >> (8 * (j & 3))) & 0xFFu);
     a[j & 1] = fma(hw[j], dm, a[j & 1]);
     b[j & 1] = fma(hd[j], dm * dm, b[j & 1]);
   }

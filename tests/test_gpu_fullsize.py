@@ -35,6 +35,36 @@ def test_config4_whole_tensors_paper_preset(tensor):
     print(wl.tensors[tensor].name, rep)
 
 
+def test_config2_whole_tensors_paper_preset():
+    """The Qwen3-8B-shaped layer (outlier input columns x20): down (4096 x 12288, long rows) and v (1024 x 4096)."""
+    wl = WL.config2()
+    cfg, ref_cfg = P.cfg_pair()
+    for tensor in (6, 2):
+        w = WL.generate(wl, tensor)
+        rep = P.assert_parity(P.run_gpu(w, cfg), R.quantize(w, ref_cfg))
+        print(wl.tensors[tensor].name, rep)
+
+
+def test_config3_last_layer_tensor_paper_preset():
+    """Layer 35 of the 36-layer model (its own seed): o (4096 x 4096)."""
+    wl = WL.config3_layer(35)
+    w = WL.generate(wl, 3)
+    cfg, ref_cfg = P.cfg_pair()
+    rep = P.assert_parity(P.run_gpu(w, cfg), R.quantize(w, ref_cfg))
+    print(wl.name, wl.tensors[3].name, rep)
+
+
+def test_config5_distribution_candidate_sweep_points():
+    """Config 5's Gaussian / Student-t(2) mix at the sweep's candidate counts, on the first 1024 rows of the
+    28672 x 8192 matrix (the whole matrix takes the oracle minutes per point)."""
+    w = WL.generate(WL.config5(), 0, 0, 1024)
+    for pairs in (1, 4, 8, 16, 32):
+        n_dq = min(2, pairs)
+        cfg, ref_cfg = P.cfg_pair(max_iters=1, early_stop_rel=0.0, n_dq=n_dq, n_beta=pairs // n_dq)
+        rep = P.assert_parity(P.run_gpu(w, cfg), R.quantize(w, ref_cfg))
+        print("config5 rows 0..1023, pairs", pairs, rep)
+
+
 def test_config4_whole_tensor_coupled_pair_preset():
     """q (8192 x 8192) with two coupled candidates per block: several HBM-bound iterations."""
     wl = WL.config4()
