@@ -58,6 +58,7 @@ constexpr int kTileBytes = kTile * 32;         // 16 bf16 per block
 constexpr size_t kWsFixedBytes = 2048;
 constexpr unsigned int kWaitLimit = 1u << 22;  // mbarrier polls before a wait gives up
 constexpr unsigned int kProducerSleepNs = 32;  // the producer's pause between polls for a free stage
+constexpr int kBracketMinBeta = 6;             // grids below this many multipliers are cheaper visited in full
 
 struct Ws {
   unsigned int amax_bits;            // max over the tensor of the bf16 magnitude bit pattern
@@ -837,17 +838,96 @@ __device__ __forceinline__ float block_center(const uint2 st, float alpha, int n
 
 __device__ __forceinline__ int clip_code(int d) { return max(1, min(0x7E, d)); }
 
+// fl(alpha * fl(center * beta)): the divisor of Eq. 2 for one multiplier of the App. B.3 grid.
+__device__ __forceinline__ float grid_divisor(float alpha, float center, float beta) {
+  return __fmul_rn(alpha, __fmul_rn(center, beta));
+}
+
+// Which multipliers of the App. B.3 grid can win Eq. 8 for one E4M3 code, without visiting the grid.
+//
+// For a fixed dequantization scale sd = alpha * value(code) the error of element j,
+// (a_j - m sd)^2, is convex in its code value m with its minimum at a_j / sd.  The codes
+// m_j(k) = E2M1(fl(a_j * fl(1 / s_k))), s_k = grid_divisor(beta_k), never rise with k, because every
+// step of that binary32 chain is monotone.  While s_k <= sd (1 - 2^-23) every fl(a_j / s_k) is at
+// least a_j / sd (two roundings of 2^-24 each), so every code is at or above the nearest one
+// to a_j / sd and each element's error can only fall as k grows; once s_k >= sd (1 + 2^-22) every code is at or
+// below it and the error can only rise.  The block error of Eq. 8 is therefore smallest at the
+// last multiplier of the first kind, at the first of the second kind, or at one in between
+// (the band is 2^-21 wide against a grid step of a hundredth: almost always empty).  Returns that
+// range [ka, kb]; two multipliers in the typical case, where the grid has 101.
+//
+// Equal errors.  Different codes of an element cost the same only when a_j / sd is exactly a
+// rounding midpoint, which needs sd, and with it alpha, to have at most eight significant bits;
+// callers send such tensors through the whole grid, so that the first minimum in grid order is
+// kept as Algorithm 1's strict comparison keeps it.
+__device__ __forceinline__ void winning_range(const float* s_beta, int n_beta, float k_scale, float k_off,
+                                              float alpha, float center, float dv, double sd, int& ka, int& kb) {
+  const float lo = __double2float_rd(sd * (1.0 - 0x1p-23));
+  const float hi = __double2float_ru(sd * (1.0 + 0x1p-22));
+  // start from the multiplier nearest dv / center; the two loops below make it exact
+  int k = __float2int_rn(__fmaf_rn(__fdividef(dv, center), k_scale, k_off));
+  k = max(0, min(n_beta - 1, k));
+  while (k >= 0 && grid_divisor(alpha, center, s_beta[k]) > lo) --k;
+  while (k + 1 < n_beta && grid_divisor(alpha, center, s_beta[k + 1]) <= lo) ++k;
+  ka = max(k, 0);
+  kb = k + 1;
+  while (kb < n_beta && grid_divisor(alpha, center, s_beta[kb]) < hi) ++kb;
+  kb = min(kb, n_beta - 1);
+}
+
+// True when different codes of an element can cost exactly the same under this alpha (see
+// winning_range): alpha has at most eight significant bits.
+__device__ __forceinline__ bool alpha_allows_exact_ties(float alpha) {
+  return (__float_as_uint(alpha) & 0xFFFFu) == 0u;
+}
+
+// A block's winner of Eq. 8: error minus sum W^2, its sums, codes (signs included) and E4M3 code.
+struct Winner {
+  double g, A, B;
+  unsigned int c0, c1;
+  int d, k;
+};
+
+// Eq. 8 over the whole grid, beta ascending, then scale code ascending; strict '<' keeps the first
+// minimum.  Out of line: it serves only tensors that can have exactly equal candidates.
+__device__ __noinline__ void whole_grid_search(const Block& blk, const Fixed& fx, float alpha, float center,
+                                               const float* s_beta, int n_beta, int d_lo, int nd, Winner& w,
+                                               unsigned int& wide) {
+  const double alpha_d = static_cast<double>(alpha);
+  w.g = __longlong_as_double(0x7FF0000000000000ll);
+  w.d = clip_code(d_lo);
+  w.k = 0;
+  w.A = w.B = 0.0;
+  w.c0 = w.c1 = 0u;
+  for (int k = 0; k < n_beta; ++k) {
+    const float r = recip_scale(alpha, __fmul_rn(center, s_beta[k]));
+    unsigned int c0, c1;
+    double A, B;
+    round_block(blk, r, c0, c1);
+    block_sums(blk, fx, r, c0, c1, A, B, wide);
+    for (int d = 0; d < nd; ++d) {
+      const int dc = clip_code(d_lo + d);
+      const double sd = alpha_d * static_cast<double>(e4m3_value(dc));
+      const double g = sd * fma(sd, B, -2.0 * A);
+      if (g < w.g) { w.g = g; w.A = A; w.B = B; w.c0 = c0; w.c1 = c1; w.d = dc; w.k = k; }
+    }
+  }
+}
+
 // One iteration t of Algorithm 1 for every block: Eq. 5 (from stage-t sums), Eq. 6,
 // App. B.3 candidate sets, Eq. 8 search, winner stored, stage-(t+1) sums accumulated.
 // Codes and scale bytes are written when `emit` is set (the state after this iteration may
 // be the one returned); the per-block sums are kept when `keep` is set (another iteration
 // may follow).  Modes 1 and 2 are the shapes with one quantization scale per E4M3 code and at most two
-// codes, whose passes are bound by HBM rather than by the candidate loop.
-template <int kMode>   // 0: candidate grid; 1: one candidate scale (beta = 1), at most two codes; 2: the same with the
-                       // coupled scale; 3: one candidate scale, any number of codes
+// codes, whose passes are bound by HBM rather than by the candidate loop.  Mode 4 is the candidate
+// grid of App. B.3 searched through winning_range: per E4M3 code only the multipliers that can win
+// are rounded and scored, which gives the winner of the whole grid.
+template <int kMode>   // 0: candidate grid, every multiplier visited; 1: one candidate scale (beta = 1), at most two
+                       // codes; 2: the same with the coupled scale; 3: one candidate scale, any number of codes;
+                       // 4: candidate grid, only the multipliers that can win
 __global__ void __launch_bounds__(kThreads, (kMode == 1 || kMode == 3) ? 3 : 2)
 iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, int keep) {
-  constexpr bool kSingle = kMode != 0;
+  constexpr bool kSingle = kMode == 1 || kMode == 2 || kMode == 3;
   __shared__ RingWithState ring;
   __shared__ Slots<3> slots;
   __shared__ float s_beta[kSingle ? 1 : SOAR_MAX_BETA];
@@ -877,6 +957,10 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
   }
   float alpha = 1.0f;
   double alpha_d = 1.0;
+  bool whole_grid = false;           // mode 4: the current tensor's alpha allows exactly equal candidates
+  // mode 4: multiplier index of a scale ratio, k = (ratio - 1) * 100 / step + n_beta / 2
+  const float k_scale = 100.0f / static_cast<float>(max(bt.t[0].beta_step_pct, 1));
+  const float k_off = static_cast<float>(n_beta / 2) - k_scale;
 
   double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum of stage t+1
   unsigned int wide = 0, unused_zeros = 0;
@@ -900,11 +984,12 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
       cur = ti;
       alpha = s_alpha[ti];
       alpha_d = static_cast<double>(alpha);
-      if (kSingle) p = tensor_view(bt.t[ti]);
+      whole_grid = alpha_allows_exact_ties(alpha);
+      if (kMode != 0) p = tensor_view(bt.t[ti]);
     }
     // the long candidate loop does better re-reading these from the parameter block per tile than
     // carrying them in registers
-    if (!kSingle) p = tensor_view(bt.t[ti]);
+    if (kMode == 0) p = tensor_view(bt.t[ti]);
     const unsigned int b = tile * kTile + threadIdx.x;
     if (b >= p.nblk || (st.y >> 16) == 0) continue;   // past the end, or an all-zero block: nothing to optimise
     Block blk;
@@ -954,6 +1039,45 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
           if (g < best) { best = g; best_d = dc; }
         }
       }
+    } else if (kMode == 4) {
+      const int nd = d_hi - d_lo + 1;
+      Winner w;
+      if (whole_grid) {   // the same for every block of the tensor
+        whole_grid_search(blk, fx, alpha, center, s_beta, n_beta, d_lo, nd, w, wide);
+      } else {
+        w.g = __longlong_as_double(0x7FF0000000000000ll);
+        w.d = dc0;
+        w.k = 0;
+        w.A = w.B = 0.0;
+        w.c0 = w.c1 = 0u;
+        int prev = -1;
+        for (int d = d_lo; d <= d_hi; ++d) {
+          const int dc = clip_code(d);
+          if (dc == prev) continue;   // clipping at the ends of the E4M3 range repeats a code
+          prev = dc;
+          const float dv = e4m3_value(dc);
+          const double sd = alpha_d * static_cast<double>(dv);
+          int ka, kb;
+          winning_range(s_beta, n_beta, k_scale, k_off, alpha, center, dv, sd, ka, kb);
+          for (int k = ka; k <= kb; ++k) {
+            const float s = grid_divisor(alpha, center, s_beta[k]);
+            const float r = recip_fast_ok(s) ? recip_fast(s) : __frcp_rn(s);
+            unsigned int c0, c1;
+            double A, B;
+            round_block(blk, r, c0, c1);
+            block_sums(blk, fx, r, c0, c1, A, B, wide);
+            const double g = sd * fma(sd, B, -2.0 * A);
+            // equal errors: the earlier multiplier, then the smaller code, as in grid order
+            if (g < w.g || (g == w.g && k < w.k)) { w.g = g; w.A = A; w.B = B; w.c0 = c0; w.c1 = c1; w.d = dc; w.k = k; }
+          }
+        }
+      }
+      best = w.g;
+      bestA = w.A;
+      bestB = w.B;
+      best0 = w.c0;
+      best1 = w.c1;
+      best_d = w.d;
     } else {
       // Eq. 8 over beta ascending, then scale code ascending; strict '<' keeps the first
       // minimum.  Every candidate is scored in full, with no test for "same codes as the
@@ -1925,11 +2049,17 @@ int run_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void*
                                                                                       cfg->max_iters == 0 ? 1 : 0);
     }
     if (stages & kStageIterate) {
-      const int mode = !single ? 0 : ((cfg->flags & SOAR_FLAG_COUPLED_SCALE) ? 2 : (cfg->n_dq <= 2 ? 1 : 3));
+      // a grid of several multipliers with one quantization scale per multiplier: only those that can win
+      // are visited (mode 4); the coupled arm and grids of a few multipliers visit them all (mode 0)
+      const bool bracketed = !(cfg->flags & SOAR_FLAG_COUPLED_SCALE) && cfg->n_beta >= kBracketMinBeta &&
+                             cfg->beta_step_pct >= 1;
+      const int mode = !single ? (bracketed ? 4 : 0)
+                               : ((cfg->flags & SOAR_FLAG_COUPLED_SCALE) ? 2 : (cfg->n_dq <= 2 ? 1 : 3));
       const unsigned int g_it = mode == 0   ? persistent_grid(iterate_kernel<0>, tiles, kThreads)
                                 : mode == 1 ? persistent_grid(iterate_kernel<1>, tiles, kThreads)
                                 : mode == 2 ? persistent_grid(iterate_kernel<2>, tiles, kThreads)
-                                            : persistent_grid(iterate_kernel<3>, tiles, kThreads);
+                                : mode == 3 ? persistent_grid(iterate_kernel<3>, tiles, kThreads)
+                                            : persistent_grid(iterate_kernel<4>, tiles, kThreads);
       for (int t = t_lo; t < t_hi; ++t) {
         const int reverse = t & 1;
         // with the early stop on, any iteration may turn out to be the last one
@@ -1939,7 +2069,8 @@ int run_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void*
         if (mode == 0) iterate_kernel<0><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
         else if (mode == 1) iterate_kernel<1><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
         else if (mode == 2) iterate_kernel<2><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
-        else iterate_kernel<3><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
+        else if (mode == 3) iterate_kernel<3><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
+        else iterate_kernel<4><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
       }
     }
     if (!(stages & kStageFinalize)) continue;
