@@ -848,24 +848,31 @@ __device__ __forceinline__ float grid_divisor(float alpha, float center, float b
 // For a fixed dequantization scale sd = alpha * value(code) the error of element j,
 // (a_j - m sd)^2, is convex in its code value m with its minimum at a_j / sd.  The codes
 // m_j(k) = E2M1(fl(a_j * fl(1 / s_k))), s_k = grid_divisor(beta_k), never rise with k, because every
-// step of that binary32 chain is monotone.  While s_k <= sd (1 - 2^-23) every fl(a_j / s_k) is at
+// step of that binary32 chain is monotone.  While s_k <= sd (1 - 2^-23) every fl(a_j * fl(1 / s_k)) is at
 // least a_j / sd (two roundings of 2^-24 each), so every code is at or above the nearest one
-// to a_j / sd and each element's error can only fall as k grows; once s_k >= sd (1 + 2^-22) every code is at or
-// below it and the error can only rise.  The block error of Eq. 8 is therefore smallest at the
-// last multiplier of the first kind, at the first of the second kind, or at one in between
-// (the band is 2^-21 wide against a grid step of a hundredth: almost always empty).  Returns that
-// range [ka, kb]; two multipliers in the typical case, where the grid has 101.
+// to a_j / sd and each element's error can only fall as k grows; once s_k >= sd (1 + 2^-22) every code
+// is at or below it and the error can only rise.  The block error of Eq. 8 is therefore smallest at
+// the last multiplier of the first kind, at the first of the second kind, or at one in between
+// (the band is 2^-21 wide against a grid step of a hundredth: almost always empty): two
+// multipliers in the typical case, where the grid has 101.
 //
 // Equal errors.  Different codes of an element cost the same only when a_j / sd is exactly a
 // rounding midpoint, which needs sd, and with it alpha, to have at most eight significant bits;
 // callers send such tensors through the whole grid, so that the first minimum in grid order is
 // kept as Algorithm 1's strict comparison keeps it.
-__device__ __forceinline__ void winning_range(const float* s_beta, int n_beta, float k_scale, float k_off,
-                                              float alpha, float center, float dv, double sd, int& ka, int& kb) {
-  const float lo = __double2float_rd(sd * (1.0 - 0x1p-23));
-  const float hi = __double2float_ru(sd * (1.0 + 0x1p-22));
-  // start from the multiplier nearest dv / center; the two loops below make it exact
-  int k = __float2int_rn(__fmaf_rn(__fdividef(dv, center), k_scale, k_off));
+
+// Binary32 bounds of the band around sd = alpha * dv (the exact product): lo <= sd (1 - 2^-23) and
+// hi >= sd (1 + 2^-22), from the directed roundings of the product moved two and four units in the
+// last place (one unit is more than 2^-24 of the value).
+__device__ __forceinline__ void divisor_band(float alpha, float dv, float& lo, float& hi) {
+  lo = __uint_as_float(__float_as_uint(__fmul_rd(alpha, dv)) - 2u);
+  hi = __uint_as_float(__float_as_uint(__fmul_ru(alpha, dv)) + 4u);
+}
+
+// The range [ka, kb] of multipliers that can win for a code whose band is [lo, hi], for any start
+// index k: walks to the last multiplier with s_k <= lo, then on to the first with s_k >= hi.
+__device__ __forceinline__ void winning_range(const float* s_beta, int n_beta, float alpha, float center, float lo,
+                                           float hi, int k, int& ka, int& kb) {
   k = max(0, min(n_beta - 1, k));
   while (k >= 0 && grid_divisor(alpha, center, s_beta[k]) > lo) --k;
   while (k + 1 < n_beta && grid_divisor(alpha, center, s_beta[k + 1]) <= lo) ++k;
@@ -876,7 +883,7 @@ __device__ __forceinline__ void winning_range(const float* s_beta, int n_beta, f
 }
 
 // True when different codes of an element can cost exactly the same under this alpha (see
-// winning_range): alpha has at most eight significant bits.
+// above): alpha has at most eight significant bits.
 __device__ __forceinline__ bool alpha_allows_exact_ties(float alpha) {
   return (__float_as_uint(alpha) & 0xFFFFu) == 0u;
 }
@@ -885,20 +892,27 @@ __device__ __forceinline__ bool alpha_allows_exact_ties(float alpha) {
 struct Winner {
   double g, A, B;
   unsigned int c0, c1;
-  int d, k;
+  int d;
 };
 
-// Eq. 8 over the whole grid, beta ascending, then scale code ascending; strict '<' keeps the first
-// minimum.  Out of line: it serves only tensors that can have exactly equal candidates.
-__device__ __noinline__ void whole_grid_search(const Block& blk, const Fixed& fx, float alpha, float center,
-                                               const float* s_beta, int n_beta, int d_lo, int nd, Winner& w,
-                                               unsigned int& wide) {
+// Eq. 8 over the whole grid for the block at `w16` (sixteen bf16 values in global memory), beta
+// ascending, then scale code ascending; strict '<' keeps the first minimum.  Out of line, and
+// fed from memory rather than from the caller's registers: it serves only tensors that can
+// have exactly equal candidates.
+__device__ __forceinline__ void whole_grid_search(const uint16_t* w16, float alpha, float center, const float* s_beta,
+                                               int n_beta, int d_lo, int nd, Winner* out, unsigned int* wide_out) {
+  const uint4* src = reinterpret_cast<const uint4*>(w16);
+  Block blk;
+  unpack_block(__ldg(src), __ldg(src + 1), blk);
+  Fixed fx;
+  make_fixed(blk, fx);
   const double alpha_d = static_cast<double>(alpha);
+  Winner w;
   w.g = __longlong_as_double(0x7FF0000000000000ll);
   w.d = clip_code(d_lo);
-  w.k = 0;
   w.A = w.B = 0.0;
   w.c0 = w.c1 = 0u;
+  unsigned int wide = 0;
   for (int k = 0; k < n_beta; ++k) {
     const float r = recip_scale(alpha, __fmul_rn(center, s_beta[k]));
     unsigned int c0, c1;
@@ -909,9 +923,23 @@ __device__ __noinline__ void whole_grid_search(const Block& blk, const Fixed& fx
       const int dc = clip_code(d_lo + d);
       const double sd = alpha_d * static_cast<double>(e4m3_value(dc));
       const double g = sd * fma(sd, B, -2.0 * A);
-      if (g < w.g) { w.g = g; w.A = A; w.B = B; w.c0 = c0; w.c1 = c1; w.d = dc; w.k = k; }
+      if (g < w.g) { w.g = g; w.A = A; w.B = B; w.c0 = c0; w.c1 = c1; w.d = dc; }
     }
   }
+  *out = w;
+  *wide_out += wide;
+}
+
+// One candidate of the search scored on the exact integer sums: codes (signs included), afix, 4B and
+// e = rho * 4B - afix, which orders candidates of one E4M3 code like their errors.
+struct Scored {
+  unsigned int c0, c1, afix, b4;
+  double e;
+};
+__device__ __forceinline__ void score_candidate(const Block& blk, const Fixed& fx, float s, double rho, Scored& o) {
+  round_block(blk, recip_fast(s), o.c0, o.c1);
+  code_sums(fx, o.c0, o.c1, o.afix, o.b4);
+  o.e = fma(rho, uint_to_double(o.b4), -uint_to_double(o.afix));
 }
 
 // One iteration t of Algorithm 1 for every block: Eq. 5 (from stage-t sums), Eq. 6,
@@ -960,7 +988,7 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
   bool whole_grid = false;           // mode 4: the current tensor's alpha allows exactly equal candidates
   // mode 4: multiplier index of a scale ratio, k = (ratio - 1) * 100 / step + n_beta / 2
   const float k_scale = 100.0f / static_cast<float>(max(bt.t[0].beta_step_pct, 1));
-  const float k_off = static_cast<float>(n_beta / 2) - k_scale;
+  const float k_off = static_cast<float>(n_beta / 2) - k_scale;   // k = (dv / center) * k_scale + k_off
 
   double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum of stage t+1
   unsigned int wide = 0, unused_zeros = 0;
@@ -1041,43 +1069,97 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
       }
     } else if (kMode == 4) {
       const int nd = d_hi - d_lo + 1;
-      Winner w;
       if (whole_grid) {   // the same for every block of the tensor
-        whole_grid_search(blk, fx, alpha, center, s_beta, n_beta, d_lo, nd, w, wide);
+        const Params& q = bt.t[ti];
+        const unsigned int row = b / q.nbc, cb = b - row * q.nbc;
+        Winner w;
+        whole_grid_search(q.W + static_cast<long long>(row) * q.ld + static_cast<long long>(cb) * 16, alpha, center,
+                          s_beta, n_beta, d_lo, nd, &w, &wide);
+        best = w.g;
+        bestA = w.A;
+        bestB = w.B;
+        best0 = w.c0;
+        best1 = w.c1;
+        best_d = w.d;
       } else {
-        w.g = __longlong_as_double(0x7FF0000000000000ll);
-        w.d = dc0;
-        w.k = 0;
-        w.A = w.B = 0.0;
-        w.c0 = w.c1 = 0u;
-        int prev = -1;
-        for (int d = d_lo; d <= d_hi; ++d) {
-          const int dc = clip_code(d);
-          if (dc == prev) continue;   // clipping at the ends of the E4M3 range repeats a code
-          prev = dc;
-          const float dv = e4m3_value(dc);
-          const double sd = alpha_d * static_cast<double>(dv);
-          int ka, kb;
-          winning_range(s_beta, n_beta, k_scale, k_off, alpha, center, dv, sd, ka, kb);
-          for (int k = ka; k <= kb; ++k) {
-            const float s = grid_divisor(alpha, center, s_beta[k]);
-            const float r = recip_fast_ok(s) ? recip_fast(s) : __frcp_rn(s);
-            unsigned int c0, c1;
-            double A, B;
-            round_block(blk, r, c0, c1);
-            block_sums(blk, fx, r, c0, c1, A, B, wide);
-            const double g = sd * fma(sd, B, -2.0 * A);
-            // equal errors: the earlier multiplier, then the smaller code, as in grid order
-            if (g < w.g || (g == w.g && k < w.k)) { w.g = g; w.A = A; w.B = B; w.c0 = c0; w.c1 = c1; w.d = dc; w.k = k; }
+        // Typical block: two E4M3 codes at most, each with exactly two multipliers that can win (the one
+        // just below value(code) / center and its successor), the exact integer sums valid and the
+        // fast reciprocal in range for the whole grid.  Those four candidates are scored in straight
+        // line; any other block takes the loops below.
+        const bool second = nd == 2 && dc1 != dc0;
+        const float per_center = __fdividef(k_scale, center);
+        const float dv0 = e4m3_value(dc0), dv1 = e4m3_value(dc1);
+        float lo0, hi0, lo1, hi1;
+        divisor_band(alpha, dv0, lo0, hi0);
+        divisor_band(alpha, dv1, lo1, hi1);
+        const int k0 = max(0, min(n_beta - 2, __float2int_rd(__fmaf_rn(dv0, per_center, k_off))));
+        const int k1 = max(0, min(n_beta - 2, __float2int_rd(__fmaf_rn(dv1, per_center, k_off))));
+        const float s00 = grid_divisor(alpha, center, s_beta[k0]), s01 = grid_divisor(alpha, center, s_beta[k0 + 1]);
+        const float s10 = grid_divisor(alpha, center, s_beta[k1]), s11 = grid_divisor(alpha, center, s_beta[k1 + 1]);
+        const float s_first = grid_divisor(alpha, center, s_beta[0]);
+        bool direct = nd <= 2 && fx.ok && recip_fast_ok(s_first) &&
+                      recip_fast_ok(grid_divisor(alpha, center, s_beta[n_beta - 1])) &&
+                      __fmul_rn(blk.bmax, recip_fast(s_first)) <= 32.0f && s00 <= lo0 && s01 >= hi0;
+        if (second) direct = direct && s10 <= lo1 && s11 >= hi1;
+        if (direct) {
+          // error minus sum W^2 = 2 sd unit (rho * 4B - afix) with rho = sd / (8 unit): per code the two
+          // candidates are ranked on the exact integer sums, the codes' winners compared once
+          Scored a, c;
+          score_candidate(blk, fx, s00, sd0 * fx.inv8, a);
+          {
+            Scored b2;
+            score_candidate(blk, fx, s01, sd0 * fx.inv8, b2);
+            if (b2.e < a.e) a = b2;
+          }
+          double ga = 2.0 * sd0 * fx.unit * a.e;
+          best_d = dc0;
+          if (second) {
+            score_candidate(blk, fx, s10, sd1 * fx.inv8, c);
+            Scored b2;
+            score_candidate(blk, fx, s11, sd1 * fx.inv8, b2);
+            const bool later = b2.e < c.e;
+            if (later) c = b2;
+            const double gc = 2.0 * sd1 * fx.unit * c.e;
+            // equal errors: the earlier multiplier, as in grid order (k1 >= k0 always)
+            if (gc < ga) { ga = gc; a = c; best_d = dc1; }
+          }
+          best = ga;
+          best0 = a.c0;
+          best1 = a.c1;
+          bestA = uint_to_double(a.afix) * fx.unit;
+          bestB = uint_to_double(a.b4) * 0.25;
+        } else {
+          best = __longlong_as_double(0x7FF0000000000000ll);
+          bestA = bestB = 0.0;
+          best0 = best1 = 0u;
+          int best_k = 0, prev = -1;
+          for (int d = d_lo; d <= d_hi; ++d) {
+            const int dc = clip_code(d);
+            if (dc == prev) continue;   // clipping at the ends of the E4M3 range repeats a code
+            prev = dc;
+            const float dv = e4m3_value(dc);
+            const double sd = alpha_d * static_cast<double>(dv);
+            float lo, hi;
+            divisor_band(alpha, dv, lo, hi);
+            int ka, kb;
+            winning_range(s_beta, n_beta, alpha, center, lo, hi, __float2int_rd(__fmaf_rn(dv, per_center, k_off)), ka,
+                          kb);
+            for (int k = ka; k <= kb; ++k) {
+              const float sk = grid_divisor(alpha, center, s_beta[k]);
+              const float r = recip_fast_ok(sk) ? recip_fast(sk) : __frcp_rn(sk);
+              unsigned int c0, c1;
+              double A, B;
+              round_block(blk, r, c0, c1);
+              block_sums(blk, fx, r, c0, c1, A, B, wide);
+              const double g = sd * fma(sd, B, -2.0 * A);
+              // equal errors: the earlier multiplier, then the smaller code, as in grid order
+              if (g < best || (g == best && k < best_k)) {
+                best = g; bestA = A; bestB = B; best0 = c0; best1 = c1; best_d = dc; best_k = k;
+              }
+            }
           }
         }
       }
-      best = w.g;
-      bestA = w.A;
-      bestB = w.B;
-      best0 = w.c0;
-      best1 = w.c1;
-      best_d = w.d;
     } else {
       // Eq. 8 over beta ascending, then scale code ascending; strict '<' keeps the first
       // minimum.  Every candidate is scored in full, with no test for "same codes as the
@@ -1389,67 +1471,24 @@ __device__ __forceinline__ void weighted_sums_split(const double (&hw)[16], cons
   B = 0.25 * (b[0] + b[1]);
 }
 
-// Fixed-point images of sixteen non-negative binary64 values below 2^(e+1), `bits` (33..48) wide:
-// F_j = rn(v_j * 2^(bits - 1 - e)) <= 2^bits, cut into three 16-bit limbs and packed two elements
-// per word, the operand layout of the 16-bit x 8-bit dot-product instruction.
-struct Limbs {
-  unsigned int hi[8], mid[8], lo[8];
-};
-
-__device__ __forceinline__ int exponent_of(double v) {
-  return ((__double2hiint(v) >> 20) & 0x7FF) - 1023;
-}
-
-__device__ __forceinline__ double two_to(int e) { return __hiloint2double((1023 + e) << 20, 0); }
-
-__device__ __forceinline__ void make_limbs(const double (&v)[16], int e, int bits, Limbs& L) {
-  const double scale = two_to(bits - 1 - e);
+// A and B of a code vector (sign bits ignored) from the block's sixteen column weights and signed
+// elements, in element order like weighted_sums and with the same roundings, but widening each
+// weight and magnitude where it is used, so that only a few binary64 values are live at a time.
+__device__ __forceinline__ void weighted_sums_streamed(const float (&h)[16], const float (&w)[16], unsigned int c0,
+                                                       unsigned int c1, double& A, double& B) {
+  const unsigned int m0 = c0 & 0x77777777u, m1 = c1 & 0x77777777u;
+  const unsigned int t[4] = {twice_magnitude_x4(m0), twice_magnitude_x4(m0 >> 16), twice_magnitude_x4(m1),
+                             twice_magnitude_x4(m1 >> 16)};
+  double a = 0.0, b = 0.0;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const unsigned long long f0 = __double2ull_rn(v[2 * i] * scale), f1 = __double2ull_rn(v[2 * i + 1] * scale);
-    const unsigned int a0 = static_cast<unsigned int>(f0), a1 = static_cast<unsigned int>(f1);
-    L.hi[i] = (static_cast<unsigned int>(f0 >> 32) & 0xFFFFu) | (static_cast<unsigned int>(f1 >> 32) << 16);
-    L.mid[i] = __byte_perm(a0, a1, 0x7632);
-    L.lo[i] = __byte_perm(a0, a1, 0x5410);
+  for (int j = 0; j < 16; ++j) {
+    const double dm = uint_to_double_bits((t[j >> 2] >> (8 * (j & 3))) & 0xFFu);   // 2 m_j
+    const double hd = static_cast<double>(h[j]);
+    a = fma(hd * static_cast<double>(fabsf(w[j])), dm, a);
+    b = fma(hd, dm * dm, b);
   }
-}
-
-// Widths of the images of h_j |w_j| and of h_j: sum F_j 2m_j <= 192 * 2^45 and
-// sum G_j (2m_j)^2 <= 2304 * 2^41 both stay below 2^53.
-constexpr int kImageBitsA = 45, kImageBitsB = 41;
-
-// Four magnitude codes to four bytes holding (2m)^2: 0,1,4,9,16,36,64,144.
-__device__ __forceinline__ unsigned int twice_magnitude_squared_x4(unsigned int codes) {
-  unsigned int out;
-  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(0x09040100u), "r"(0x90402410u), "r"(codes));
-  return out;
-}
-
-// Integer images of the weighted sums of a magnitude code vector:
-// At = sum F_j (2 m_j) and Bt = sum G_j (2 m_j)^2, exact, as binary64.
-__device__ __forceinline__ void limb_sums(const Limbs& F, const Limbs& G, unsigned int c0, unsigned int c1, double& At,
-                                          double& Bt) {
-  const unsigned int c[4] = {c0, c0 >> 16, c1, c1 >> 16};
-  unsigned int ah = 0, am = 0, al = 0, bh = 0, bm = 0, bl = 0;
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const unsigned int t = twice_magnitude_x4(c[q]), u = twice_magnitude_squared_x4(c[q]);
-    ah = __dp2a_lo(F.hi[2 * q], t, ah);
-    ah = __dp2a_hi(F.hi[2 * q + 1], t, ah);
-    am = __dp2a_lo(F.mid[2 * q], t, am);
-    am = __dp2a_hi(F.mid[2 * q + 1], t, am);
-    al = __dp2a_lo(F.lo[2 * q], t, al);
-    al = __dp2a_hi(F.lo[2 * q + 1], t, al);
-    bh = __dp2a_lo(G.hi[2 * q], u, bh);
-    bh = __dp2a_hi(G.hi[2 * q + 1], u, bh);
-    bm = __dp2a_lo(G.mid[2 * q], u, bm);
-    bm = __dp2a_hi(G.mid[2 * q + 1], u, bm);
-    bl = __dp2a_lo(G.lo[2 * q], u, bl);
-    bl = __dp2a_hi(G.lo[2 * q + 1], u, bl);
-  }
-  // every limb sum is below 2^28 and, for kImageBitsA/B wide images, the whole below 2^53: exact
-  At = fma(fma(uint_to_double(ah), 65536.0, uint_to_double(am)), 65536.0, uint_to_double(al));
-  Bt = fma(fma(uint_to_double(bh), 65536.0, uint_to_double(bm)), 65536.0, uint_to_double(bl));
+  A = 0.5 * a;
+  B = 0.25 * b;
 }
 
 // hd[j] = h_j and hw[j] = h_j |w_j| of a block, binary64 (both exact).
@@ -1579,13 +1618,21 @@ weighted_init_kernel(const __grid_constant__ Batch bt, const Weighted wq, int re
   add_counters(p.ws, zeros, unused_wide);
 }
 
-// Eq. 8 for one block with binary64 sums for every candidate: index nd * k + d of the first minimum
-// in (beta, code) order.  Serves the coupled arm, code windows wider than two, and the blocks the
-// fixed-point ranking cannot decide; kept out of line so that its registers do not weigh on
-// that ranking's loop.
-__device__ __noinline__ int weighted_exact_argmin(const float* h, unsigned int cb, const Block& mags, float alpha,
+// Eq. 8 for one block over the whole grid with binary64 sums for every candidate: index nd * k + d of
+// the first minimum in (beta, code) order.  Serves the coupled arm and the blocks whose candidates
+// can cost exactly the same (see weighted_iterate_kernel); kept out of line so that its registers
+// do not weigh on the common path.
+__device__ __noinline__ int weighted_exact_argmin(const float* h, unsigned int cb, const uint16_t* w16, float alpha,
                                                   float center, const float* s_beta, int n_beta, int d_lo, int nd,
                                                   bool coupled, bool fast_rcp) {
+  // the block comes from memory (sixteen bf16 values at w16), not from the caller's registers
+  Block mags;
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(w16);
+    unpack_block(__ldg(src), __ldg(src + 1), mags);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) mags.w[j] = fabsf(mags.w[j]);
+  }
   double hd[16], hw[16];
   block_weights(h, cb, mags, hd, hw);
   const double alpha_d = static_cast<double>(alpha);
@@ -1648,6 +1695,10 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
   const double alpha_d = static_cast<double>(alpha);
   const bool coupled = (p.flags & SOAR_FLAG_COUPLED_SCALE) != 0;
   const bool keep_scale = (p.flags & SOAR_FLAG_KEEP_BLOCK_SCALE) != 0;
+  // multiplier index of a scale ratio: k = (ratio - 1) * 100 / step + n_beta / 2
+  const bool bracketed = p.beta_step_pct >= 1 && n_beta >= 2;
+  const float k_scale = 100.0f / static_cast<float>(max(p.beta_step_pct, 1));
+  const float k_off = static_cast<float>(n_beta / 2) - k_scale;
   double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum of stage t+1
   unsigned int exact_blocks = 0, unused_zeros = 0;
   for (unsigned int n = 0;; ++n) {
@@ -1662,10 +1713,7 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
     const double2 ab = wq.sums[b];
     Block blk;
     unpack_block(v0, v1, blk);
-    Block mags;                 // the block's magnitudes: the candidate loop only ranks
-    const unsigned int cb = b % p.nbc;
-#pragma unroll
-    for (int j = 0; j < 16; ++j) mags.w[j] = fabsf(blk.w[j]);
+    const unsigned int row = b / p.nbc, cb = b - row * p.nbc;
     // Eq. 6 (binary32 steps); a block whose weighted codes are all zero keeps its stored scale
     const float center = (ab.y > 0.0 && !keep_scale)
                              ? __fdiv_rn(static_cast<float>(ab.x), __fmul_rn(alpha, static_cast<float>(ab.y)))
@@ -1673,88 +1721,67 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
     int d_lo, d_hi;
     candidate_window(center, n_dq, d_lo, d_hi);
     const int nd = d_hi - d_lo + 1;
-    int best_key = 0;
     // the products alpha * center * beta are monotone in beta: the end points bound them all
     const bool fast_rcp = !coupled && recip_fast_ok(__fmul_rn(alpha, __fmul_rn(center, s_beta[0]))) &&
                           recip_fast_ok(__fmul_rn(alpha, __fmul_rn(center, s_beta[n_beta - 1])));
-
-    // Fast ranking.  The weighted error minus sum h w^2 is  g = sd^2 B - 2 sd A.  With 45- and 41-bit fixed-point
-    // images F_j of h_j |w_j| and G_j of h_j (relative to the block's largest), the integer sums
-    // At = sum F_j 2m_j and Bt = sum G_j (2m_j)^2 are exact and cost one dot-product instruction per
-    // two elements and limb; A = cA At and B = cB Bt up to the rounding of the images, at most 96 cA and
-    // 1152 cB.  The loop keeps, per E4M3 code, the best and the second-best distinct value; when the
-    // overall runner-up is further from the winner than those roundings could account for, the
-    // winner is the exact loop's winner.  Otherwise (rarely) the exact loop below decides.
-    bool decided = false;
-    if (!coupled && nd <= 2 && fast_rcp) {
-      double hmax = 0.0, hwmax = 0.0;
-      Limbs F, G;
-      {
-        double hd[16], hw[16];
-        block_weights(wq.h, cb, mags, hd, hw);
+    float hf[16];
+    {
+      const float4* src = reinterpret_cast<const float4*>(wq.h) + static_cast<size_t>(cb) * 4;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          hmax = fmax(hmax, hd[j]);
-          hwmax = fmax(hwmax, hw[j]);
-        }
-        if (hwmax > 0.0) {
-          make_limbs(hw, exponent_of(hwmax), kImageBitsA, F);
-          make_limbs(hd, exponent_of(hmax), kImageBitsB, G);
-        }
+      for (int q = 0; q < 4; ++q) {
+        const float4 v = __ldg(src + q);
+        hf[4 * q] = v.x; hf[4 * q + 1] = v.y; hf[4 * q + 2] = v.z; hf[4 * q + 3] = v.w;
       }
-      if (hwmax > 0.0) {
-        const int ea = exponent_of(hwmax), eb = exponent_of(hmax);
-        const double cA = two_to(ea - kImageBitsA), cB = two_to(eb - kImageBitsB - 1);   // A = cA At, B = cB Bt
-        const double sd0 = alpha_d * static_cast<double>(e4m3_value(clip_code(d_lo)));
-        const double sd1 = alpha_d * static_cast<double>(e4m3_value(clip_code(d_lo + 1)));
-        // g = 2 sd cA (rho Bt - At)  with  rho = sd cB / (2 cA)
-        const double ratio = two_to(eb - ea + kImageBitsA - kImageBitsB - 2);   // cB / (2 cA)
-        const double rho0 = sd0 * ratio, rho1 = sd1 * ratio;
-        const double inf = __longlong_as_double(0x7FF0000000000000ll);
-        double h0 = inf, s0 = inf, h1 = inf, s1 = inf;
-        int k0 = 0, k1 = 0;
-        for (int k = 0; k < n_beta; ++k) {
+    }
+    // The weighted error of element j, h_j (a_j - m sd)^2, is convex in m like the unweighted one, so per
+    // E4M3 code only the multipliers of winning_range can win (see there).  Candidates can cost exactly the
+    // same when alpha has few significant bits or when a column's weight is zero (its code then costs
+    // nothing, whatever it is): such blocks, and the coupled arm, walk the whole grid.
+    bool zero_weight = false;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) zero_weight = zero_weight || hf[j] == 0.0f;
+    unsigned int best0 = 0, best1 = 0;
+    double bestA = 0.0, bestB = 0.0;
+    int best_d = clip_code(d_lo);
+    if (!coupled && bracketed && !zero_weight && !alpha_allows_exact_ties(alpha)) {
+      double best = __longlong_as_double(0x7FF0000000000000ll);
+      int best_k = 0, prev = -1;
+      const float per_center = __fdividef(k_scale, center);
+      for (int d = d_lo; d <= d_hi; ++d) {
+        const int dc = clip_code(d);
+        if (dc == prev) continue;   // clipping at the ends of the E4M3 range repeats a code
+        prev = dc;
+        const float dv = e4m3_value(dc);
+        const double sd = alpha_d * static_cast<double>(dv);
+        float lo, hi;
+        divisor_band(alpha, dv, lo, hi);
+        int ka = max(0, min(n_beta - 2, __float2int_rd(__fmaf_rn(dv, per_center, k_off))));
+        int kb = ka + 1;
+        if (!(grid_divisor(alpha, center, s_beta[ka]) <= lo && grid_divisor(alpha, center, s_beta[kb]) >= hi))
+          winning_range(s_beta, n_beta, alpha, center, lo, hi, ka, ka, kb);
+        for (int k = ka; k <= kb; ++k) {
+          const float sk = grid_divisor(alpha, center, s_beta[k]);
           unsigned int c0, c1;
-          round_block(mags, recip_fast(__fmul_rn(alpha, __fmul_rn(center, s_beta[k]))), c0, c1);
-          double At, Bt;
-          limb_sums(F, G, c0, c1, At, Bt);
-          // An equal value is the same outcome again (a neighbouring beta with the same codes) and is
-          // passed over, as the exact loop's strict comparison passes it over.  (Different codes with
-          // equal images differ in exact error by less than the margin below: a tie either way.)
-          const double e0 = fma(rho0, Bt, -At);
-          if (e0 < h0) { s0 = h0; h0 = e0; k0 = k; }
-          else if (e0 > h0 && e0 < s0) s0 = e0;
-          if (nd == 2) {
-            const double e1 = fma(rho1, Bt, -At);
-            if (e1 < h1) { s1 = h1; h1 = e1; k1 = k; }
-            else if (e1 > h1 && e1 < s1) s1 = e1;
+          round_block(blk, fast_rcp ? recip_fast(sk) : __frcp_rn(sk), c0, c1);
+          double A, B;
+          weighted_sums_streamed(hf, blk.w, c0, c1, A, B);
+          const double g = sd * fma(sd, B, -2.0 * A);
+          // equal errors: the earlier multiplier, then the smaller code, as in grid order
+          if (g < best || (g == best && k < best_k)) {
+            best = g; bestA = A; bestB = B; best0 = c0; best1 = c1; best_d = dc; best_k = k;
           }
         }
-        const double q0 = 2.0 * sd0 * cA, q1 = 2.0 * sd1 * cA;
-        const double g0 = q0 * h0, g1 = (nd == 2) ? q1 * h1 : inf;
-        const bool second = g1 < g0;
-        const double win = second ? g1 : g0;
-        const double runner = fmin(second ? g0 : g1, second ? q1 * s1 : q0 * s0);
-        const double sdm = fmax(sd0, sd1);
-        const double margin = 2.02 * sdm * fma(sdm, 1152.0 * cB, 192.0 * cA);
-        decided = runner - win > margin;
-        best_key = second ? nd * k1 + 1 : nd * k0;
       }
-    }
-    if (!decided) {
-      best_key = weighted_exact_argmin(wq.h, cb, mags, alpha, center, s_beta, n_beta, d_lo, nd, coupled, fast_rcp);
+    } else {
+      const int best_key =
+          weighted_exact_argmin(wq.h, cb, p.W + static_cast<long long>(row) * p.ld + static_cast<long long>(cb) * 16,
+                                alpha, center, s_beta, n_beta, d_lo, nd, coupled, fast_rcp);
       ++exact_blocks;
-    }
-    // the winner, made again from its index, now with the signs and the sums in element order
-    const int bk = best_key / nd;
-    const int best_d = clip_code(d_lo + (best_key - bk * nd));
-    unsigned int best0, best1;
-    double bestA, bestB;
-    round_block(blk, recip_scale(alpha, __fmul_rn(coupled ? e4m3_value(best_d) : center, s_beta[bk])), best0, best1);
-    {
-      double hd[16], hw[16];
-      block_weights(wq.h, cb, mags, hd, hw);
-      weighted_sums(hw, hd, best0, best1, bestA, bestB);
+      // the winner, made again from its index, now with the signs and the sums in element order
+      const int bk = best_key / nd;
+      best_d = clip_code(d_lo + (best_key - bk * nd));
+      round_block(blk, recip_scale(alpha, __fmul_rn(coupled ? e4m3_value(best_d) : center, s_beta[bk])), best0, best1);
+      weighted_sums_streamed(hf, blk.w, best0, best1, bestA, bestB);
     }
     if (emit) {
       reinterpret_cast<uint2*>(p.packed)[b] = make_uint2(best0, best1);
