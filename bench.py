@@ -8,9 +8,10 @@ C-ABI library with all inputs already resident in HBM.  Prints ONE JSON line on 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                   [--workload config1|config2|config3|config4|config5] [--preset paper|single_pass]
 
-Multi-GPU runs are launched by torch.distributed.run, one rank per GPU; the tensors of a
-model are independent, so every rank quantizes its own copy of the workload with no
-collective on the data path (weak scaling).
+Multi-GPU runs are one rank per GPU under torch.distributed.run (started by the caller, or by
+this script itself when --gpus N is given to a plain process); the tensors of a model are
+independent, so every rank quantizes its own copy of the workload with no collective on the
+data path (weak scaling).
 """
 from __future__ import annotations
 
@@ -32,11 +33,6 @@ if ROOT not in sys.path:
 from paper_2605_12245_b200 import workloads as WL  # noqa: E402
 
 SM_COUNT = 148
-FP32_LANES_PER_SM = 128
-# Instructions an element of one candidate needs at the least: scale multiply, rounding to
-# the E2M1 grid, and the two accumulations of Eq. 5/6's block sums.
-OPS_PER_ELEMENT_EVAL = 4
-OPS_PER_PAIR_SCORE = 3
 
 
 def load_peaks():
@@ -96,9 +92,20 @@ def ref_cfg_of(R, cfg):
                     n_beta=cfg.n_beta, beta_step_pct=cfg.beta_step_pct, flags=cfg.flags)
 
 
-# Algorithmic work per 16-element block: what the method itself demands, not what a kernel happens to execute
-def iterate_ops_per_block(cfg) -> float:
-    return cfg.n_beta * (16 * OPS_PER_ELEMENT_EVAL + cfg.n_dq * OPS_PER_PAIR_SCORE)
+def ref_preset_cfg(R, preset: str, args):
+    """The oracle's settings for a preset, from the oracle's own defaults (the paper's: Sec. 4.1, App. B.3)
+    and the same command-line overrides as ``preset_cfg``; the CUDA library plays no part in it."""
+    c = R.RefCfg()
+    if preset == "single_pass":
+        c = R.RefCfg(max_iters=1, early_stop_rel=0.0, n_dq=2, n_beta=1)
+    elif preset == "coupled_pair":
+        c = R.RefCfg(n_dq=2, n_beta=1, flags=R.FLAG_COUPLED_SCALE)
+    if args.pairs:
+        c.n_dq = min(2, args.pairs)
+        c.n_beta = max(1, args.pairs // c.n_dq)
+    if args.iters is not None:
+        c.max_iters, c.early_stop_rel = args.iters, 0.0
+    return c
 
 
 OUT_BYTES = 0.5 + 1.0 / 16          # codes + scale byte per element
@@ -130,6 +137,8 @@ NCU_TRAFFIC = {
     "kernel_source_sha256_16": "7b27270025a5ae1d",
     "bytes_per_elem": {"amax_kernel": 2.02, "init_kernel": 2.43, "iterate_kernel/single": 3.00,
                        "iterate_kernel/grid": 3.45, "weighted_iterate_kernel": 4.58},
+    "inst_per_block": {"amax_kernel": 125, "init_kernel": 218, "iterate_kernel/single": 258,
+                       "iterate_kernel/grid": 6117, "weighted_iterate_kernel": 14400},
 }
 
 
@@ -150,12 +159,23 @@ def kernel_source_hash() -> str | None:
     return hashlib.sha256(text.split(HOST_MARKER)[0]).hexdigest()[:16]
 
 
+def _profile_key(name: str, cfg) -> str:
+    if name == "iterate_kernel":
+        name += "/single" if cfg.n_beta == 1 and not (cfg.n_dq > 2 and cfg.flags & 1) else "/grid"
+    return name
+
+
 def ncu_traffic_per_elem(name: str, cfg):
     if kernel_source_hash() != NCU_TRAFFIC["kernel_source_sha256_16"]:
         return None
-    if name == "iterate_kernel":
-        name += "/single" if cfg.n_beta == 1 and not (cfg.n_dq > 2 and cfg.flags & 1) else "/grid"
-    return NCU_TRAFFIC["bytes_per_elem"].get(name)
+    return NCU_TRAFFIC["bytes_per_elem"].get(_profile_key(name, cfg))
+
+
+def ncu_inst_per_block(name: str, cfg):
+    """Executed instructions per 16-element block and launch (ncu, same captures), or None once the kernels changed."""
+    if kernel_source_hash() != NCU_TRAFFIC["kernel_source_sha256_16"]:
+        return None
+    return NCU_TRAFFIC["inst_per_block"].get(_profile_key(name, cfg))
 
 
 def call_bytes_per_elem(cfg, iters_run: int) -> float:
@@ -239,17 +259,15 @@ def run_reference(args):
     if rank != 0:
         return
     from oracle import soar_ref as R
-    from paper_2605_12245_b200 import api
     wl = pick_workload(args.workload)
-    cfg = preset_cfg(api, args.preset, args)
-    rcfg = ref_cfg_of(R, cfg)
+    cfg = rcfg = ref_preset_cfg(R, args.preset, args)
     spec = wl.tensors[0]
     rows = min(spec.rows, max(1, args.ref_rows))
     rows = max(1, rows // WL._chunk_rows(spec.cols)) * WL._chunk_rows(spec.cols)
     w = wl.generate(0, 0, rows)
     h = WL.column_weights(spec.cols, 1000) if args.objective == "weighted" else None
     for _ in range(args.warmup):
-        R.quantize(w[: max(1, rows // 8)], rcfg, h=h)
+        R.quantize(w, rcfg, h=h)
     t0 = time.perf_counter()
     for _ in range(args.steps):
         R.quantize(w, rcfg, h=h)
@@ -374,10 +392,10 @@ def run_ours(args):
     value = world * 2.0 * elements / (ms * 1e-3) / 1e9
     launches = sum(v[0] for v in trace.values())
 
-    # ---- roofline of the dominant kernel
+    # ---- roofline of the dominant kernel: its algorithmic bytes over its measured device time, against the
+    # measured HBM copy bandwidth; beside it the issue-slot side from the committed profile
     dom = max(trace, key=lambda k: trace[k][1])
     n_launch, tot_ms = trace[dom]
-    # DRAM traffic of an average working launch of the dominant kernel (ncu figure per element x elements)
     if args.no_batch:
         active = sum(iters) if dom == "iterate_kernel" else len(wl.tensors)
     else:      # one launch serves a group of up to 16 tensors; an iteration launch works while any of them runs
@@ -387,30 +405,28 @@ def run_ours(args):
     work_elems = (sum(s.rows * s.cols * it for s, it in zip(wl.tensors, iters)) if dom == "iterate_kernel"
                   else elements)
     traffic = None if tpe is None or active == 0 else tpe * work_elems / active
-    if dom == "iterate_kernel" and iterate_ops_per_block(cfg) > 16 * 180:
-        # candidate loop dominates: bound by plain FP32/INT issue
-        blocks_iters = sum((s.rows * s.cols // 16) * it for s, it in zip(wl.tensors, iters)) * args.steps
-        ops = blocks_iters * iterate_ops_per_block(cfg)
-        achieved = ops / (tot_ms * 1e-3) / 1e12
-        peak = SM_COUNT * FP32_LANES_PER_SM * peaks["sm_max_mhz"] * 1e6 / 1e12
-        roofline = dict(bound="alu", kernel=dom, achieved=achieved, peak=peak, unit="Tlane-op/s",
-                        frac=achieved / peak, traffic=traffic, launches=n_launch,
-                        active_launches=active * args.steps, kernel_ms_per_step=tot_ms / args.steps,
-                        peak_source="148 SMs x 128 FP32 lanes x clocks.max.sm",
-                        hbm_gbs_for_context=sum(
-                            s.rows * s.cols * kernel_bytes_per_elem(dom, cfg, t)
-                            for s, it in zip(wl.tensors, iters) for t in range(it)) * args.steps / (tot_ms * 1e-3) / 1e9)
+    if dom == "iterate_kernel":
+        byts = sum(s.rows * s.cols * kernel_bytes_per_elem(dom, cfg, t)
+                   for s, it in zip(wl.tensors, iters) for t in range(it)) * args.steps
     else:
-        if dom == "iterate_kernel":
-            byts = sum(s.rows * s.cols * kernel_bytes_per_elem(dom, cfg, t)
-                       for s, it in zip(wl.tensors, iters) for t in range(it)) * args.steps
-        else:
-            byts = elements * args.steps * kernel_bytes_per_elem(dom, cfg)
-        achieved = byts / (tot_ms * 1e-3) / 1e9
-        roofline = dict(bound="hbm", kernel=dom, achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
-                        frac=achieved / peaks["hbm_gbs"], traffic=traffic, launches=n_launch,
-                        kernel_ms_per_step=tot_ms / args.steps, peak_source=peaks["source"],
-                        frac_of_nominal_8000=achieved / 8000.0)
+        byts = elements * args.steps * kernel_bytes_per_elem(dom, cfg)
+    achieved = byts / (tot_ms * 1e-3) / 1e9
+    ipb = ncu_inst_per_block(dom, cfg)
+    issue = None
+    if ipb is not None and dom == "iterate_kernel":
+        warp_inst = ipb * (work_elems / 16) / 32 * args.steps
+        issue_peak = SM_COUNT * 4 * peaks["sm_max_mhz"] * 1e6            # one warp instruction per scheduler and clock
+        issue = dict(instructions_per_block=ipb, frac_of_issue_peak=warp_inst / (tot_ms * 1e-3) / issue_peak,
+                     peak="148 SMs x 4 schedulers x clocks.max.sm", source="ncu, profiles/ (same kernel source)")
+    roofline = dict(bound="hbm", kernel=dom, achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
+                    frac=achieved / peaks["hbm_gbs"], traffic=traffic, launches=n_launch,
+                    active_launches=active * args.steps, kernel_ms_per_step=tot_ms / args.steps,
+                    peak_source=peaks["source"], frac_of_nominal_8000=achieved / 8000.0, issue=issue)
+    call_bytes = sum(s.rows * s.cols * call_bytes_per_elem(cfg, it) for s, it in zip(wl.tensors, iters))
+    call_gbs = world * call_bytes / (ms * 1e-3) / 1e9
+    whole_call = dict(algorithmic_bytes_per_step=call_bytes, achieved_gbs=call_gbs,
+                      frac_of_measured_hbm=call_gbs / world / peaks["hbm_gbs"],
+                      frac_of_nominal_8000=call_gbs / world / 8000.0)
     kernels = {k: dict(launches=v[0], ms_per_step=v[1] / args.steps, share=v[1] / sum(x[1] for x in trace.values()))
                for k, v in trace.items()}
 
@@ -468,36 +484,62 @@ def run_ours(args):
                                  frac_of_measured_hbm=k_bytes / (k_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]))
         extra["sweep_dq"] = rows_out
 
-    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    # ---- the timed batch's outputs against one soar_quantize call per tensor (same bytes expected)
+    bad = []
+    for i, (W, o) in enumerate(zip(dev_w, outs)):
+        one = api.soar_quantize(W, cfg)
+        torch.cuda.synchronize()
+        if not (torch.equal(one.packed, o.packed) and torch.equal(one.scales, o.scales) and torch.equal(one.alpha, o.alpha)
+                and one.read_result().iters_run == iters[i]):
+            bad.append(i)
+        del one
+    outputs_checked = dict(tensors=len(outs), differing_from_single_calls=bad)
+    if bad:
+        raise SystemExit(f"batched outputs differ from per-tensor calls for tensors {bad}")
+
+    # ---- end to end through the C ABI's host-buffer pipeline (soar_pipeline_run): pinned host buffers in and out,
+    # every copy inside the timed region
     import ctypes
     ctypes_sizeof_result = ctypes.sizeof(api.SoarResult)
     e2e = None
-    if not args.no_e2e and args.workload != "config3":      # config 3 would pin 18 GB of host memory
-        pipe = api.HostPipeline([(s.rows, s.cols) for s in wl.tensors], cfg, depth=6)
+    if not args.no_e2e:
+        # config 3 would pin 18 GB: its 36 layers go through a ring of four layers' worth of pinned buffers
+        # (36 x 7 copies in and out per step all the same; layer l reads the ring's layer l mod 4)
+        per_layer = 7 if args.workload == "config3" else len(wl.tensors)
+        ring_layers = 4 if args.workload == "config3" else 1
+        pipe = api.HostPipeline([(s.rows, s.cols) for s in wl.tensors[:per_layer]], cfg, depth=6)
         hosts = []
-        for h, spec in zip(host_w, wl.tensors):
+        for h, spec in zip(host_w[:per_layer * ring_layers], wl.tensors):
             hb = api.alloc_host_buffers(spec.rows, spec.cols, cfg)
             hb.W.copy_(h)
             hosts.append(hb)
+        order = [hosts[i % len(hosts)] for i in range(len(wl.tensors))]
 
         def e2e_step():
-            pipe.run(hosts)
+            pipe.run(order)
 
         for _ in range(2):
             e2e_step()
+        pipe.synchronize()
         barrier()
         t0 = time.perf_counter()
         for _ in range(args.steps):
             e2e_step()
-        torch.cuda.synchronize()
+        pipe.synchronize()
         dt = (time.perf_counter() - t0) / args.steps
         dt = SH.max_over_ranks(dt, "cuda")
         # results must equal the resident-input run
-        assert hosts[0].read_result().iters_run == iters[0]
+        r_last = hosts[(len(wl.tensors) - 1) % len(hosts)].read_result()
+        assert r_last.status == 0 and hosts[0].read_result().iters_run == iters[0]
+        assert torch.equal(hosts[0].packed, outs[0].packed.cpu())
         e2e = dict(value=world * 2.0 * elements / dt / 1e9, unit="GB/s", ms_per_step=dt * 1e3,
                    h2d_bytes_per_step=2 * elements,
                    d2h_bytes_per_step=elements // 2 + elements // 16 + len(wl.tensors) * (4 + ctypes_sizeof_result),
-                   api="HostPipeline: pinned host buffers, copy-in / soar_quantize / copy-out on three streams, 6 slots")
+                   api="soar_pipeline_run (C ABI): pinned host buffers, copy-in / soar_quantize / copy-out on three "
+                       "streams over 6 device slots",
+                   host_buffers=("%d distinct pinned layers reused in turn" % ring_layers) if ring_layers > 1
+                   else "one pinned buffer set per tensor")
+        pipe.close()
 
     # ---- the oracle on the host cores, bounded sample (rank 0, single GPU only)
     cpu = None
@@ -526,17 +568,14 @@ def run_ours(args):
                         parallelism=f"{world} rank(s), one layer of these shapes each, no collective"),
             elements_per_s=world * elements / (ms * 1e-3), host_clock_ms_per_step=host_ms[0],
             hbm_frac_end_to_end_of_measured=value / peaks["hbm_gbs"],
-            traced_ms_per_step=traced_ms, cuda_graph=bool(args.graph), batched=not args.no_batch, roofline=roofline, kernels=kernels, cpu_baseline=cpu, e2e=e2e, gpu_launches=launches,
-            clocks=clocks, **extra)
+            traced_ms_per_step=traced_ms, cuda_graph=bool(args.graph), batched=not args.no_batch, roofline=roofline,
+            whole_call=whole_call, kernels=kernels, outputs_checked=outputs_checked, cpu_baseline=cpu, e2e=e2e,
+            gpu_launches=launches, clocks=clocks, **extra)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
 
-# Column-weighted objective: per candidate and element the scale multiply, the rounding and two binary64
-# accumulations (A and B carry arbitrary weights, so they cannot be integer dot products); a binary64
-# fused multiply-add issues at half the FP32 rate and counts as two lane-operations.
-WEIGHTED_OPS_PER_ELEMENT_EVAL = 6
 WEIGHTED_STATE_BYTES = 17.0 / 16    # {A, B} in binary64 and the scale code per 16-element block
 
 
@@ -623,27 +662,21 @@ def run_weighted(args):
     launches = sum(v[0] for v in trace.values())
     dom = max(trace, key=lambda k: trace[k][1])
     n_launch, tot_ms = trace[dom]
-    ops_per_block = cfg.n_beta * (16 * WEIGHTED_OPS_PER_ELEMENT_EVAL + cfg.n_dq * OPS_PER_PAIR_SCORE)
     it_bytes = sum(s.rows * s.cols * weighted_kernel_bytes_per_elem("weighted_iterate_kernel", cfg, t)
                    for s, it in zip(wl.tensors, iters) for t in range(it)) * args.steps
-    if dom == "weighted_iterate_kernel":
-        blocks_iters = sum((s.rows * s.cols // 16) * it for s, it in zip(wl.tensors, iters)) * args.steps
-        achieved = blocks_iters * ops_per_block / (tot_ms * 1e-3) / 1e12
-        peak = SM_COUNT * FP32_LANES_PER_SM * peaks["sm_max_mhz"] * 1e6 / 1e12
-        tpe = ncu_traffic_per_elem(dom, cfg)
-        work_elems = sum(s.rows * s.cols * it for s, it in zip(wl.tensors, iters))
-        roofline = dict(bound="alu", kernel=dom, achieved=achieved, peak=peak, unit="Tlane-op/s", frac=achieved / peak,
-                        traffic=None if tpe is None or sum(iters) == 0 else tpe * work_elems / sum(iters),
-                        launches=n_launch, active_launches=sum(iters) * args.steps,
-                        kernel_ms_per_step=tot_ms / args.steps,
-                        peak_source="148 SMs x 128 FP32 lanes x clocks.max.sm",
-                        hbm_gbs_for_context=it_bytes / (tot_ms * 1e-3) / 1e9)
-    else:
-        byts = elements * args.steps * weighted_kernel_bytes_per_elem(dom, cfg)
-        achieved = byts / (tot_ms * 1e-3) / 1e9
-        roofline = dict(bound="hbm", kernel=dom, achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
-                        frac=achieved / peaks["hbm_gbs"], traffic=None, launches=n_launch,
-                        kernel_ms_per_step=tot_ms / args.steps, peak_source=peaks["source"])
+    byts = it_bytes if dom == "weighted_iterate_kernel" else elements * args.steps * weighted_kernel_bytes_per_elem(dom, cfg)
+    achieved = byts / (tot_ms * 1e-3) / 1e9
+    tpe = ncu_traffic_per_elem(dom, cfg)
+    work_elems = sum(s.rows * s.cols * it for s, it in zip(wl.tensors, iters))
+    roofline = dict(bound="hbm", kernel=dom, achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
+                    frac=achieved / peaks["hbm_gbs"],
+                    traffic=None if tpe is None or sum(iters) == 0 or dom != "weighted_iterate_kernel"
+                    else tpe * work_elems / sum(iters),
+                    launches=n_launch, active_launches=sum(iters) * args.steps if dom == "weighted_iterate_kernel" else n_launch,
+                    kernel_ms_per_step=tot_ms / args.steps, peak_source=peaks["source"],
+                    frac_of_nominal_8000=achieved / 8000.0,
+                    note="the block sums carry arbitrary weights, so they are binary64 sums in element order: "
+                         "the pass is bound by binary64 issue, not by HBM")
     kernels = {k: dict(launches=v[0], ms_per_step=v[1] / args.steps, share=v[1] / sum(x[1] for x in trace.values()))
                for k, v in trace.items()}
 
@@ -682,8 +715,9 @@ def run_weighted(args):
         e2e = dict(value=world * 2.0 * elements / dt / 1e9, unit="GB/s", ms_per_step=dt * 1e3,
                    h2d_bytes_per_step=2 * elements,
                    d2h_bytes_per_step=elements // 2 + elements // 16 + len(wl.tensors) * (4 + ctypes.sizeof(api.SoarResult)),
-                   api="HostPipeline: pinned host buffers, copy-in / soar_quantize_weighted / copy-out on three streams, "
-                       "6 slots (the column weights stay on the device)")
+                   api="soar_pipeline_run (C ABI): pinned host buffers, copy-in / soar_quantize_weighted / copy-out on "
+                       "three streams over 6 device slots (the column weights stay on the device)")
+        pipe.close()
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -785,10 +819,9 @@ def run_row_sharded(args):
     res = out.read_result()
     dom = max(trace, key=lambda k: trace[k][1])
     n_launch, tot_ms = trace[dom]
-    local_blocks = (r1 - r0) * spec.cols // 16
-    ops = local_blocks * res.iters_run * iterate_ops_per_block(cfg) * args.steps
-    peak = SM_COUNT * FP32_LANES_PER_SM * peaks["sm_max_mhz"] * 1e6 / 1e12
-    achieved = ops / (tot_ms * 1e-3) / 1e12
+    local_elems = (r1 - r0) * spec.cols
+    byts = local_elems * sum(kernel_bytes_per_elem(dom, cfg, t) for t in range(res.iters_run if dom == "iterate_kernel" else 1)) * args.steps
+    achieved = byts / (tot_ms * 1e-3) / 1e9
     if rank == 0:
         line = dict(
             metric="soar_quantize_bf16_input_throughput", value=2.0 * elements / (ms * 1e-3) / 1e9, unit="GB/s",
@@ -800,12 +833,47 @@ def run_row_sharded(args):
                         l2="inputs (%.2f GB per rank) exceed the 126 MB L2" % (2 * (r1 - r0) * spec.cols / 1e9),
                         parallelism=f"{world} rank(s), rows split evenly, two small all-reduces per stage"),
             elements_per_s=elements / (ms * 1e-3),
-            roofline=dict(bound="alu", kernel=dom, achieved=achieved, peak=peak, unit="Tlane-op/s",
-                          frac=achieved / peak, traffic=None, launches=n_launch, kernel_ms_per_step=tot_ms / args.steps,
-                          peak_source="148 SMs x 128 FP32 lanes x clocks.max.sm (rank 0's kernels and rows)"),
+            roofline=dict(bound="hbm", kernel=dom, achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
+                          frac=achieved / peaks["hbm_gbs"], traffic=None, launches=n_launch,
+                          kernel_ms_per_step=tot_ms / args.steps,
+                          peak_source=peaks["source"] + " (rank 0's kernels and rows)"),
             kernels={k: dict(launches=v[0], ms_per_step=v[1] / args.steps) for k, v in trace.items()},
             cpu_baseline=None, e2e=None, gpu_launches=sum(v[0] for v in trace.values()), clocks=clocks)
         print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def launcher_command(n_ranks: int, argv, port: int):
+    """The command that starts ``n_ranks`` ranks of this script on one node, one per GPU."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_ranks}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+
+
+def self_launch(args, argv) -> int:
+    """``bench.py --gpus N`` started as a plain process: start the N ranks here and pass their output on."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    return subprocess.call(launcher_command(args.gpus, argv, port))
+
+
+def run_dry(args):
+    """The multi-rank plumbing alone, on CPU ranks over gloo (no GPU, no quantizer): rendezvous, barrier and
+    the maximum over ranks that every timed number goes through.  Rank 0 prints the rank count."""
+    import torch.distributed as dist
+
+    from paper_2605_12245_b200 import sharding as SH
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    ms = SH.max_over_ranks(1.0 + rank, "cpu")
+    units = SH.sum_over_ranks(1.0, "cpu")
+    if rank == 0:
+        print(json.dumps(dict(dry_run=True, n_gpus=world, ranks_seen=int(units), ms_per_step=ms)), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
@@ -833,9 +901,15 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-single-pass", action="store_true")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="CPU ranks over gloo: only the launch and the rank bookkeeping (for tests)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.impl == "reference":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        raise SystemExit(self_launch(args, sys.argv[1:]))      # one rank per GPU, started from here
+    if args.dry_run:
+        run_dry(args)
+    elif args.impl == "reference":
         run_reference(args)
     elif args.row_sharded:
         run_row_sharded(args)

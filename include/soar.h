@@ -33,7 +33,8 @@ extern "C" {
 #define SOAR_ERR_UNSUPPORTED (-2)      /* cols % 16, ld < cols, alignment, block != 16, ... */
 #define SOAR_ERR_WORKSPACE (-3)        /* workspace missing or too small                    */
 #define SOAR_ERR_CUDA (-4)             /* a CUDA runtime call or kernel launch failed       */
-#define SOAR_ERR_TOO_LARGE (-5)        /* matrix exceeds the built-in scratch of soar_quantize_static */
+#define SOAR_ERR_TOO_LARGE (-5)        /* matrix exceeds the built-in scratch of soar_quantize_static,
+                                          or the capacity of a pipeline slot                */
 
 /* soar_result.status bits (device side, data dependent) */
 #define SOAR_STATUS_ZERO_TENSOR 1      /* every element is zero: alpha = 1, scales = 0      */
@@ -240,6 +241,61 @@ int soar_quantize_host(const void* W_host, int64_t rows, int64_t cols, int64_t l
                        const soar_cfg* cfg, void* out_fp4_packed_host, void* out_e4m3_scales_host,
                        void* out_e4m3_scales_sw_host, float* out_global_host,
                        soar_result* out_result_host, const soar_staging* dev, void* stream);
+
+/*
+ * Overlapped form of soar_quantize_host for a list of matrices in host memory (Algorithm 1 on each;
+ * same outputs).  A pipeline owns three caller-supplied streams and a ring of caller-supplied device
+ * staging slots: the copy of matrix i+1 into its slot (first stream) runs while matrix i is
+ * quantized (second stream) and the results of matrix i-1 are copied back (third stream), chained
+ * by the pipeline's own events, so that on a machine whose host link is slower than the quantizer
+ * the list costs about as much as its copies.  Slots are taken in turn and the turn carries over
+ * from one soar_pipeline_run to the next, so a new list starts on the slot that has been free the
+ * longest and its copies overlap the previous list's work.
+ *
+ *   soar_pipeline_create   slots: n_slots >= 1 descriptors (host memory, copied): device buffers as in
+ *                          soar_staging plus their capacities in bytes; a matrix fits a slot when its
+ *                          rows*ld*2 input bytes, its outputs and its workspace need fit.  The three streams
+ *                          (cudaStream_t as void*) must differ from each other and belong to the
+ *                          current device.  Allocates no device memory (host bookkeeping and CUDA
+ *                          events only).  *out receives the handle.
+ *   soar_pipeline_run      enqueues the n matrices `mats` (host memory, read before the call returns).
+ *                          Host buffers should be page-locked; they are valid once
+ *                          soar_pipeline_synchronize (or a synchronize of the third stream) returns.
+ *                          col_weights: NULL, or n device pointers (`cols` floats each, as in
+ *                          soar_quantize_weighted; a NULL entry means unweighted); slots used with
+ *                          weights need a workspace of soar_weighted_workspace_bytes().  Every
+ *                          matrix is checked against every rule of soar_quantize and against the
+ *                          slot capacities before anything is enqueued.
+ *   soar_pipeline_synchronize  blocks the calling host thread until everything enqueued so far has
+ *                          landed in the host buffers.
+ *   soar_pipeline_destroy  waits for the pipeline's work, then releases its events.
+ * Not thread-safe: one host thread drives a pipeline at a time.
+ */
+typedef struct soar_slot {
+  soar_staging dev;          /* device buffers of the slot (see soar_staging)                         */
+  size_t W_bytes;            /* capacity of dev.W                                                      */
+  size_t packed_bytes;       /* capacity of dev.packed                                                 */
+  size_t scales_bytes;       /* capacity of dev.scales (0 when NULL)                                   */
+  size_t scales_sw_bytes;    /* capacity of dev.scales_sw (0 when NULL)                                */
+} soar_slot;
+
+typedef struct soar_host_matrix {
+  const void* W_host;              /* rows x cols bf16, row stride ld elements                         */
+  int64_t rows, cols, ld;
+  void* out_fp4_packed_host;       /* rows*cols/2 bytes                                                */
+  void* out_e4m3_scales_host;      /* rows*cols/16 bytes, or NULL when the layout is not requested     */
+  void* out_e4m3_scales_sw_host;   /* soar_swizzled_scale_bytes(), or NULL                             */
+  float* out_global_host;          /* one float                                                        */
+  soar_result* out_result_host;    /* or NULL                                                          */
+} soar_host_matrix;
+
+typedef struct soar_pipeline soar_pipeline;
+int soar_pipeline_create(soar_pipeline** out, const soar_slot* slots, int n_slots, void* stream_h2d,
+                         void* stream_compute, void* stream_d2h);
+int soar_pipeline_run(soar_pipeline* pipe, const soar_host_matrix* mats, int n, const soar_cfg* cfg,
+                      const float* const* col_weights);
+int soar_pipeline_synchronize(soar_pipeline* pipe);
+void soar_pipeline_destroy(soar_pipeline* pipe);
 
 /*
  * Reconstruction error of a stored NVFP4 triple against W (Eq. 3 and Eq. 4):

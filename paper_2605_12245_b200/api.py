@@ -30,7 +30,8 @@ EXPORTS = (
     "soar_trace_begin", "soar_trace_end", "soar_quantize_static", "soar_selftest_reciprocal",
     "soar_batch_workspace_bytes", "soar_quantize_batch",
     "soar_weighted_workspace_bytes", "soar_quantize_weighted", "soar_dequant_error_weighted",
-    "soar_quantize_stage",
+    "soar_quantize_stage", "soar_pipeline_create", "soar_pipeline_run", "soar_pipeline_synchronize",
+    "soar_pipeline_destroy",
 )
 
 
@@ -128,6 +129,15 @@ def lib() -> C.CDLL:
         L.soar_quantize_stage.restype = C.c_int
         L.soar_quantize_stage.argtypes = [C.POINTER(SoarTensorDesc), C.c_int, C.POINTER(SoarCfg), vp, C.c_size_t,
                                           C.c_int, vp]
+        L.soar_pipeline_create.restype = C.c_int
+        L.soar_pipeline_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(SoarSlot), C.c_int, vp, vp, vp]
+        L.soar_pipeline_run.restype = C.c_int
+        L.soar_pipeline_run.argtypes = [vp, C.POINTER(SoarHostMatrix), C.c_int, C.POINTER(SoarCfg),
+                                        C.POINTER(C.c_void_p)]
+        L.soar_pipeline_synchronize.restype = C.c_int
+        L.soar_pipeline_synchronize.argtypes = [vp]
+        L.soar_pipeline_destroy.restype = None
+        L.soar_pipeline_destroy.argtypes = [vp]
         L.soar_selftest_reciprocal.restype = C.c_int
         L.soar_selftest_reciprocal.argtypes = [C.c_int, C.c_int, vp, vp]
         L.soar_trace_begin.restype = C.c_int
@@ -173,13 +183,24 @@ def _ptr(t):
 
 def _stream_ptr(stream):
     s = torch.cuda.current_stream() if stream is None else stream
+    if s.device.index != torch.cuda.current_device():
+        raise SoarError(f"stream belongs to cuda:{s.device.index} but the current device is "
+                        f"cuda:{torch.cuda.current_device()}")
     return C.c_void_p(s.cuda_stream)
 
 
 def _require_cuda(*tensors):
+    """Every tensor must live on the current CUDA device: the library launches there, on a stream of that
+    device, and a pointer into another GPU's memory would reach kernels that cannot address it."""
+    cur = torch.cuda.current_device() if torch.cuda.is_available() else None
     for t in tensors:
-        if t is not None and not t.is_cuda:
+        if t is None:
+            continue
+        if not t.is_cuda:
             raise SoarError("device pointers required: tensor is not on a CUDA device")
+        if t.device.index != cur:
+            raise SoarError(f"tensor lives on cuda:{t.device.index} but the current device is cuda:{cur}: "
+                            "make the tensor's device current (torch.cuda.device) before the call")
 
 
 @dataclass
@@ -410,27 +431,57 @@ def soar_quantize_host(host: HostBuffers, cfg: SoarCfg, dev_W: torch.Tensor, dev
     _check(rc, "soar_quantize_host")
 
 
+class SoarSlot(C.Structure):
+    """Mirror of ``soar_slot``."""
+
+    _fields_ = [("dev", SoarStaging), ("W_bytes", C.c_size_t), ("packed_bytes", C.c_size_t),
+                ("scales_bytes", C.c_size_t), ("scales_sw_bytes", C.c_size_t)]
+
+
+class SoarHostMatrix(C.Structure):
+    """Mirror of ``soar_host_matrix``."""
+
+    _fields_ = [("W_host", C.c_void_p), ("rows", C.c_int64), ("cols", C.c_int64), ("ld", C.c_int64),
+                ("out_fp4_packed_host", C.c_void_p), ("out_e4m3_scales_host", C.c_void_p),
+                ("out_e4m3_scales_sw_host", C.c_void_p), ("out_global_host", C.c_void_p),
+                ("out_result_host", C.c_void_p)]
+
+
 class HostPipeline:
-    """Quantizes matrices that live in pinned host memory with the three legs overlapped:
-    host-to-device copies on one stream, ``soar_quantize`` on a second, device-to-host copies of
-    the results on a third, chained by events over ``depth`` device staging slots sized for the
-    largest matrix.  Stream plumbing only; the work is ``soar_quantize`` (``soar_quantize_weighted``
-    when column weights are given)."""
+    """``soar_pipeline_*`` of the C ABI: quantizes matrices that live in pinned host memory with the
+    copies in, the quantizer and the copies out overlapped on three streams over ``depth`` device
+    staging slots sized for the largest matrix.  This class allocates the slots and the streams and
+    marshals the lists; the chaining is the library's."""
 
     def __init__(self, shapes, cfg: SoarCfg, depth: int = 3, device="cuda", weighted: bool = False):
         self.cfg = cfg
         self.weighted = weighted
         rows, cols = max(shapes, key=lambda rc: rc[0] * rc[1])
-        self.slots = []
-        for _ in range(depth):
-            self.slots.append(dict(
-                W=torch.empty(rows * cols, dtype=torch.bfloat16, device=device),
-                out=alloc_buffers(rows, cols, cfg, device, weighted=weighted),
-                loaded=torch.cuda.Event(), computed=torch.cuda.Event(), stored=torch.cuda.Event()))
+        sw_bytes = max(soar_swizzled_scale_bytes(r, c) for r, c in shapes) if cfg.scale_layout & SCALES_SWIZZLED else 0
+        ws_bytes = max((soar_weighted_workspace_bytes if weighted else soar_workspace_bytes)(r, c, cfg)
+                       for r, c in shapes)
+        self._keep = []                                  # the slots' tensors
+        slots = (SoarSlot * depth)()
+        for i in range(depth):
+            W = torch.empty(rows * cols, dtype=torch.bfloat16, device=device)
+            out = alloc_buffers(rows, cols, cfg, device, weighted=weighted)
+            if out.scales_sw is not None and out.scales_sw.numel() < sw_bytes:
+                out.scales_sw = torch.empty(sw_bytes, dtype=torch.uint8, device=device)
+            if out.workspace.numel() < ws_bytes:
+                out.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
+            _require_cuda(W, out.packed, out.scales, out.scales_sw, out.alpha, out.result, out.workspace)
+            self._keep.append((W, out))
+            nul = lambda t: None if t is None else t.data_ptr()  # noqa: E731
+            slots[i] = SoarSlot(
+                SoarStaging(W.data_ptr(), out.packed.data_ptr(), nul(out.scales), nul(out.scales_sw),
+                            out.alpha.data_ptr(), out.result.data_ptr(), out.workspace.data_ptr(),
+                            out.workspace.numel()),
+                W.numel() * 2, out.packed.numel(), 0 if out.scales is None else out.scales.numel(),
+                0 if out.scales_sw is None else out.scales_sw.numel())
         self.h2d, self.compute, self.d2h = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
-        for sl in self.slots:
-            sl["stored"].record(self.d2h)
-        self._next = 0      # slots are taken in turn across calls, so a new list starts on the slot freed longest ago
+        self._handle = C.c_void_p()
+        _check(lib().soar_pipeline_create(C.byref(self._handle), slots, depth, _stream_ptr(self.h2d),
+                                          _stream_ptr(self.compute), _stream_ptr(self.d2h)), "soar_pipeline_create")
 
     def run(self, hosts, col_weights=None) -> None:
         """Enqueue the whole list (``HostBuffers`` each); results are in the host buffers once
@@ -440,41 +491,32 @@ class HostPipeline:
         pipeline must have been built with ``weighted=True``)."""
         if col_weights is not None and not self.weighted:
             raise SoarError("this pipeline's workspaces are not sized for the weighted objective")
-        for k, hb in enumerate(hosts):
-            sl = self.slots[self._next % len(self.slots)]
-            self._next += 1
+        n = len(hosts)
+        mats = (SoarHostMatrix * n)()
+        nul = lambda t: None if t is None else t.data_ptr()  # noqa: E731
+        for i, hb in enumerate(hosts):
             rows, cols = hb.W.shape
-            n = rows * cols
-            big = sl["out"]
-            W = sl["W"][:n].view(rows, cols)
-            view = QuantBuffers(
-                packed=big.packed.view(-1)[: n // 2].view(rows, cols // 2),
-                scales=None if big.scales is None else big.scales.view(-1)[: n // 16].view(rows, cols // 16),
-                scales_sw=None if big.scales_sw is None else big.scales_sw[: soar_swizzled_scale_bytes(rows, cols)],
-                alpha=big.alpha, result=big.result, workspace=big.workspace)
-            self.h2d.wait_event(sl["stored"])            # the slot's previous results have left
-            with torch.cuda.stream(self.h2d):
-                W.copy_(hb.W, non_blocking=True)
-                sl["loaded"].record(self.h2d)
-            self.compute.wait_event(sl["loaded"])
-            if col_weights is None:
-                soar_quantize(W, self.cfg, view, self.compute)
-            else:
-                soar_quantize_weighted(W, col_weights[k], self.cfg, view, self.compute)
-            sl["computed"].record(self.compute)
-            self.d2h.wait_event(sl["computed"])
-            with torch.cuda.stream(self.d2h):
-                hb.packed.copy_(view.packed, non_blocking=True)
-                if view.scales is not None:
-                    hb.scales.copy_(view.scales, non_blocking=True)
-                if view.scales_sw is not None:
-                    hb.scales_sw.copy_(view.scales_sw, non_blocking=True)
-                hb.alpha.copy_(view.alpha, non_blocking=True)
-                hb.result.copy_(view.result, non_blocking=True)
-                sl["stored"].record(self.d2h)
+            mats[i] = SoarHostMatrix(hb.W.data_ptr(), rows, cols, hb.W.stride(0), hb.packed.data_ptr(), nul(hb.scales),
+                                     nul(hb.scales_sw), hb.alpha.data_ptr(), hb.result.data_ptr())
+        wp = None
+        if col_weights is not None:
+            _require_cuda(*col_weights)
+            wp = (C.c_void_p * n)(*[h.data_ptr() for h in col_weights])
+        _check(lib().soar_pipeline_run(self._handle, mats, n, C.byref(self.cfg), wp), "soar_pipeline_run")
 
     def synchronize(self) -> None:
-        self.d2h.synchronize()
+        _check(lib().soar_pipeline_synchronize(self._handle), "soar_pipeline_synchronize")
+
+    def close(self) -> None:
+        if self._handle:
+            lib().soar_pipeline_destroy(self._handle)
+            self._handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def soar_selftest_reciprocal(lo_exp: int = 2, hi_exp: int = 252, stream=None) -> int:

@@ -45,6 +45,7 @@
 #include <string.h>
 
 #include <mutex>
+#include <new>
 #include <vector>
 
 #include "soar.h"
@@ -2166,6 +2167,9 @@ int soar_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, co
 // Built-in scratch of soar_quantize_static.  In host code the symbol below is only a handle:
 // the device address comes from cudaGetSymbolAddress, looked up once per device.
 static __device__ __align__(256) unsigned char g_static_scratch[SOAR_STATIC_SCRATCH_BYTES];
+// the largest accepted matrix needs exactly this much: the header, 8 bytes of state and one scale byte per block
+static_assert(kWsFixedBytes + (SOAR_STATIC_MAX_ELEMENTS / 16) * (sizeof(uint2) + 1) == SOAR_STATIC_SCRATCH_BYTES,
+              "SOAR_STATIC_SCRATCH_BYTES does not match the workspace of SOAR_STATIC_MAX_ELEMENTS");
 
 namespace {
 std::mutex g_static_mu;
@@ -2380,6 +2384,13 @@ int soar_quantize_host(const void* W_host, int64_t rows, int64_t cols, int64_t l
   if (want_sw && (out_e4m3_scales_sw_host == nullptr || dev->scales_sw == nullptr)) return SOAR_ERR_INVALID_ARG;
   if (dev->packed == nullptr || dev->alpha == nullptr) return SOAR_ERR_INVALID_ARG;
   if (out_result_host != nullptr && dev->result == nullptr) return SOAR_ERR_INVALID_ARG;
+  // every check soar_quantize would make on the staging buffers, before anything is enqueued
+  rc = check_shape(dev->W, rows, cols, ld);
+  if (rc != SOAR_OK) return rc;
+  if (reinterpret_cast<uintptr_t>(dev->packed) % 16 != 0) return SOAR_ERR_UNSUPPORTED;
+  const size_t need = soar_workspace_bytes(rows, cols, cfg);
+  if (dev->workspace == nullptr || need == 0 || dev->workspace_bytes < need) return SOAR_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(dev->workspace) % 256 != 0) return SOAR_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t in_bytes = static_cast<size_t>(rows) * static_cast<size_t>(ld) * 2;
   if (cudaMemcpyAsync(dev->W, W_host, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SOAR_ERR_CUDA;
@@ -2398,6 +2409,154 @@ int soar_quantize_host(const void* W_host, int64_t rows, int64_t cols, int64_t l
     ok = ok && cudaMemcpyAsync(out_result_host, dev->result, sizeof(soar_result), cudaMemcpyDeviceToHost, st) ==
                    cudaSuccess;
   return ok ? SOAR_OK : SOAR_ERR_CUDA;
+}
+
+}  // extern "C"
+
+// Host bookkeeping of a pipeline: the slots, three events per slot, the streams and whose turn it is.
+struct soar_pipeline {
+  std::vector<soar_slot> slots;
+  std::vector<cudaEvent_t> loaded, computed, stored;   // per slot: input landed, quantized, results left
+  cudaStream_t h2d, compute, d2h;
+  size_t next;
+};
+
+namespace {
+void release_events(soar_pipeline* p) {
+  for (cudaEvent_t e : p->loaded) cudaEventDestroy(e);
+  for (cudaEvent_t e : p->computed) cudaEventDestroy(e);
+  for (cudaEvent_t e : p->stored) cudaEventDestroy(e);
+}
+
+// Every rule a matrix must meet to go through slot `sl` (nothing is enqueued before all matrices pass).
+int check_host_matrix(const soar_host_matrix& m, const soar_slot& sl, const soar_cfg* cfg, bool weighted) {
+  if (m.W_host == nullptr || m.out_fp4_packed_host == nullptr || m.out_global_host == nullptr)
+    return SOAR_ERR_INVALID_ARG;
+  int rc = check_shape(sl.dev.W, m.rows, m.cols, m.ld);
+  if (rc != SOAR_OK) return rc;
+  const bool want_lin = (cfg->scale_layout & SOAR_SCALES_LINEAR) != 0;
+  const bool want_sw = (cfg->scale_layout & SOAR_SCALES_SWIZZLED) != 0;
+  if (want_lin && (m.out_e4m3_scales_host == nullptr || sl.dev.scales == nullptr)) return SOAR_ERR_INVALID_ARG;
+  if (want_sw && (m.out_e4m3_scales_sw_host == nullptr || sl.dev.scales_sw == nullptr)) return SOAR_ERR_INVALID_ARG;
+  if (m.out_result_host != nullptr && sl.dev.result == nullptr) return SOAR_ERR_INVALID_ARG;
+  const size_t n = static_cast<size_t>(m.rows) * static_cast<size_t>(m.cols);
+  if (static_cast<size_t>(m.rows) * static_cast<size_t>(m.ld) * 2 > sl.W_bytes || n / 2 > sl.packed_bytes)
+    return SOAR_ERR_TOO_LARGE;
+  if (want_lin && n / 16 > sl.scales_bytes) return SOAR_ERR_TOO_LARGE;
+  if (want_sw && soar_swizzled_scale_bytes(m.rows, m.cols) > sl.scales_sw_bytes) return SOAR_ERR_TOO_LARGE;
+  const size_t need = weighted ? soar_weighted_workspace_bytes(m.rows, m.cols, cfg)
+                               : soar_workspace_bytes(m.rows, m.cols, cfg);
+  if (need == 0 || sl.dev.workspace_bytes < need) return SOAR_ERR_WORKSPACE;
+  return SOAR_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int soar_pipeline_create(soar_pipeline** out, const soar_slot* slots, int n_slots, void* stream_h2d,
+                         void* stream_compute, void* stream_d2h) {
+  if (out == nullptr || slots == nullptr || n_slots < 1) return SOAR_ERR_INVALID_ARG;
+  if (stream_h2d == stream_compute || stream_compute == stream_d2h || stream_h2d == stream_d2h)
+    return SOAR_ERR_INVALID_ARG;
+  for (int i = 0; i < n_slots; ++i) {
+    const soar_staging& d = slots[i].dev;
+    if (d.W == nullptr || d.packed == nullptr || d.alpha == nullptr || d.workspace == nullptr)
+      return SOAR_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d.W) % 16 != 0 || reinterpret_cast<uintptr_t>(d.packed) % 16 != 0 ||
+        reinterpret_cast<uintptr_t>(d.workspace) % 256 != 0)
+      return SOAR_ERR_UNSUPPORTED;
+  }
+  soar_pipeline* p = new (std::nothrow) soar_pipeline();
+  if (p == nullptr) return SOAR_ERR_INVALID_ARG;
+  p->slots.assign(slots, slots + n_slots);
+  p->h2d = static_cast<cudaStream_t>(stream_h2d);
+  p->compute = static_cast<cudaStream_t>(stream_compute);
+  p->d2h = static_cast<cudaStream_t>(stream_d2h);
+  p->next = 0;
+  bool ok = true;
+  for (int i = 0; i < 3 * n_slots && ok; ++i) {
+    cudaEvent_t e;
+    ok = cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+    if (ok) (i % 3 == 0 ? p->loaded : i % 3 == 1 ? p->computed : p->stored).push_back(e);
+  }
+  // a slot is free from the start: its "results left" event is recorded once on the third stream
+  for (size_t i = 0; i < p->stored.size() && ok; ++i) ok = cudaEventRecord(p->stored[i], p->d2h) == cudaSuccess;
+  if (!ok || p->stored.size() != static_cast<size_t>(n_slots)) {
+    release_events(p);
+    delete p;
+    return SOAR_ERR_CUDA;
+  }
+  *out = p;
+  return SOAR_OK;
+}
+
+int soar_pipeline_run(soar_pipeline* pipe, const soar_host_matrix* mats, int n, const soar_cfg* cfg,
+                      const float* const* col_weights) {
+  if (pipe == nullptr || mats == nullptr || n < 0) return SOAR_ERR_INVALID_ARG;
+  int rc = check_cfg(cfg);
+  if (rc != SOAR_OK) return rc;
+  const size_t ns = pipe->slots.size();
+  for (int i = 0; i < n; ++i) {   // everything is checked before anything is enqueued
+    const float* h = col_weights != nullptr ? col_weights[i] : nullptr;
+    if (h != nullptr && reinterpret_cast<uintptr_t>(h) % 16 != 0) return SOAR_ERR_UNSUPPORTED;
+    rc = check_host_matrix(mats[i], pipe->slots[(pipe->next + static_cast<size_t>(i)) % ns], cfg, h != nullptr);
+    if (rc != SOAR_OK) return rc;
+  }
+  const bool want_lin = (cfg->scale_layout & SOAR_SCALES_LINEAR) != 0;
+  const bool want_sw = (cfg->scale_layout & SOAR_SCALES_SWIZZLED) != 0;
+  for (int i = 0; i < n; ++i) {
+    const soar_host_matrix& m = mats[i];
+    const size_t si = pipe->next % ns;
+    ++pipe->next;
+    const soar_staging& d = pipe->slots[si].dev;
+    const float* h = col_weights != nullptr ? col_weights[i] : nullptr;
+    // copy in, once the slot's previous results have left
+    bool ok = cudaStreamWaitEvent(pipe->h2d, pipe->stored[si], 0) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(d.W, m.W_host, static_cast<size_t>(m.rows) * static_cast<size_t>(m.ld) * 2,
+                               cudaMemcpyHostToDevice, pipe->h2d) == cudaSuccess;
+    ok = ok && cudaEventRecord(pipe->loaded[si], pipe->h2d) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(pipe->compute, pipe->loaded[si], 0) == cudaSuccess;
+    if (!ok) return SOAR_ERR_CUDA;
+    soar_result* res = m.out_result_host != nullptr ? d.result : nullptr;
+    rc = h == nullptr ? soar_quantize(d.W, m.rows, m.cols, m.ld, cfg, d.packed, d.scales, d.scales_sw, d.alpha,
+                                      d.workspace, d.workspace_bytes, res, pipe->compute)
+                      : soar_quantize_weighted(d.W, m.rows, m.cols, m.ld, h, cfg, d.packed, d.scales, d.scales_sw,
+                                               d.alpha, d.workspace, d.workspace_bytes, res, pipe->compute);
+    if (rc != SOAR_OK) return rc;
+    ok = cudaEventRecord(pipe->computed[si], pipe->compute) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(pipe->d2h, pipe->computed[si], 0) == cudaSuccess;
+    const size_t ne = static_cast<size_t>(m.rows) * static_cast<size_t>(m.cols);
+    ok = ok && cudaMemcpyAsync(m.out_fp4_packed_host, d.packed, ne / 2, cudaMemcpyDeviceToHost, pipe->d2h) ==
+                   cudaSuccess;
+    if (want_lin)
+      ok = ok && cudaMemcpyAsync(m.out_e4m3_scales_host, d.scales, ne / 16, cudaMemcpyDeviceToHost, pipe->d2h) ==
+                     cudaSuccess;
+    if (want_sw)
+      ok = ok && cudaMemcpyAsync(m.out_e4m3_scales_sw_host, d.scales_sw, soar_swizzled_scale_bytes(m.rows, m.cols),
+                                 cudaMemcpyDeviceToHost, pipe->d2h) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(m.out_global_host, d.alpha, sizeof(float), cudaMemcpyDeviceToHost, pipe->d2h) ==
+                   cudaSuccess;
+    if (res != nullptr)
+      ok = ok && cudaMemcpyAsync(m.out_result_host, d.result, sizeof(soar_result), cudaMemcpyDeviceToHost,
+                                 pipe->d2h) == cudaSuccess;
+    ok = ok && cudaEventRecord(pipe->stored[si], pipe->d2h) == cudaSuccess;
+    if (!ok) return SOAR_ERR_CUDA;
+  }
+  return SOAR_OK;
+}
+
+int soar_pipeline_synchronize(soar_pipeline* pipe) {
+  if (pipe == nullptr) return SOAR_ERR_INVALID_ARG;
+  return cudaStreamSynchronize(pipe->d2h) == cudaSuccess ? SOAR_OK : SOAR_ERR_CUDA;
+}
+
+void soar_pipeline_destroy(soar_pipeline* pipe) {
+  if (pipe == nullptr) return;
+  cudaStreamSynchronize(pipe->h2d);
+  cudaStreamSynchronize(pipe->compute);
+  cudaStreamSynchronize(pipe->d2h);
+  release_events(pipe);
+  delete pipe;
 }
 
 int soar_selftest_reciprocal(int lo_exp, int hi_exp, unsigned long long* out_mismatches, void* stream) {
@@ -2454,7 +2613,7 @@ const char* soar_status_string(int status) {
     case SOAR_ERR_UNSUPPORTED: return "unsupported shape, alignment or block size";
     case SOAR_ERR_WORKSPACE: return "workspace missing or too small";
     case SOAR_ERR_CUDA: return "CUDA runtime or launch error";
-    case SOAR_ERR_TOO_LARGE: return "matrix exceeds the built-in scratch of soar_quantize_static";
+    case SOAR_ERR_TOO_LARGE: return "matrix exceeds the built-in scratch of soar_quantize_static or a pipeline slot";
     default: return "unknown status";
   }
 }

@@ -59,6 +59,21 @@ def run_gpu(w_bits: np.ndarray, cfg, ld: int | None = None) -> GpuOut:
     return GpuOut(out.packed.cpu().numpy(), scales, float(out.alpha.cpu()[0]), res, out)
 
 
+def run_gpu_batch(ws, cfg, lds=None) -> list:
+    """One ``soar_quantize_batch`` call over the matrices ``ws`` (uint16 bit patterns each): the launch
+    shape the benchmark times, every persistent CTA walking from one matrix into the next."""
+    dev = [to_device(w, None if lds is None else lds[i]) for i, w in enumerate(ws)]
+    outs = [api.alloc_buffers(w.shape[0], w.shape[1], cfg) for w in ws]
+    api.soar_quantize_batch(dev, cfg, outs)
+    torch.cuda.synchronize()
+    del dev
+    got = []
+    for o in outs:
+        scales = o.scales.cpu().numpy() if o.scales is not None else None
+        got.append(GpuOut(o.packed.cpu().numpy(), scales, float(o.alpha.cpu()[0]), o.read_result(), o))
+    return got
+
+
 @dataclass
 class Report:
     blocks: int

@@ -109,3 +109,81 @@ def test_config4_largest_tensor():
     W = P.to_device(w)
     e = api.soar_dequant_error(W, gpu.buffers.packed, gpu.buffers.scales, gpu.buffers.alpha).cpu().numpy()
     assert e[0] == pytest.approx(sse, rel=1e-9) and e[1] == pytest.approx(res.sumsq, rel=1e-13)
+
+
+# ---- the launch shape the benchmark times: one batched call, CTAs walking from tensor to tensor
+
+def _batch_against_oracle(wl_name, ws, names, cfg, ref_cfg):
+    got = P.run_gpu_batch(ws, cfg)
+    for name, w, g in zip(names, ws, got):          # the oracle per tensor, so that a failure names it
+        g.buffers = None
+        rep = P.assert_parity(g, R.quantize(w, ref_cfg))
+        print(wl_name, name, rep)
+
+
+def test_config4_whole_layer_in_one_batched_call_paper_preset_and_single_pass():
+    """All seven tensors of the Llama-3-70B-shaped layer through soar_quantize_batch, exactly as
+    bench.py launches them, every tensor element by element against the oracle."""
+    wl = WL.config4()
+    ws = [WL.generate(wl, i) for i in range(len(wl.tensors))]
+    names = [t.name for t in wl.tensors]
+    cfg, ref_cfg = P.cfg_pair()
+    _batch_against_oracle("config4 paper", ws, names, cfg, ref_cfg)
+    torch.cuda.empty_cache()
+    cfg, ref_cfg = P.cfg_pair(max_iters=1, early_stop_rel=0.0, n_dq=2, n_beta=1)
+    _batch_against_oracle("config4 single pass", ws, names, cfg, ref_cfg)
+
+
+@pytest.mark.parametrize("cfgkw", [
+    dict(),                                                   # the paper's preset
+    dict(max_iters=1, early_stop_rel=0.0, n_dq=2, n_beta=1),  # single pass
+    dict(max_iters=0),                                        # Eq. 1-3 only
+    dict(max_iters=2, early_stop_rel=0.0, n_dq=4, n_beta=1),  # several codes on one rounding
+])
+def test_batch_of_mid_size_tensors_hands_over_inside_every_kernel(cfgkw):
+    """Nineteen matrices, sixteen of them several hundred tiles long: the first launch group has
+    thousands of tiles, far more than any kernel's grid, so in every pass (forward and backward)
+    each CTA leaves one matrix and enters the next in mid-sequence.  Same bytes as separate calls,
+    and the oracle's."""
+    shapes = [(520 + 24 * i, 4096) if i % 2 == 0 else (1040 + 8 * i, 2064) for i in range(16)] + \
+             [(1, 16), (300, 4096), (5, 48)]
+    ws = [WL.small_case(r, c, 700 + i, dist=("laplace" if i % 3 == 0 else "student_t4"),
+                        outlier_entry_frac=0.002 * (i % 2), outlier_scale=40.0) for i, (r, c) in enumerate(shapes)]
+    ws.insert(3, WL.small_case(1, 16, 777))                  # a one-block matrix between two long ones
+    ws[7] = np.zeros_like(ws[7])                             # an all-zero matrix in mid-sequence
+    cfg, ref_cfg = P.cfg_pair(**cfgkw)
+    lds = [w.shape[1] + (40 if i == 5 else 0) for i, w in enumerate(ws)]
+    got = P.run_gpu_batch(ws, cfg, lds)
+    for i, (w, g) in enumerate(zip(ws, got)):
+        one = P.run_gpu(w, cfg, lds[i])
+        assert g.result.status == one.result.status and g.result.iters_run == one.result.iters_run, i
+        assert np.array_equal(g.packed, one.packed) and np.array_equal(g.scales, one.scales), i
+        assert g.alpha == one.alpha, i
+        assert g.result.sse == pytest.approx(one.result.sse, rel=1e-12), i
+        if g.result.status == 0:
+            P.assert_parity(g, R.quantize(w, ref_cfg))
+        else:
+            assert g.result.status == api.STATUS_ZERO_TENSOR and not g.scales.any()
+
+
+def test_config3_whole_layer_batched_and_tensors_of_the_first_and_last_layer():
+    """Layer 17 of the 36-layer Qwen3-8B-shaped model through the batched call, all seven tensors against
+    the oracle; k of layer 0 and of layer 35 (each layer has its own seed) through single calls."""
+    wl = WL.config3_layer(17)
+    ws = [WL.generate(wl, i) for i in range(len(wl.tensors))]
+    cfg, ref_cfg = P.cfg_pair()
+    _batch_against_oracle(wl.name, ws, [t.name for t in wl.tensors], cfg, ref_cfg)
+    for layer in (0, 35):
+        wl = WL.config3_layer(layer)
+        w = WL.generate(wl, 1)
+        print(wl.name, wl.tensors[1].name, P.assert_parity(P.run_gpu(w, cfg), R.quantize(w, ref_cfg)))
+
+
+def test_config5_candidate_sweep_points_with_fifteen_iterations():
+    """The sweep of config 5 at T = 15 (early stop off), on the first 1024 rows."""
+    w = WL.generate(WL.config5(), 0, 0, 1024)
+    for pairs in (1, 4, 8, 16, 32):
+        n_dq = min(2, pairs)
+        cfg, ref_cfg = P.cfg_pair(max_iters=15, early_stop_rel=0.0, n_dq=n_dq, n_beta=pairs // n_dq)
+        rep = P.assert_parity(P.run_gpu(w, cfg), R.quantize(w, ref_cfg))
+        print("config5 rows 0..1023, T = 15, pairs", pairs, rep)

@@ -225,6 +225,21 @@ def test_host_entry_point_and_launch_trace():
     assert all(v[1] > 0 for v in trace.values())
 
 
+def test_host_entry_point_enqueues_nothing_on_an_argument_error():
+    """A workspace that is too small is refused before the copy of W into the staging buffer starts."""
+    w = WL.small_case(64, 512, 92)
+    cfg, _ = P.cfg_pair(max_iters=2)
+    hb = api.alloc_host_buffers(64, 512, cfg)
+    hb.W.copy_(torch.from_numpy(w.view(np.int16)).view(torch.bfloat16))
+    dev_W = torch.full((64, 512), 7.0, dtype=torch.bfloat16, device="cuda")
+    dev = api.alloc_buffers(64, 512, cfg)
+    dev.workspace = dev.workspace[:1024]
+    with pytest.raises(api.SoarError, match="workspace"):
+        api.soar_quantize_host(hb, cfg, dev_W, dev)
+    torch.cuda.synchronize()
+    assert bool((dev_W == 7.0).all())
+
+
 def test_host_pipeline_returns_what_direct_calls_return():
     """Seven matrices through three staging slots: every slot is reused, sizes differ."""
     shapes = [(64, 1024), (16, 256), (300, 512), (8, 4096), (130, 2064), (1, 16), (257, 1024)]

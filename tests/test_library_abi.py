@@ -54,7 +54,8 @@ def test_python_mirrors_of_the_public_structs_match_the_header(tmp_path):
     import subprocess
     structs = {"soar_cfg": api.SoarCfg, "soar_result": api.SoarResult, "soar_tensor_desc": api.SoarTensorDesc,
                "soar_staging": api.SoarStaging, "soar_trace_entry": api.SoarTraceEntry,
-               "soar_workspace_header": api.SoarWorkspaceHeader}
+               "soar_workspace_header": api.SoarWorkspaceHeader, "soar_slot": api.SoarSlot,
+               "soar_host_matrix": api.SoarHostMatrix}
     lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "soar.h"', "int main(void) {"]
     for cname, py in structs.items():
         lines.append(f'  printf("{cname} %zu\\n", sizeof({cname}));')

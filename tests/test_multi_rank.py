@@ -143,3 +143,30 @@ def test_row_sharded_schedule_combines_every_written_entry_exactly_once():
     RS.header_view(header, "amax_bits").fill_(0x3F80)
     h = api.SoarWorkspaceHeader.from_buffer_copy(bytes(raw[:C.sizeof(api.SoarWorkspaceHeader)]))
     assert h.den[3] == 2.5 and h.amax_bits == 0x3F80 and h.num[3] == 0.0
+
+
+def test_bench_starts_its_own_ranks_when_given_a_rank_count():
+    """``bench.py --gpus 2`` as a plain process starts two ranks itself; the dry run keeps them on CPU
+    (gloo) and reports how many ranks met."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--dry-run"],
+                         capture_output=True, text=True, env=env, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads([l for l in out.stdout.splitlines() if l.startswith("{")][-1])
+    assert line["n_gpus"] == 2 and line["ranks_seen"] == 2 and line["ms_per_step"] == 2.0
+
+
+def test_launcher_command_is_one_rank_per_gpu_on_the_loopback_address():
+    import importlib.util
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    spec = importlib.util.spec_from_file_location("bench_module", os.path.join(root, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    cmd = bench.launcher_command(4, ["--gpus", "4", "--steps", "2"], 29517)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=4" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29517"
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "2"]
