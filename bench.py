@@ -392,6 +392,20 @@ def run_ours(args):
     value = world * 2.0 * elements / (ms * 1e-3) / 1e9
     launches = sum(v[0] for v in trace.values())
 
+    # ---- the timed batch's outputs against one soar_quantize call per tensor (same bytes expected)
+    bad = []
+    for i, (W, o) in enumerate(zip(dev_w, outs)):
+        one = api.soar_quantize(W, cfg)
+        torch.cuda.synchronize()
+        if not (torch.equal(one.packed, o.packed) and torch.equal(one.scales, o.scales) and torch.equal(one.alpha, o.alpha)
+                and one.read_result().iters_run == iters[i]):
+            bad.append(i)
+        del one
+    outputs_checked = dict(tensors=len(outs), differing_from_single_calls=bad)
+    packed0 = outs[0].packed.cpu()            # the later sections reuse the output buffers
+    if bad:
+        raise SystemExit(f"batched outputs differ from per-tensor calls for tensors {bad}")
+
     # ---- roofline of the dominant kernel: its algorithmic bytes over its measured device time, against the
     # measured HBM copy bandwidth; beside it the issue-slot side from the committed profile
     dom = max(trace, key=lambda k: trace[k][1])
@@ -484,19 +498,6 @@ def run_ours(args):
                                  frac_of_measured_hbm=k_bytes / (k_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]))
         extra["sweep_dq"] = rows_out
 
-    # ---- the timed batch's outputs against one soar_quantize call per tensor (same bytes expected)
-    bad = []
-    for i, (W, o) in enumerate(zip(dev_w, outs)):
-        one = api.soar_quantize(W, cfg)
-        torch.cuda.synchronize()
-        if not (torch.equal(one.packed, o.packed) and torch.equal(one.scales, o.scales) and torch.equal(one.alpha, o.alpha)
-                and one.read_result().iters_run == iters[i]):
-            bad.append(i)
-        del one
-    outputs_checked = dict(tensors=len(outs), differing_from_single_calls=bad)
-    if bad:
-        raise SystemExit(f"batched outputs differ from per-tensor calls for tensors {bad}")
-
     # ---- end to end through the C ABI's host-buffer pipeline (soar_pipeline_run): pinned host buffers in and out,
     # every copy inside the timed region
     import ctypes
@@ -531,7 +532,7 @@ def run_ours(args):
         # results must equal the resident-input run
         r_last = hosts[(len(wl.tensors) - 1) % len(hosts)].read_result()
         assert r_last.status == 0 and hosts[0].read_result().iters_run == iters[0]
-        assert torch.equal(hosts[0].packed, outs[0].packed.cpu())
+        assert torch.equal(hosts[0].packed, packed0)
         e2e = dict(value=world * 2.0 * elements / dt / 1e9, unit="GB/s", ms_per_step=dt * 1e3,
                    h2d_bytes_per_step=2 * elements,
                    d2h_bytes_per_step=elements // 2 + elements // 16 + len(wl.tensors) * (4 + ctypes_sizeof_result),

@@ -67,6 +67,17 @@ extern "C" {
 #define SOAR_FLAG_KEEP_BLOCK_SCALE 4   /* skip Eq. 6: candidate sets are centred on the stored scale
                                           (with KEEP_ALPHA: Sec. 3.3 (i),(ii) alone) */
 
+#define SOAR_FLAG_DETERMINISTIC 8       /* bit-identical results from run to run.  By default the tensor-wide
+                                          sums of Eq. 5 and of the error are binary64 additions in the order
+                                          the thread blocks finish, so their last bits, and through alpha in
+                                          rare cases a code, can differ between runs.  With this flag every
+                                          thread block stores its sums in a slot of its own and the next kernel
+                                          adds the slots in a fixed order.  Needs 56 KB more workspace per
+                                          matrix (soar_workspace_bytes accounts for it).  soar_quantize,
+                                          soar_quantize_batch, soar_quantize_host and the pipeline only:
+                                          soar_quantize_stage and soar_quantize_weighted return
+                                          SOAR_ERR_UNSUPPORTED */
+
 #define SOAR_MAX_ITERS 64
 #define SOAR_MAX_BETA 512
 #define SOAR_MAX_DQ 16
@@ -403,6 +414,18 @@ int soar_trace_end(soar_trace_entry* out, int capacity, int* count);
  * differ, into *out_mismatches (device, 8 bytes).  The full range takes about two seconds.
  */
 int soar_selftest_reciprocal(int lo_exp, int hi_exp, unsigned long long* out_mismatches, void* stream);
+
+/*
+ * Test hook for the kernels' bounded waits (no counterpart in the paper).  Every wait inside a
+ * kernel (a consumer warp waiting for the tile its producer fetches) counts its polls and gives
+ * up at a limit; the call then reports SOAR_STATUS_INTERNAL instead of hanging.  While the hook
+ * is on, kernels launched afterwards fetch no tiles at all, so their consumers' waits run to
+ * the limit (about four million polls, well under a second per kernel) with no copy in flight:
+ * the pass kernels then return, the remaining kernels of the call return at once,
+ * soar_result.status carries SOAR_STATUS_INTERNAL and the outputs are unspecified.  on = 0
+ * restores normal operation.  Process-wide; not for production use.
+ */
+int soar_debug_fail_waits(int on);
 
 /* Text for a host-side return value. */
 const char* soar_status_string(int status);

@@ -21,7 +21,7 @@ STATUS_ZERO_TENSOR, STATUS_NONFINITE, STATUS_RANGE, STATUS_INTERNAL = 1, 2, 4, 8
 STATUS_BAD_WEIGHT = 16
 SCALES_LINEAR, SCALES_SWIZZLED = 1, 2
 PRESET_PAPER, PRESET_SINGLE_PASS, PRESET_RTN, PRESET_CJSO_ONLY, PRESET_DSS_ONLY, PRESET_COUPLED_PAIR = 0, 1, 2, 3, 4, 5
-FLAG_COUPLED_SCALE, FLAG_KEEP_ALPHA, FLAG_KEEP_BLOCK_SCALE = 1, 2, 4
+FLAG_COUPLED_SCALE, FLAG_KEEP_ALPHA, FLAG_KEEP_BLOCK_SCALE, FLAG_DETERMINISTIC = 1, 2, 4, 8
 MAX_ITERS = 64
 
 EXPORTS = (
@@ -31,7 +31,7 @@ EXPORTS = (
     "soar_batch_workspace_bytes", "soar_quantize_batch",
     "soar_weighted_workspace_bytes", "soar_quantize_weighted", "soar_dequant_error_weighted",
     "soar_quantize_stage", "soar_pipeline_create", "soar_pipeline_run", "soar_pipeline_synchronize",
-    "soar_pipeline_destroy",
+    "soar_pipeline_destroy", "soar_debug_fail_waits",
 )
 
 
@@ -138,6 +138,8 @@ def lib() -> C.CDLL:
         L.soar_pipeline_synchronize.argtypes = [vp]
         L.soar_pipeline_destroy.restype = None
         L.soar_pipeline_destroy.argtypes = [vp]
+        L.soar_debug_fail_waits.restype = C.c_int
+        L.soar_debug_fail_waits.argtypes = [C.c_int]
         L.soar_selftest_reciprocal.restype = C.c_int
         L.soar_selftest_reciprocal.argtypes = [C.c_int, C.c_int, vp, vp]
         L.soar_trace_begin.restype = C.c_int
@@ -524,6 +526,11 @@ def soar_selftest_reciprocal(lo_exp: int = 2, hi_exp: int = 252, stream=None) ->
     out = torch.zeros(1, dtype=torch.int64, device="cuda")
     _check(lib().soar_selftest_reciprocal(lo_exp, hi_exp, _ptr(out), _stream_ptr(stream)), "soar_selftest_reciprocal")
     return int(out.cpu()[0])
+
+
+def soar_debug_fail_waits(on: bool) -> None:
+    """Test hook: while on, the kernels' waits for tiles run out (see ``soar_debug_fail_waits`` in soar.h)."""
+    _check(lib().soar_debug_fail_waits(1 if on else 0), "soar_debug_fail_waits")
 
 
 def soar_trace_begin() -> None:

@@ -86,7 +86,18 @@ static_assert(kWsFixedBytes == SOAR_WORKSPACE_HEADER_BYTES && sizeof(Ws) == size
 constexpr unsigned int kErrWait = 1u;     // a bounded wait gave up
 constexpr unsigned int kErrWeight = 2u;   // a column weight outside the accepted set
 
+// Deterministic reduce mode (SOAR_FLAG_DETERMINISTIC): instead of adding its sums to the tensor's
+// accumulators with atomics (in arrival order), every CTA of a pass stores them in a slot of its
+// own, and the head of the next kernel adds the slots in index order.  Two stage buffers alternate
+// so that a pass can fill one while late CTAs of it still read the other.
+constexpr int kMaxGrid = 1024;   // no pass has more CTAs (SM count x occupancy, at most 6 per SM)
+struct DetParts {
+  double sumsq[kMaxGrid];          // amax pass
+  double stage[2][3][kMaxGrid];    // num, den, gsum of stage s in buffer s & 1
+};
+
 struct Params {
+  DetParts* det;       // per-CTA partial sums; null unless SOAR_FLAG_DETERMINISTIC
   const uint16_t* W;
   uint8_t* packed;
   uint8_t* scales;     // row-major scale bytes, either the caller's buffer or workspace
@@ -110,6 +121,7 @@ struct Params {
 constexpr int kMaxBatch = 16;
 struct Batch {
   int n;
+  int idle_producer;          // test hook: the producer fetches nothing, so every consumer wait runs out
   unsigned int total_tiles;
   unsigned int tile_end[kMaxBatch];   // running sum of the tensors' tile counts
   Params t[kMaxBatch];
@@ -339,6 +351,7 @@ __device__ __forceinline__ void record_failure(const Batch& bt) {
 // then give up on their own.
 template <typename R>
 __device__ __forceinline__ void ring_produce(R& ring, const Batch& bt, int reverse, unsigned int run_mask) {
+  if (bt.idle_producer) return;   // test hook: nothing is fetched and nothing is in flight; the consumers give up
   unsigned int n = 0;
   bool ok = true;
   for (unsigned int g0 = blockIdx.x; g0 < bt.total_tiles; g0 += gridDim.x) {
@@ -578,36 +591,63 @@ __device__ __forceinline__ void load_weights(const float* h, unsigned int cb, do
 // tensor once (when the CTA's tile sequence leaves the tensor, or ends); the warp that arrives
 // last forwards the CTA's total to the tensor's global accumulators, one atomicAdd each.  No
 // CTA-wide barrier is involved.
-template <int N>
+template <int N, bool kDet = false>
 struct Slots {
   double acc[kMaxBatch][N];
+  // deterministic mode: each consumer warp's sums, added in warp order
+  double part[kMaxBatch][kDet ? kTile / 32 : 1][kDet ? N : 1];
   unsigned int count[kMaxBatch];
 };
 
 // All threads, before the tile loop (a __syncthreads follows in ring_init).
-template <int N>
-__device__ __forceinline__ void slots_clear(Slots<N>& sl) {
+template <int N, bool kDet>
+__device__ __forceinline__ void slots_clear(Slots<N, kDet>& sl) {
   for (int i = threadIdx.x; i < kMaxBatch * N; i += blockDim.x) (&sl.acc[0][0])[i] = 0.0;
   for (int i = threadIdx.x; i < kMaxBatch; i += blockDim.x) sl.count[i] = 0;
 }
 
-// Whole consumer warp: adds v[] for tensor `ti` and clears it.
-template <int N>
-__device__ __forceinline__ void slots_add(Slots<N>& sl, int ti, double (&v)[N], double* const (&dst)[N]) {
+// Whole consumer warp: adds v[] for tensor `ti` and clears it.  With `ordered` the warps' sums are kept
+// apart and the last warp adds them in warp order and stores the CTA's total to dst (this CTA's own
+// slot) instead of adding it to a shared accumulator: the same bits on every run.
+template <int N, bool kDet>
+__device__ __forceinline__ void slots_add(Slots<N, kDet>& sl, int ti, double (&v)[N], double* const (&dst)[N]) {
+  constexpr bool ordered = kDet;
 #pragma unroll
   for (int i = 0; i < N; ++i) v[i] = warp_sum(v[i]);
   if ((threadIdx.x & 31) == 0) {
+    if (ordered) {
 #pragma unroll
-    for (int i = 0; i < N; ++i) atomicAdd(&sl.acc[ti][i], v[i]);
+      for (int i = 0; i < N; ++i) sl.part[ti][threadIdx.x >> 5][i] = v[i];
+    } else {
+#pragma unroll
+      for (int i = 0; i < N; ++i) atomicAdd(&sl.acc[ti][i], v[i]);
+    }
     __threadfence_block();
     if (atomicAdd(&sl.count[ti], 1u) == kTile / 32 - 1) {
       __threadfence_block();
+      if (ordered) {
 #pragma unroll
-      for (int i = 0; i < N; ++i) atomicAdd(dst[i], atomicAdd(&sl.acc[ti][i], 0.0));
+        for (int i = 0; i < N; ++i) {
+          double tot = 0.0;
+          for (int w = 0; w < kTile / 32; ++w) tot += *static_cast<volatile double*>(&sl.part[ti][w][i]);
+          *dst[i] = tot;
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < N; ++i) atomicAdd(dst[i], atomicAdd(&sl.acc[ti][i], 0.0));
+      }
     }
   }
 #pragma unroll
   for (int i = 0; i < N; ++i) v[i] = 0.0;
+}
+
+// Deterministic mode, whole warp: the sum of the n per-CTA values at `parts` in a fixed order (lane l
+// adds entries l, l + 32, ... in turn, then a fixed exchange tree); every lane gets the same bits.
+__device__ __forceinline__ double ordered_sum(const double* parts, int n) {
+  double acc = 0.0;
+  for (int j = threadIdx.x & 31; j < n; j += 32) acc += parts[j];
+  return warp_sum(acc);
 }
 
 // Data-dependent status from the tensor maximum (bf16 magnitude bits).
@@ -642,10 +682,13 @@ __device__ __forceinline__ void sumsq_block(const unsigned int (&u)[8], double& 
 }
 
 // Eq. 1's tensor maximum, plus sum W^2 (binary64) for the error report.
+template <bool kDet>
 __global__ void __launch_bounds__(kThreads, 6) amax_kernel(const __grid_constant__ Batch bt, int reverse) {
   __shared__ Ring ring;
-  __shared__ Slots<1> slots;
+  __shared__ Slots<1, kDet> slots;
   slots_clear(slots);
+  constexpr bool det = kDet;
+  if (det && threadIdx.x < bt.n) bt.t[threadIdx.x].det->sumsq[blockIdx.x] = 0.0;   // a CTA may never meet a tensor
   ring_init(ring);
   if (is_producer_warp()) {
     if (threadIdx.x == kTile) ring_produce(ring, bt, reverse, 0xFFFFFFFFu);
@@ -665,7 +708,7 @@ __global__ void __launch_bounds__(kThreads, 6) amax_kernel(const __grid_constant
         mx = __reduce_max_sync(0xFFFFFFFFu, mx);
         if ((threadIdx.x & 31) == 0 && mx) atomicMax(&bt.t[cur].ws->amax_bits, mx);
         double acc[1] = {sq[0] + sq[1]};
-        double* const dst[1] = {&bt.t[cur].ws->sumsq};
+        double* const dst[1] = {det ? &bt.t[cur].det->sumsq[blockIdx.x] : &bt.t[cur].ws->sumsq};
         slots_add(slots, cur, acc, dst);
         mx = 0;
         sq[0] = sq[1] = 0.0;
@@ -706,10 +749,22 @@ __device__ __forceinline__ void add_counters(Ws* ws, unsigned int& zeros, unsign
 // dq0 = dd0; first codes (Eq. 2); stage-0 sums for Eq. 5 and the starting error.  Codes and
 // scales are written here only when no iteration follows (final != 0).  Tensors with
 // non-finite or out-of-range input are skipped.
-__global__ void __launch_bounds__(kThreads) init_kernel(const __grid_constant__ Batch bt, int reverse, int final) {
+template <bool kDet>
+__global__ void __launch_bounds__(kThreads) init_kernel(const __grid_constant__ Batch bt, int reverse, int final,
+                                                        int prev_grid) {
   __shared__ Ring ring;
-  __shared__ Slots<3> slots;
+  __shared__ Slots<3, kDet> slots;
   slots_clear(slots);
+  constexpr bool det = kDet;
+  if (det) {
+    // this CTA's stage-0 slots start at zero; CTA 0 adds up the amax pass's per-CTA sums of squares in order
+    for (int i = threadIdx.x; i < bt.n * 3; i += kThreads) bt.t[i / 3].det->stage[0][i % 3][blockIdx.x] = 0.0;
+    if (blockIdx.x == 0)
+      for (int ti = threadIdx.x >> 5; ti < bt.n; ti += kThreads / 32) {
+        const double sq = ordered_sum(bt.t[ti].det->sumsq, prev_grid);
+        if ((threadIdx.x & 31) == 0) bt.t[ti].ws->sumsq = sq;
+      }
+  }
   ring_init(ring);
   if (is_producer_warp()) {
     if (threadIdx.x == kTile) {
@@ -734,7 +789,10 @@ __global__ void __launch_bounds__(kThreads) init_kernel(const __grid_constant__ 
     if (rc != 0 || ti != cur) {
       if (cur >= 0) {
         Ws* ws = bt.t[cur].ws;
-        double* const dst[3] = {&ws->num[0], &ws->den[0], &ws->gsum[0]};
+        DetParts* dp = bt.t[cur].det;
+        double* const dst[3] = {det ? &dp->stage[0][0][blockIdx.x] : &ws->num[0],
+                                det ? &dp->stage[0][1][blockIdx.x] : &ws->den[0],
+                                det ? &dp->stage[0][2][blockIdx.x] : &ws->gsum[0]};
         slots_add(slots, cur, acc, dst);
         add_counters(ws, zeros, wide);
       }
@@ -791,7 +849,9 @@ __device__ __forceinline__ double stage_sse(const Ws* ws, int s) {
 
 // Head of an iteration (one thread): has the loop already stopped (Sec. 4.1), and the global
 // scale of Eq. 5 from the sums of the stages so far.
-__device__ __forceinline__ void iteration_head(const Params& p, int t, float& alpha_out, int& run_out) {
+// `latest` (deterministic mode): num, den, gsum of stage t, which the workspace does not hold yet.
+__device__ __forceinline__ void iteration_head(const Params& p, int t, float& alpha_out, int& run_out,
+                                               const double* latest = nullptr) {
   const Ws* ws = p.ws;
   int run = 1;
   const unsigned int amax_bits = ws->amax_bits;
@@ -799,17 +859,51 @@ __device__ __forceinline__ void iteration_head(const Params& p, int t, float& al
   float alpha = __fdiv_rn(bits_to_mag(amax_bits), 2688.0f);
   if (run) {
     double prev = stage_sse(ws, 0);
+    if (latest != nullptr && t == 0) prev = fmax(ws->sumsq + latest[2], 0.0);
     for (int i = 0; i < t; ++i) {           // did an earlier iteration trigger the stop?
-      const double cur = stage_sse(ws, i + 1);
+      const double cur = (latest != nullptr && i + 1 == t) ? fmax(ws->sumsq + latest[2], 0.0) : stage_sse(ws, i + 1);
       if (stops_after(prev, cur, p.early_stop_rel)) { run = 0; break; }
       prev = cur;
     }
     if (!(p.flags & SOAR_FLAG_KEEP_ALPHA))
-      for (int i = 0; i <= t; ++i)          // Eq. 5: alpha^(i+1) from stage-i sums
-        if (ws->den[i] > 0.0) alpha = static_cast<float>(ws->num[i] / ws->den[i]);
+      for (int i = 0; i <= t; ++i) {        // Eq. 5: alpha^(i+1) from stage-i sums
+        const double num = (latest != nullptr && i == t) ? latest[0] : ws->num[i];
+        const double den = (latest != nullptr && i == t) ? latest[1] : ws->den[i];
+        if (den > 0.0) alpha = static_cast<float>(num / den);
+      }
   }
   alpha_out = alpha;
   run_out = run;
+}
+
+// Deterministic mode, head of the kernel that follows the pass which filled stage s (iteration s, or
+// the last kernel of the call): whole CTA.  For every tensor whose stage-s slots are current (the
+// filling pass worked on it), the slots of the `prev_grid` CTAs are added in index order into
+// latest[tensor][0..2]; CTA 0 also files the sums in the workspace header, where later kernels
+// read the stages before their own.  Every CTA computes the same bits.
+__device__ __forceinline__ void gather_stage(const Batch& bt, int s, int prev_grid, double (*latest)[3]) {
+  for (int ti = threadIdx.x >> 5; ti < bt.n; ti += blockDim.x >> 5) {
+    const Params& p = bt.t[ti];
+    int filled = 1;   // stage 0 comes from the init pass, which fills every tensor's slots
+    if (s > 0) {
+      float unused;
+      iteration_head(p, s - 1, unused, filled);
+    }
+    double v[3] = {0.0, 0.0, 0.0};
+    if (filled) {
+#pragma unroll
+      for (int i = 0; i < 3; ++i) v[i] = ordered_sum(p.det->stage[s & 1][i], prev_grid);
+    }
+    if ((threadIdx.x & 31) == 0) {
+#pragma unroll
+      for (int i = 0; i < 3; ++i) latest[ti][i] = v[i];
+      if (filled && blockIdx.x == 0) {
+        p.ws->num[s] = v[0];
+        p.ws->den[s] = v[1];
+        p.ws->gsum[s] = v[2];
+      }
+    }
+  }
 }
 
 // App. B.3's E4M3 codes around a block's analytic scale: d_lo .. d_hi before clipping (the
@@ -951,23 +1045,30 @@ __device__ __forceinline__ void score_candidate(const Block& blk, const Fixed& f
 // codes, whose passes are bound by HBM rather than by the candidate loop.  Mode 4 is the candidate
 // grid of App. B.3 searched through winning_range: per E4M3 code only the multipliers that can win
 // are rounded and scored, which gives the winner of the whole grid.
-template <int kMode>   // 0: candidate grid, every multiplier visited; 1: one candidate scale (beta = 1), at most two
+template <int kMode, bool kDet>   // 0: candidate grid, every multiplier visited; 1: one candidate scale (beta = 1), at most two
                        // codes; 2: the same with the coupled scale; 3: one candidate scale, any number of codes;
                        // 4: candidate grid, only the multipliers that can win
 __global__ void __launch_bounds__(kThreads, (kMode == 1 || kMode == 3) ? 3 : 2)
-iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, int keep) {
+iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, int keep, int prev_grid) {
   constexpr bool kSingle = kMode == 1 || kMode == 2 || kMode == 3;
   __shared__ RingWithState ring;
-  __shared__ Slots<3> slots;
+  __shared__ Slots<3, kDet> slots;
   __shared__ float s_beta[kSingle ? 1 : SOAR_MAX_BETA];
   __shared__ float s_alpha[kMaxBatch];
+  __shared__ double s_latest[kDet ? kMaxBatch : 1][3];
   __shared__ unsigned int s_run;
+  constexpr bool det = kDet;
   if (threadIdx.x == 0) s_run = 0;
+  if (det) {
+    // this CTA's slots of the stage it will fill start at zero; the stage the previous pass filled is added up
+    for (int i = threadIdx.x; i < bt.n * 3; i += kThreads) bt.t[i / 3].det->stage[(t + 1) & 1][i % 3][blockIdx.x] = 0.0;
+    gather_stage(bt, t, prev_grid, s_latest);
+  }
   __syncthreads();
   if (threadIdx.x < bt.n) {   // per tensor: still running?  its alpha for this iteration
     float a;
     int run;
-    iteration_head(bt.t[threadIdx.x], t, a, run);
+    iteration_head(bt.t[threadIdx.x], t, a, run, det ? s_latest[threadIdx.x] : nullptr);
     s_alpha[threadIdx.x] = a;
     if (run) atomicOr(&s_run, 1u << threadIdx.x);
   }
@@ -1005,7 +1106,11 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
     if (rc != 0 || ti != cur) {
       if (cur >= 0) {
         Ws* ws = bt.t[cur].ws;
-        double* const dst[3] = {&ws->num[t + 1], &ws->den[t + 1], &ws->gsum[t + 1]};
+        DetParts* dp = bt.t[cur].det;
+        const int sb = (t + 1) & 1;
+        double* const dst[3] = {det ? &dp->stage[sb][0][blockIdx.x] : &ws->num[t + 1],
+                                det ? &dp->stage[sb][1][blockIdx.x] : &ws->den[t + 1],
+                                det ? &dp->stage[sb][2][blockIdx.x] : &ws->gsum[t + 1]};
         slots_add(slots, cur, acc, dst);
         add_counters(ws, unused_zeros, wide);
       }
@@ -1261,13 +1366,36 @@ struct Reports {
 
 // Replays the early-stop rule over the stage sums, writes alpha and the report; one CTA per tensor.
 __global__ void __launch_bounds__(128) finalize_kernel(const __grid_constant__ Batch bt,
-                                                       const __grid_constant__ Reports rp) {
+                                                       const __grid_constant__ Reports rp, int prev_grid) {
   const Params& p = bt.t[blockIdx.x];
   float* out_alpha = rp.alpha[blockIdx.x];
   soar_result* res = rp.result[blockIdx.x];
   __shared__ double s_num[SOAR_MAX_ITERS + 1], s_den[SOAR_MAX_ITERS + 1], s_sse[SOAR_MAX_ITERS + 1];
   __shared__ double s_ta[SOAR_MAX_ITERS + 1];
   __shared__ int s_iters;
+  if (p.det != nullptr) {
+    // deterministic mode: the stage the last pass filled is still in the per-CTA slots; this CTA (the
+    // only one working on this tensor) adds them up in order and files them in the header
+    if (threadIdx.x < 32) {
+      int filled = 1;
+      if (p.max_iters > 0) {
+        float unused;
+        iteration_head(p, p.max_iters - 1, unused, filled);
+      }
+      if (filled) {
+        double v[3];
+#pragma unroll
+        for (int i = 0; i < 3; ++i) v[i] = ordered_sum(p.det->stage[p.max_iters & 1][i], prev_grid);
+        if (threadIdx.x == 0) {
+          p.ws->num[p.max_iters] = v[0];
+          p.ws->den[p.max_iters] = v[1];
+          p.ws->gsum[p.max_iters] = v[2];
+        }
+      }
+    }
+    __threadfence_block();
+    __syncthreads();
+  }
   const Ws* ws = p.ws;
   const unsigned int amax_bits = ws->amax_bits;
   const int st = status_from_amax(amax_bits);
@@ -1860,6 +1988,9 @@ struct ScopedLaunch {
 
 int g_sm_count[64];
 
+// Test hook (soar_debug_fail_waits): what the launches put into Batch::idle_producer.
+int g_idle_producer = 0;
+
 int sm_count() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
@@ -1878,7 +2009,8 @@ unsigned int persistent_grid(K kernel, unsigned int tiles, int threads) {
   int per_sm = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, 0) != cudaSuccess || per_sm <= 0)
     per_sm = 2;
-  const unsigned int cap = static_cast<unsigned int>(sm_count() * per_sm);
+  unsigned int cap = static_cast<unsigned int>(sm_count() * per_sm);
+  if (cap > static_cast<unsigned int>(kMaxGrid)) cap = kMaxGrid;   // the deterministic mode keeps one slot per CTA
   return tiles < cap ? (tiles ? tiles : 1u) : cap;
 }
 
@@ -1907,7 +2039,8 @@ int check_cfg(const soar_cfg* cfg) {
   if (100 - (cfg->n_beta / 2) * cfg->beta_step_pct <= 0) return SOAR_ERR_INVALID_ARG;
   if ((cfg->scale_layout & ~(SOAR_SCALES_LINEAR | SOAR_SCALES_SWIZZLED)) != 0 || cfg->scale_layout == 0)
     return SOAR_ERR_INVALID_ARG;
-  if ((cfg->flags & ~(SOAR_FLAG_COUPLED_SCALE | SOAR_FLAG_KEEP_ALPHA | SOAR_FLAG_KEEP_BLOCK_SCALE)) != 0)
+  if ((cfg->flags & ~(SOAR_FLAG_COUPLED_SCALE | SOAR_FLAG_KEEP_ALPHA | SOAR_FLAG_KEEP_BLOCK_SCALE |
+                      SOAR_FLAG_DETERMINISTIC)) != 0)
     return SOAR_ERR_INVALID_ARG;
   return SOAR_OK;
 }
@@ -1956,6 +2089,7 @@ size_t soar_workspace_bytes(int64_t rows, int64_t cols, const soar_cfg* cfg) {
   size_t n = kWsFixedBytes;
   if (cfg->max_iters > 0) n += round256(nblk * sizeof(uint2));
   if (!(cfg->scale_layout & SOAR_SCALES_LINEAR)) n += round256(nblk);
+  if (cfg->flags & SOAR_FLAG_DETERMINISTIC) n += round256(sizeof(DetParts));
   return n;
 }
 
@@ -1997,6 +2131,9 @@ int run_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void*
   if (tensors == nullptr || n <= 0) return SOAR_ERR_INVALID_ARG;
   const bool want_lin = (cfg->scale_layout & SOAR_SCALES_LINEAR) != 0;
   const bool want_sw = (cfg->scale_layout & SOAR_SCALES_SWIZZLED) != 0;
+  const bool det = (cfg->flags & SOAR_FLAG_DETERMINISTIC) != 0;
+  // a stage run alone leaves its sums in the per-CTA slots, which the caller of the stages cannot combine
+  if (det && stages != kStageAll) return SOAR_ERR_UNSUPPORTED;
   for (int i = 0; i < n; ++i) {   // every argument is checked before anything is enqueued
     const soar_tensor_desc& d = tensors[i];
     rc = check_shape(d.W_bf16, d.rows, d.cols, d.ld);
@@ -2028,6 +2165,7 @@ int run_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void*
     memset(&bt, 0, sizeof(bt));
     memset(&rp, 0, sizeof(rp));
     bt.n = (n - first < kMaxBatch) ? n - first : kMaxBatch;
+    bt.idle_producer = g_idle_producer;
     unsigned int tiles = 0;
     for (int j = 0; j < bt.n; ++j) {
       const soar_tensor_desc& d = tensors[first + j];
@@ -2051,6 +2189,11 @@ int run_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void*
         p.scales = next;
         next += round256(p.nblk);
       }
+      p.det = nullptr;
+      if (det) {
+        p.det = reinterpret_cast<DetParts*>(next);
+        next += round256(sizeof(DetParts));
+      }
       p.max_iters = cfg->max_iters;
       p.early_stop_rel = cfg->early_stop_rel;
       p.n_dq = cfg->n_dq;
@@ -2067,14 +2210,21 @@ int run_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void*
 
     // Passes alternate direction over the tiles (amax forward, init backward, iteration t forward
     // for even t): each starts where the previous one ended, on data still in L2.
+    const unsigned int g_amax = det ? persistent_grid(amax_kernel<true>, tiles, kThreads)
+                                    : persistent_grid(amax_kernel<false>, tiles, kThreads);
+    const unsigned int g_init = det ? persistent_grid(init_kernel<true>, tiles, kThreads)
+                                    : persistent_grid(init_kernel<false>, tiles, kThreads);
+    unsigned int g_last = g_init;   // grid of the pass whose sums the next kernel's head reads
     if (stages & kStageAmax) {
       ScopedLaunch sl(K_AMAX, st);
-      amax_kernel<<<persistent_grid(amax_kernel, tiles, kThreads), kThreads, 0, st>>>(bt, 0);
+      if (det) amax_kernel<true><<<g_amax, kThreads, 0, st>>>(bt, 0);
+      else amax_kernel<false><<<g_amax, kThreads, 0, st>>>(bt, 0);
     }
     if (stages & kStageInit) {
       ScopedLaunch sl(K_INIT, st);
-      init_kernel<<<persistent_grid(init_kernel, tiles, kThreads), kThreads, 0, st>>>(bt, 1,
-                                                                                      cfg->max_iters == 0 ? 1 : 0);
+      const int final = cfg->max_iters == 0 ? 1 : 0;
+      if (det) init_kernel<true><<<g_init, kThreads, 0, st>>>(bt, 1, final, static_cast<int>(g_amax));
+      else init_kernel<false><<<g_init, kThreads, 0, st>>>(bt, 1, final, static_cast<int>(g_amax));
     }
     if (stages & kStageIterate) {
       // a grid of several multipliers with one quantization scale per multiplier: only those that can win
@@ -2083,28 +2233,40 @@ int run_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void*
                              cfg->beta_step_pct >= 1;
       const int mode = !single ? (bracketed ? 4 : 0)
                                : ((cfg->flags & SOAR_FLAG_COUPLED_SCALE) ? 2 : (cfg->n_dq <= 2 ? 1 : 3));
-      const unsigned int g_it = mode == 0   ? persistent_grid(iterate_kernel<0>, tiles, kThreads)
-                                : mode == 1 ? persistent_grid(iterate_kernel<1>, tiles, kThreads)
-                                : mode == 2 ? persistent_grid(iterate_kernel<2>, tiles, kThreads)
-                                : mode == 3 ? persistent_grid(iterate_kernel<3>, tiles, kThreads)
-                                            : persistent_grid(iterate_kernel<4>, tiles, kThreads);
+      unsigned int g_it = 0;
       for (int t = t_lo; t < t_hi; ++t) {
         const int reverse = t & 1;
         // with the early stop on, any iteration may turn out to be the last one
         const int last = (t == cfg->max_iters - 1) ? 1 : 0;
         const int emit = (may_stop || last) ? 1 : 0;
+        const int pg = static_cast<int>(g_last);
         ScopedLaunch sl(K_ITERATE, st);
-        if (mode == 0) iterate_kernel<0><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
-        else if (mode == 1) iterate_kernel<1><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
-        else if (mode == 2) iterate_kernel<2><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
-        else if (mode == 3) iterate_kernel<3><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
-        else iterate_kernel<4><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last);
+#define SOAR_LAUNCH_ITERATE(M, D)                                                           \
+  do {                                                                                      \
+    if (g_it == 0) g_it = persistent_grid(iterate_kernel<M, D>, tiles, kThreads);           \
+    iterate_kernel<M, D><<<g_it, kThreads, 0, st>>>(bt, t, reverse, emit, !last, pg);       \
+  } while (0)
+        if (det) {
+          if (mode == 0) SOAR_LAUNCH_ITERATE(0, true);
+          else if (mode == 1) SOAR_LAUNCH_ITERATE(1, true);
+          else if (mode == 2) SOAR_LAUNCH_ITERATE(2, true);
+          else if (mode == 3) SOAR_LAUNCH_ITERATE(3, true);
+          else SOAR_LAUNCH_ITERATE(4, true);
+        } else {
+          if (mode == 0) SOAR_LAUNCH_ITERATE(0, false);
+          else if (mode == 1) SOAR_LAUNCH_ITERATE(1, false);
+          else if (mode == 2) SOAR_LAUNCH_ITERATE(2, false);
+          else if (mode == 3) SOAR_LAUNCH_ITERATE(3, false);
+          else SOAR_LAUNCH_ITERATE(4, false);
+        }
+#undef SOAR_LAUNCH_ITERATE
+        g_last = g_it;
       }
     }
     if (!(stages & kStageFinalize)) continue;
     {
       ScopedLaunch sl(K_FINALIZE, st);
-      finalize_kernel<<<bt.n, 128, 0, st>>>(bt, rp);
+      finalize_kernel<<<bt.n, 128, 0, st>>>(bt, rp, static_cast<int>(g_last));
     }
     if (want_sw) {
       for (int j = 0; j < bt.n; ++j) {
@@ -2233,6 +2395,7 @@ int dequant_error_impl(const void* W_bf16, int64_t rows, int64_t cols, int64_t l
     Batch bt;
     memset(&bt, 0, sizeof(bt));
     bt.n = 1;
+    bt.idle_producer = g_idle_producer;
     bt.t[0] = p;
     bt.total_tiles = p.ntiles;
     for (int j = 0; j < kMaxBatch; ++j) bt.tile_end[j] = j == 0 ? p.ntiles : 0xFFFFFFFFu;
@@ -2281,6 +2444,7 @@ int soar_quantize_weighted(const void* W_bf16, int64_t rows, int64_t cols, int64
                            size_t workspace_bytes, soar_result* out_result, void* stream) {
   int rc = check_cfg(cfg);
   if (rc != SOAR_OK) return rc;
+  if (cfg->flags & SOAR_FLAG_DETERMINISTIC) return SOAR_ERR_UNSUPPORTED;   // the weighted passes add with atomics only
   rc = check_shape(W_bf16, rows, cols, ld);
   if (rc != SOAR_OK) return rc;
   const bool want_lin = (cfg->scale_layout & SOAR_SCALES_LINEAR) != 0;
@@ -2329,6 +2493,7 @@ int soar_quantize_weighted(const void* W_bf16, int64_t rows, int64_t cols, int64
   p.beta_step_pct = cfg->beta_step_pct;
   p.flags = cfg->flags;
   bt.n = 1;
+  bt.idle_producer = g_idle_producer;
   bt.total_tiles = p.ntiles;
   for (int j = 0; j < kMaxBatch; ++j) bt.tile_end[j] = j == 0 ? p.ntiles : 0xFFFFFFFFu;
   rp.alpha[0] = out_global_fp32;
@@ -2355,7 +2520,7 @@ int soar_quantize_weighted(const void* W_bf16, int64_t rows, int64_t cols, int64
   }
   {
     ScopedLaunch sl(K_FINALIZE, st);
-    finalize_kernel<<<1, 128, 0, st>>>(bt, rp);
+    finalize_kernel<<<1, 128, 0, st>>>(bt, rp, 0);
   }
   if (want_sw) {
     const unsigned int rt = static_cast<unsigned int>((rows + 127) / 128);
@@ -2566,6 +2731,11 @@ int soar_selftest_reciprocal(int lo_exp, int hi_exp, unsigned long long* out_mis
   selftest_reciprocal_kernel<<<sm_count() * 8, 256, 0, st>>>(static_cast<unsigned int>(lo_exp),
                                                              static_cast<unsigned int>(hi_exp), out_mismatches);
   return cudaGetLastError() == cudaSuccess ? SOAR_OK : SOAR_ERR_CUDA;
+}
+
+int soar_debug_fail_waits(int on) {
+  g_idle_producer = on ? 1 : 0;
+  return SOAR_OK;
 }
 
 int soar_trace_begin(void) {

@@ -165,6 +165,78 @@ def test_batch_gives_each_matrix_what_a_single_call_gives(cfgkw):
             P.assert_parity(g, R.quantize(w, ref_cfg))
 
 
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_library_usable():
+    """The kernels' waits are bounded.  With the test hook on, no tile is ever fetched, every consumer
+    wait runs to its poll limit, the kernels return, and the report says so; a normal call on the
+    same buffers right afterwards gives the right bytes."""
+    w = WL.small_case(300, 2048, 95, outlier_entry_frac=0.002, outlier_scale=30.0)
+    cfg, ref_cfg = P.cfg_pair(max_iters=3)
+    W = P.to_device(w)
+    out = api.alloc_buffers(300, 2048, cfg)
+    api.soar_debug_fail_waits(True)
+    try:
+        api.soar_quantize(W, cfg, out)
+        e = api.soar_dequant_error(W, out.packed, out.scales, out.alpha)
+        torch.cuda.synchronize()
+    finally:
+        api.soar_debug_fail_waits(False)
+    res = out.read_result()
+    assert res.status & api.STATUS_INTERNAL and res.iters_run == 0
+    assert bool(torch.isnan(e).all())
+    api.soar_quantize(W, cfg, out)                                  # same workspace, right after
+    torch.cuda.synchronize()
+    g = P.GpuOut(out.packed.cpu().numpy(), out.scales.cpu().numpy(), float(out.alpha.cpu()[0]), out.read_result(), out)
+    P.assert_parity(g, R.quantize(w, ref_cfg))
+
+
+def test_deterministic_mode_repeats_bit_for_bit():
+    """With SOAR_FLAG_DETERMINISTIC the tensor-wide sums are added in a fixed order: twenty runs of a
+    tensor of a thousand tiles (every CTA of every pass contributes) and of a batch give the same
+    bits in every output and every reported number; and they are the oracle's results."""
+    w = WL.small_case(2048, 2048, 301, outlier_entry_frac=0.0005, outlier_scale=50.0)
+    small = [WL.small_case(r, c, 310 + i) for i, (r, c) in enumerate([(300, 1024), (1, 16), (77, 4096)])]
+    cfg, ref_cfg = P.cfg_pair()
+    cfg.flags |= api.FLAG_DETERMINISTIC
+    assert api.soar_workspace_bytes(2048, 2048, cfg) >= api.soar_workspace_bytes(2048, 2048, P.cfg_pair()[0]) + 56 * 1024
+    W = P.to_device(w)
+    dev = [P.to_device(x) for x in small]
+    first = None
+    for rep in range(20):
+        out = api.soar_quantize(W, cfg)
+        outs = [api.alloc_buffers(x.shape[0], x.shape[1], cfg) for x in small]
+        api.soar_quantize_batch(dev, cfg, outs)
+        torch.cuda.synchronize()
+        got = []
+        for o in [out] + outs:
+            r = o.read_result()
+            got.append((o.packed.cpu().numpy().tobytes(), o.scales.cpu().numpy().tobytes(), o.alpha.cpu().numpy().tobytes(),
+                        r.iters_run, r.sse, r.sse_init, r.sumsq, tuple(r.trace_sse), tuple(r.trace_alpha)))
+        if first is None:
+            first = got
+            g = P.GpuOut(out.packed.cpu().numpy(), out.scales.cpu().numpy(), float(out.alpha.cpu()[0]),
+                         out.read_result(), out)
+            P.assert_parity(g, R.quantize(w, ref_cfg))
+            for x, o in zip(small, outs):
+                g = P.GpuOut(o.packed.cpu().numpy(), o.scales.cpu().numpy(), float(o.alpha.cpu()[0]), o.read_result(), o)
+                P.assert_parity(g, R.quantize(x, ref_cfg), mismatch_cap=0)
+        else:
+            assert got == first, rep
+    # settings without iterations, and the one-candidate shape
+    for kw in (dict(max_iters=0), dict(max_iters=1, early_stop_rel=0.0, n_dq=2, n_beta=1)):
+        c, rc = P.cfg_pair(**kw)
+        c.flags |= api.FLAG_DETERMINISTIC
+        a, b = P.run_gpu(w, c), P.run_gpu(w, c)
+        assert (a.result.sse, a.result.sumsq, a.alpha) == (b.result.sse, b.result.sumsq, b.alpha)
+        assert np.array_equal(a.packed, b.packed)
+        P.assert_parity(a, R.quantize(w, rc))
+    # the staged and the weighted entry points do not take the flag
+    with pytest.raises(api.SoarError):
+        o = api.alloc_buffers(2048, 2048, cfg)
+        api.soar_quantize_stage([W], cfg, [o], o.workspace, api.STAGE_AMAX)
+    with pytest.raises(api.SoarError):
+        api.soar_quantize_weighted(W, torch.ones(2048, device="cuda"), cfg)
+
+
 def test_calls_on_two_streams_with_their_own_workspaces_do_not_disturb_each_other():
     w1 = WL.small_case(300, 2048, 81, outlier_entry_frac=0.003, outlier_scale=30.0)
     w2 = WL.small_case(200, 4096, 82, dist="laplace")
@@ -271,7 +343,7 @@ def test_argument_errors_are_reported_on_the_host():
     with pytest.raises(api.SoarError):
         api.soar_quantize(w, bad)
     with pytest.raises(api.SoarError):
-        api.soar_quantize(w, api.soar_default_cfg(flags=8))    # unknown flag bit
+        api.soar_quantize(w, api.soar_default_cfg(flags=16))   # unknown flag bit
     out = api.alloc_buffers(4, 64, cfg)
     out.workspace = out.workspace[:16]
     with pytest.raises(api.SoarError):

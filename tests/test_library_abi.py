@@ -36,7 +36,7 @@ def test_host_side_helpers():
     assert (cj.max_iters, cj.n_dq, cj.n_beta, cj.flags) == (15, 1, 1, api.FLAG_COUPLED_SCALE)
     ds = api.soar_default_cfg(api.PRESET_DSS_ONLY)
     assert (ds.max_iters, ds.n_dq, ds.n_beta, ds.flags) == (1, 2, 101, api.FLAG_KEEP_ALPHA | api.FLAG_KEEP_BLOCK_SCALE)
-    assert api.soar_workspace_bytes(128, 256, api.soar_default_cfg(flags=8)) == 0
+    assert api.soar_workspace_bytes(128, 256, api.soar_default_cfg(flags=16)) == 0
     assert api.soar_workspace_bytes(128, 256, cfg) >= 1024
     assert api.soar_workspace_bytes(128, 250, cfg) == 0
     sw = api.soar_default_cfg(scale_layout=api.SCALES_SWIZZLED)
