@@ -1202,10 +1202,11 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
         const int k1 = max(0, min(n_beta - 2, __float2int_rd(__fmaf_rn(dv1, per_center, k_off))));
         const float s00 = grid_divisor(alpha, center, s_beta[k0]), s01 = grid_divisor(alpha, center, s_beta[k0 + 1]);
         const float s10 = grid_divisor(alpha, center, s_beta[k1]), s11 = grid_divisor(alpha, center, s_beta[k1 + 1]);
-        const float s_first = grid_divisor(alpha, center, s_beta[0]);
-        bool direct = nd <= 2 && fx.ok && recip_fast_ok(s_first) &&
-                      recip_fast_ok(grid_divisor(alpha, center, s_beta[n_beta - 1])) &&
-                      __fmul_rn(blk.bmax, recip_fast(s_first)) <= 32.0f && s00 <= lo0 && s01 >= hi0;
+        // the four divisors lie between s00 and s11 (or s01 without a second code): those two bound the range
+        // of the fast reciprocal, and the smallest one decides whether the exact integer sums hold
+        const float s_hi = second ? s11 : s01;
+        bool direct = nd <= 2 && fx.ok && recip_fast_ok(s00) && recip_fast_ok(s_hi) &&
+                      __fmul_rn(blk.bmax, recip_fast(s00)) <= 32.0f && s00 <= lo0 && s01 >= hi0;
         if (second) direct = direct && s10 <= lo1 && s11 >= hi1;
         if (direct) {
           // error minus sum W^2 = 2 sd unit (rho * 4B - afix) with rho = sd / (8 unit): per code the two
@@ -1747,46 +1748,63 @@ weighted_init_kernel(const __grid_constant__ Batch bt, const Weighted wq, int re
   add_counters(p.ws, zeros, unused_wide);
 }
 
-// Eq. 8 for one block over the whole grid with binary64 sums for every candidate: index nd * k + d of
-// the first minimum in (beta, code) order.  Serves the coupled arm and the blocks whose candidates
-// can cost exactly the same (see weighted_iterate_kernel); kept out of line so that its registers
-// do not weigh on the common path.
-__device__ __noinline__ int weighted_exact_argmin(const float* h, unsigned int cb, const uint16_t* w16, float alpha,
-                                                  float center, const float* s_beta, int n_beta, int d_lo, int nd,
-                                                  bool coupled, bool fast_rcp) {
-  // the block comes from memory (sixteen bf16 values at w16), not from the caller's registers
-  Block mags;
+// Eq. 8 for one block over the whole grid with binary64 sums for every candidate, first minimum in
+// (beta, code) order; the winner is then made again with its signs and its sums in element order.
+// Serves the coupled arm and the blocks whose candidates can cost exactly the same (see
+// weighted_iterate_kernel).  Out of line and fed from memory (sixteen bf16 values at w16, the weights
+// at h), so that nothing of it weighs on the registers of the common path.
+__device__ __noinline__ void weighted_whole_grid_search(const float* h, unsigned int cb, const uint16_t* w16,
+                                                        float alpha, float center, const float* s_beta, int n_beta,
+                                                        int d_lo, int nd, bool coupled, bool fast_rcp, Winner* out) {
+  Block blk, mags;
   {
     const uint4* src = reinterpret_cast<const uint4*>(w16);
-    unpack_block(__ldg(src), __ldg(src + 1), mags);
+    unpack_block(__ldg(src), __ldg(src + 1), blk);
 #pragma unroll
-    for (int j = 0; j < 16; ++j) mags.w[j] = fabsf(mags.w[j]);
+    for (int j = 0; j < 16; ++j) mags.w[j] = fabsf(blk.w[j]);
   }
-  double hd[16], hw[16];
-  block_weights(h, cb, mags, hd, hw);
   const double alpha_d = static_cast<double>(alpha);
   double best = __longlong_as_double(0x7FF0000000000000ll);
   int best_key = 0;
-  for (int k = 0; k < n_beta; ++k) {
-    unsigned int c0, c1;
-    double A = 0.0, B = 0.0;
-    if (!coupled) {
-      const float s = __fmul_rn(alpha, __fmul_rn(center, s_beta[k]));
-      round_block(mags, fast_rcp ? recip_fast(s) : __frcp_rn(s), c0, c1);
-      weighted_sums_split(hw, hd, c0, c1, A, B);
-    }
-    for (int d = 0; d < nd; ++d) {
-      const float dv = e4m3_value(clip_code(d_lo + d));
-      if (coupled) {
-        round_block(mags, recip_scale(alpha, __fmul_rn(dv, s_beta[k])), c0, c1);
+  {
+    double hd[16], hw[16];
+    block_weights(h, cb, mags, hd, hw);
+    for (int k = 0; k < n_beta; ++k) {
+      unsigned int c0, c1;
+      double A = 0.0, B = 0.0;
+      if (!coupled) {
+        const float s = __fmul_rn(alpha, __fmul_rn(center, s_beta[k]));
+        round_block(mags, fast_rcp ? recip_fast(s) : __frcp_rn(s), c0, c1);
         weighted_sums_split(hw, hd, c0, c1, A, B);
       }
-      const double sd = alpha_d * static_cast<double>(dv);
-      const double g = sd * fma(sd, B, -2.0 * A);
-      if (g < best) { best = g; best_key = nd * k + d; }
+      for (int d = 0; d < nd; ++d) {
+        const float dv = e4m3_value(clip_code(d_lo + d));
+        if (coupled) {
+          round_block(mags, recip_scale(alpha, __fmul_rn(dv, s_beta[k])), c0, c1);
+          weighted_sums_split(hw, hd, c0, c1, A, B);
+        }
+        const double sd = alpha_d * static_cast<double>(dv);
+        const double g = sd * fma(sd, B, -2.0 * A);
+        if (g < best) { best = g; best_key = nd * k + d; }
+      }
     }
   }
-  return best_key;
+  Winner w;
+  const int bk = best_key / nd;
+  w.d = clip_code(d_lo + (best_key - bk * nd));
+  round_block(blk, recip_scale(alpha, __fmul_rn(coupled ? e4m3_value(w.d) : center, s_beta[bk])), w.c0, w.c1);
+  float hf[16];
+  {
+    const float4* src = reinterpret_cast<const float4*>(h) + static_cast<size_t>(cb) * 4;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float4 v = __ldg(src + q);
+      hf[4 * q] = v.x; hf[4 * q + 1] = v.y; hf[4 * q + 2] = v.z; hf[4 * q + 3] = v.w;
+    }
+  }
+  weighted_sums_streamed(hf, blk.w, w.c0, w.c1, w.A, w.B);
+  w.g = best;
+  *out = w;
 }
 
 // One iteration t of Algorithm 1 under the weighted objective: Eq. 5 from the stage-t sums,
@@ -1902,15 +1920,15 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
         }
       }
     } else {
-      const int best_key =
-          weighted_exact_argmin(wq.h, cb, p.W + static_cast<long long>(row) * p.ld + static_cast<long long>(cb) * 16,
-                                alpha, center, s_beta, n_beta, d_lo, nd, coupled, fast_rcp);
+      Winner w;
+      weighted_whole_grid_search(wq.h, cb, p.W + static_cast<long long>(row) * p.ld + static_cast<long long>(cb) * 16,
+                                 alpha, center, s_beta, n_beta, d_lo, nd, coupled, fast_rcp, &w);
       ++exact_blocks;
-      // the winner, made again from its index, now with the signs and the sums in element order
-      const int bk = best_key / nd;
-      best_d = clip_code(d_lo + (best_key - bk * nd));
-      round_block(blk, recip_scale(alpha, __fmul_rn(coupled ? e4m3_value(best_d) : center, s_beta[bk])), best0, best1);
-      weighted_sums_streamed(hf, blk.w, best0, best1, bestA, bestB);
+      best0 = w.c0;
+      best1 = w.c1;
+      bestA = w.A;
+      bestB = w.B;
+      best_d = w.d;
     }
     if (emit) {
       reinterpret_cast<uint2*>(p.packed)[b] = make_uint2(best0, best1);
