@@ -28,7 +28,9 @@
  * against an independent library cast; Eq. 5/6 against brute-force minimisation;
  * the Eq. 8 argmin against a separate NumPy enumeration; grid-aligned tensors
  * against their closed-form result; the weighted form against weighted least
- * squares, constant weights and zero-weight columns.  Parity unpinned: the early-stop trajectory
+ * squares, constant weights and zero-weight columns; the MXFP4 mode (end of this file)
+ * against the format's definition, a NumPy restatement and a brute-force argmin, its
+ * candidate rule being a reading the paper does not fix.  Parity unpinned: the early-stop trajectory
  * and the iteration-to-iteration path (the paper prints no numbers for them);
  * those rest on agreement between this file and the NumPy restatement.
  */
@@ -513,4 +515,180 @@ int soar_ref_num_threads(void) {
 #else
   return 1;
 #endif
+}
+
+/* ------------------------------------------------------------------ MXFP4
+ *
+ * Sec. 4.3 "DSS on MXFP4" applies the decoupled search of Sec. 3.3 to the other microscaling
+ * format: E2M1 elements in blocks of 32 with one shared power-of-two scale (an E8M0 byte,
+ * value 2^(code - 127)) and no tensor-wide scale.  The paper reports results and no
+ * procedure, so what follows is a reading (parity unpinned by the paper; pinned by the
+ * CPU tests against a separate NumPy restatement, brute force and the format's definition):
+ *
+ *   plain MXFP4   the format's own rule: shared exponent floor(log2 bmax) - 2 (2 is the
+ *                 exponent of E2M1's largest value, 6 = 1.5 * 2^2), elements rounded to nearest
+ *                 (ties to even) and saturated at 6.
+ *   with DSS      Sec. 3.3 (i)-(ii) with alpha = 1: the high-precision scale is Eq. 1's
+ *                 max-based one, D* = fl32(bmax / 6); dequantization candidates are the n_dq
+ *                 E8M0 values around D* (App. B.3's rule on powers of two: with c_f the largest
+ *                 code whose value is <= D*, codes c_f-(n/2-1) .. c_f+n/2; n = 1: the nearer of
+ *                 c_f, c_f+1, the lower one on a tie), quantization candidates D* * beta_k on
+ *                 App. B.3's multiplier grid; every pair is scored by Eq. 8 and the first
+ *                 minimum in (beta, code) order is kept.  For n_dq = 2 the plain rule's
+ *                 exponent is always one of the two candidates.
+ *
+ * Blocks whose largest magnitude is below 2^-120 (or zero) are stored as zero blocks: scale
+ * code 0 and zero codes (their sign bits kept).
+ */
+#define REF_MX_BLOCK 32
+
+double soar_ref_e8m0_decode(uint8_t code) { return ldexp(1.0, (int)code - 127); }
+
+/* Largest e with 2^e <= v, for finite v > 0. */
+static int mx_floor_log2(float v) {
+  int e;
+  (void)frexpf(v, &e);          /* v = m * 2^e, m in [0.5, 1) */
+  return e - 1;
+}
+
+/* The plain rule's scale code for a block maximum. */
+uint8_t soar_ref_mx_plain_code(float bmax) {
+  int c = mx_floor_log2(bmax) - 2 + 127;
+  return (uint8_t)(c < 0 ? 0 : (c > 254 ? 254 : c));
+}
+
+/* E8M0 codes around a positive scale; returns how many (ascending, clipped to [0, 254],
+ * duplicates dropped). */
+int soar_ref_mx_candidates(float center, int n, uint8_t* out) {
+  int cf = mx_floor_log2(center) + 127;
+  int lo, hi;
+  if (n <= 1) {
+    double mid = 1.5 * ldexp(1.0, cf - 127);
+    lo = hi = ((double)center > mid) ? cf + 1 : cf;
+  } else {
+    lo = cf - (n / 2 - 1);
+    hi = cf + n / 2;
+  }
+  int cnt = 0;
+  for (int c = lo; c <= hi; ++c) {
+    int cc = c < 0 ? 0 : (c > 254 ? 254 : c);
+    if (cnt > 0 && out[cnt - 1] == (uint8_t)cc) continue;
+    out[cnt++] = (uint8_t)cc;
+  }
+  return cnt;
+}
+
+/* Eq. 2 for a block of 32 under quantization scale dq (alpha = 1): r = fl32(1/dq),
+ * x_j = fl32(|W_j| * r), m_j = E2M1 rounding of x_j. */
+void soar_ref_mx_round_block(const uint16_t* w, float dq, double* m) {
+  float r = 1.0f / dq;
+  for (int j = 0; j < REF_MX_BLOCK; ++j) {
+    float x = fabsf(soar_ref_bf16_to_f32(w[j])) * r;
+    m[j] = soar_ref_e2m1_round((double)x);
+  }
+}
+
+/* Eq. 8's error of a block of 32 for magnitudes m and scale code d: sum (|W_j| - m_j 2^(d-127))^2. */
+double soar_ref_mx_block_error(const uint16_t* w, const double* m, uint8_t d) {
+  double s = soar_ref_e8m0_decode(d), L = 0.0;
+  for (int j = 0; j < REF_MX_BLOCK; ++j) {
+    double e = fabs((double)soar_ref_bf16_to_f32(w[j])) - m[j] * s;
+    L += e * e;
+  }
+  return L;
+}
+
+/*
+ * MXFP4 quantization of W[rows][ld] (cols used, cols % 32 == 0).  n_beta == 0: the plain rule;
+ * otherwise the search above with n_dq codes and n_beta multipliers of step step_pct/100.
+ *   out_packed  rows*cols/2 bytes, nibble layout as soar_ref_quantize
+ *   out_scales  rows*cols/32 E8M0 bytes, row-major
+ *   out_sse     sum (W - What)^2;  out_sumsq  sum W^2 (may be NULL)
+ *   tie_flags   per block (may be NULL): 1 if the best two distinct outcomes were closer than tie_rel
+ * Returns status bits (REF_STATUS_NONFINITE, REF_STATUS_ZERO_TENSOR).
+ */
+int soar_ref_mx_quantize(const uint16_t* W, int64_t rows, int64_t cols, int64_t ld, int n_dq, int n_beta,
+                         int step_pct, uint8_t* out_packed, uint8_t* out_scales, double* out_sse,
+                         double* out_sumsq, uint8_t* tie_flags, double tie_rel) {
+  const int64_t nbc = cols / REF_MX_BLOCK;
+  int status = 0;
+  double sumsq = 0.0;
+  float amax = 0.0f;
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t c = 0; c < cols; ++c) {
+      float v = fabsf(soar_ref_bf16_to_f32(W[r * ld + c]));
+      if (!(v <= 3.4e38f)) status |= REF_STATUS_NONFINITE;
+      if (v > amax) amax = v;
+      sumsq += (double)v * (double)v;
+    }
+  if (out_sumsq) *out_sumsq = sumsq;
+  *out_sse = 0.0;
+  if (status) return status;
+  if (amax == 0.0f) status |= REF_STATUS_ZERO_TENSOR;
+  double* rowL = (double*)calloc((size_t)rows, sizeof(double));
+#ifdef _OPENMP
+#pragma omp parallel for schedule(static)
+#endif
+  for (int64_t r = 0; r < rows; ++r) {
+    static _Thread_local double mk[REF_MAX_BETA][REF_MX_BLOCK];
+    static _Thread_local double Lk[REF_MAX_BETA][REF_MAX_DQ];
+    double acc = 0.0;
+    for (int64_t b = 0; b < nbc; ++b) {
+      const uint16_t* w = W + r * ld + b * REF_MX_BLOCK;
+      float bmax = 0.0f;
+      for (int j = 0; j < REF_MX_BLOCK; ++j) {
+        float v = fabsf(soar_ref_bf16_to_f32(w[j]));
+        if (v > bmax) bmax = v;
+      }
+      double m[REF_MX_BLOCK];
+      uint8_t code = 0;
+      if (tie_flags) tie_flags[r * nbc + b] = 0;
+      if (bmax < 0x1p-120f) {
+        for (int j = 0; j < REF_MX_BLOCK; ++j) m[j] = 0.0;
+      } else if (n_beta == 0) {
+        code = soar_ref_mx_plain_code(bmax);
+        soar_ref_mx_round_block(w, (float)soar_ref_e8m0_decode(code), m);
+      } else {
+        float center = bmax / 6.0f;
+        uint8_t dc[REF_MAX_DQ];
+        int nd = soar_ref_mx_candidates(center, n_dq, dc);
+        double best = 0.0;
+        int bk = -1, bd = -1;
+        for (int k = 0; k < n_beta; ++k) {
+          float dq = center * soar_ref_beta(k, n_beta, step_pct);
+          soar_ref_mx_round_block(w, dq, mk[k]);
+          for (int d = 0; d < nd; ++d) {
+            double L = soar_ref_mx_block_error(w, mk[k], dc[d]);
+            Lk[k][d] = L;
+            if (bk < 0 || L < best) { best = L; bk = k; bd = d; }
+          }
+        }
+        double second = 1e300;
+        for (int k = 0; k < n_beta; ++k)
+          for (int d = 0; d < nd; ++d) {
+            if (dc[d] == dc[bd] && memcmp(mk[k], mk[bk], sizeof(mk[k])) == 0) continue;
+            if (Lk[k][d] < second) second = Lk[k][d];
+          }
+        if (tie_flags && second < 1e300) {
+          double gap = best > 0.0 ? (second - best) / best : (second > 0.0 ? 1e300 : 0.0);
+          if (gap < tie_rel) tie_flags[r * nbc + b] = 1;
+        }
+        code = dc[bd];
+        memcpy(m, mk[bk], sizeof(m));
+      }
+      acc += soar_ref_mx_block_error(w, m, code);
+      for (int j = 0; j < REF_MX_BLOCK; j += 2) {
+        int lo = soar_ref_e2m1_code(m[j]) | ((w[j] >> 15) << 3);
+        int hi = soar_ref_e2m1_code(m[j + 1]) | ((w[j + 1] >> 15) << 3);
+        out_packed[(r * cols + b * REF_MX_BLOCK + j) / 2] = (uint8_t)(lo | (hi << 4));
+      }
+      out_scales[r * nbc + b] = code;
+    }
+    rowL[r] = acc;
+  }
+  double sse = 0.0;
+  for (int64_t r = 0; r < rows; ++r) sse += rowL[r];
+  free(rowL);
+  *out_sse = sse;
+  return status;
 }

@@ -130,6 +130,19 @@ def lib() -> C.CDLL:
         L.soar_ref_dequant_error_weighted.argtypes = [
             u16p, C.c_int64, C.c_int64, C.c_int64, fp, u8p, u8p, C.c_float, dp, dp,
         ]
+        L.soar_ref_e8m0_decode.restype = C.c_double
+        L.soar_ref_e8m0_decode.argtypes = [C.c_uint8]
+        L.soar_ref_mx_plain_code.restype = C.c_uint8
+        L.soar_ref_mx_plain_code.argtypes = [C.c_float]
+        L.soar_ref_mx_candidates.restype = C.c_int
+        L.soar_ref_mx_candidates.argtypes = [C.c_float, C.c_int, u8p]
+        L.soar_ref_mx_round_block.restype = None
+        L.soar_ref_mx_round_block.argtypes = [u16p, C.c_float, dp]
+        L.soar_ref_mx_block_error.restype = C.c_double
+        L.soar_ref_mx_block_error.argtypes = [u16p, dp, C.c_uint8]
+        L.soar_ref_mx_quantize.restype = C.c_int
+        L.soar_ref_mx_quantize.argtypes = [u16p, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_int,
+                                           u8p, u8p, dp, dp, u8p, C.c_double]
         L.soar_ref_num_threads.restype = C.c_int
         _lib = L
     return _lib
@@ -263,3 +276,58 @@ def dq_candidates(center: float, n: int):
 
 def beta(k: int, n_beta: int, step_pct: int) -> float:
     return float(lib().soar_ref_beta(k, n_beta, step_pct))
+
+
+# ---- MXFP4 (Sec. 4.3 "DSS on MXFP4") ------------------------------------------------------
+
+@dataclass
+class RefMxResult:
+    packed: np.ndarray        # uint8 [rows, cols/2]
+    scales: np.ndarray        # uint8 [rows, cols/32], E8M0 codes
+    sse: float
+    sumsq: float
+    tie_flags: np.ndarray     # uint8 [rows, cols/32]
+    status: int
+
+
+def mx_quantize(w_bits: np.ndarray, n_dq: int = 2, n_beta: int = 101, beta_step_pct: int = 1,
+                tie_rel: float = 1e-6) -> RefMxResult:
+    """MXFP4 of a 2-D uint16 array of bf16 bit patterns; ``n_beta == 0`` is the format's plain rule."""
+    assert w_bits.dtype == np.uint16 and w_bits.ndim == 2 and w_bits.shape[1] % 32 == 0
+    rows, cols = w_bits.shape
+    w = np.ascontiguousarray(w_bits)
+    packed = np.zeros((rows, cols // 2), np.uint8)
+    scales = np.zeros((rows, cols // 32), np.uint8)
+    ties = np.zeros((rows, cols // 32), np.uint8)
+    sse, ss = C.c_double(0.0), C.c_double(0.0)
+    st = lib().soar_ref_mx_quantize(_u16(w), rows, cols, cols, n_dq, n_beta, beta_step_pct, _u8(packed), _u8(scales),
+                                    C.byref(sse), C.byref(ss), _u8(ties), tie_rel)
+    return RefMxResult(packed, scales, float(sse.value), float(ss.value), ties, int(st))
+
+
+def e8m0_decode(code: int) -> float:
+    return float(lib().soar_ref_e8m0_decode(int(code)))
+
+
+def mx_plain_code(bmax: float) -> int:
+    return int(lib().soar_ref_mx_plain_code(C.c_float(bmax)))
+
+
+def mx_candidates(center: float, n: int):
+    out = np.zeros(32, np.uint8)
+    k = lib().soar_ref_mx_candidates(C.c_float(center), n, _u8(out))
+    return [int(v) for v in out[:k]]
+
+
+def mx_round_block(w32: np.ndarray, dq: float) -> np.ndarray:
+    w = np.ascontiguousarray(w32, dtype=np.uint16)
+    assert w.size == 32
+    m = np.zeros(32, np.float64)
+    lib().soar_ref_mx_round_block(_u16(w), C.c_float(dq), m.ctypes.data_as(C.POINTER(C.c_double)))
+    return m
+
+
+def mx_block_error(w32: np.ndarray, m: np.ndarray, code: int) -> float:
+    w = np.ascontiguousarray(w32, dtype=np.uint16)
+    mm = np.ascontiguousarray(m, dtype=np.float64)
+    return float(lib().soar_ref_mx_block_error(_u16(w), mm.ctypes.data_as(C.POINTER(C.c_double)), C.c_uint8(code)))
