@@ -360,6 +360,43 @@ int soar_dequant_error_weighted(const void* W_bf16, int64_t rows, int64_t cols, 
                                 double* out_sse, double* out_sumsq, void* stream);
 
 /*
+ * MXFP4 with the decoupled scale search (Sec. 4.3, "DSS on MXFP4"): E2M1 codes in blocks of 32
+ * consecutive elements of a row, one E8M0 scale byte per block (value 2^(byte - 127)), no tensor
+ * scale.  The paper reports results for this combination and gives no procedure; the library
+ * follows this reading of Sec. 3.3 with alpha = 1:
+ *   n_beta == 0  the format's plain rule: shared exponent floor(log2 bmax) - 2, elements rounded to
+ *                nearest (ties to even) and saturated at 6;
+ *   n_beta >= 1  the search: the high-precision scale is Eq. 1's max-based one, D* = bmax / 6; the
+ *                dequantization candidates are the n_dq E8M0 values around D* (n_dq = 1: the nearer
+ *                one; n_dq >= 2: n_dq/2 at or below, n_dq/2 above; with two candidates the plain
+ *                rule's exponent is always one of them), the quantization candidates D* times
+ *                App. B.3's multipliers (n_beta of them, step beta_step_pct / 100, centred on 1.00);
+ *                every pair is scored by Eq. 8 and the first minimum in (multiplier, code) order is kept.
+ * A block whose largest magnitude is below 2^-120 is stored as a zero block (scale byte 0).
+ *
+ *   W_bf16            device, as soar_quantize, and cols % 32 == 0
+ *   out_fp4_packed    device, rows*cols/2 bytes, 16-byte aligned, nibble layout as soar_quantize
+ *   out_e8m0_scales   device, rows*cols/32 bytes, row-major
+ *   out_result        device, one soar_mx_result, 8-byte aligned (required: it also carries the
+ *                     call's running sums); status holds SOAR_STATUS_NONFINITE / _ZERO_TENSOR / _INTERNAL
+ * One pass over W, no workspace, nothing allocated, enqueued on `stream`.
+ */
+typedef struct soar_mx_result {
+  int32_t status;            /* SOAR_STATUS_* bits                                              */
+  uint32_t amax_bits;        /* bf16 bit pattern of max |W|                                     */
+  float amax;                /* max |W|                                                         */
+  int32_t pad_;
+  double sse;                /* sum (W - What)^2                                                */
+  double sumsq;              /* sum W^2                                                         */
+  double reserved;           /* internal: sse - sumsq before clamping                           */
+  int64_t zero_blocks;       /* blocks stored as zero blocks                                    */
+  int64_t wide_candidates;   /* candidate evaluations on the binary64 accumulation path         */
+} soar_mx_result;
+int soar_mx_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, int n_dq, int n_beta,
+                     int beta_step_pct, void* out_fp4_packed, void* out_e8m0_scales,
+                     soar_mx_result* out_result, void* stream);
+
+/*
  * soar_quantize without a workspace argument, for callers that must not allocate device
  * memory and have none to spare: code running inside another framework's memory pool, a
  * plugin or callback that is handed only its input and output buffers, a process whose

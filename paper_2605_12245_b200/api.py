@@ -31,7 +31,7 @@ EXPORTS = (
     "soar_batch_workspace_bytes", "soar_quantize_batch",
     "soar_weighted_workspace_bytes", "soar_quantize_weighted", "soar_dequant_error_weighted",
     "soar_quantize_stage", "soar_pipeline_create", "soar_pipeline_run", "soar_pipeline_synchronize",
-    "soar_pipeline_destroy", "soar_debug_fail_waits",
+    "soar_pipeline_destroy", "soar_debug_fail_waits", "soar_mx_quantize",
 )
 
 
@@ -53,6 +53,16 @@ class SoarResult(C.Structure):
         ("sse", C.c_double), ("sse_init", C.c_double), ("sumsq", C.c_double),
         ("zero_blocks", C.c_int64), ("wide_candidates", C.c_int64),
         ("trace_alpha", C.c_double * (MAX_ITERS + 1)), ("trace_sse", C.c_double * (MAX_ITERS + 1)),
+    ]
+
+
+class SoarMxResult(C.Structure):
+    """Mirror of ``soar_mx_result``."""
+
+    _fields_ = [
+        ("status", C.c_int32), ("amax_bits", C.c_uint32), ("amax", C.c_float), ("pad_", C.c_int32),
+        ("sse", C.c_double), ("sumsq", C.c_double), ("reserved", C.c_double),
+        ("zero_blocks", C.c_int64), ("wide_candidates", C.c_int64),
     ]
 
 
@@ -138,6 +148,8 @@ def lib() -> C.CDLL:
         L.soar_pipeline_synchronize.argtypes = [vp]
         L.soar_pipeline_destroy.restype = None
         L.soar_pipeline_destroy.argtypes = [vp]
+        L.soar_mx_quantize.restype = C.c_int
+        L.soar_mx_quantize.argtypes = [vp, i64, i64, i64, C.c_int, C.c_int, C.c_int, vp, vp, vp, vp]
         L.soar_debug_fail_waits.restype = C.c_int
         L.soar_debug_fail_waits.argtypes = [C.c_int]
         L.soar_selftest_reciprocal.restype = C.c_int
@@ -354,6 +366,36 @@ def soar_quantize_static(W: torch.Tensor, cfg: SoarCfg, out: QuantBuffers, strea
         _ptr(W), rows, cols, W.stride(0), C.byref(cfg), _ptr(out.packed), _ptr(out.scales),
         _ptr(out.scales_sw), _ptr(out.alpha), _ptr(out.result), _stream_ptr(stream))
     _check(rc, "soar_quantize_static")
+    return out
+
+
+@dataclass
+class MxBuffers:
+    """Device outputs of one MXFP4 call."""
+
+    packed: torch.Tensor      # uint8 [rows, cols/2]
+    scales: torch.Tensor      # uint8 [rows, cols/32], E8M0 codes
+    result: torch.Tensor      # uint8 [sizeof(soar_mx_result)]
+
+    def read_result(self) -> SoarMxResult:
+        return SoarMxResult.from_buffer_copy(self.result.cpu().numpy().tobytes())
+
+
+def soar_mx_quantize(W: torch.Tensor, n_dq: int = 2, n_beta: int = 101, beta_step_pct: int = 1,
+                     out: MxBuffers | None = None, stream=None) -> MxBuffers:
+    """Enqueue ``soar_mx_quantize`` (MXFP4, blocks of 32; ``n_beta == 0``: the format's plain rule)."""
+    _require_cuda(W)
+    if W.dtype != torch.bfloat16 or W.dim() != 2 or W.stride(1) != 1:
+        raise SoarError("W must be a 2-D bf16 tensor with unit column stride")
+    rows, cols = W.shape
+    if out is None:
+        u8 = dict(dtype=torch.uint8, device=W.device)
+        out = MxBuffers(torch.empty((rows, cols // 2), **u8), torch.empty((rows, max(cols // 32, 1)), **u8),
+                        torch.empty(C.sizeof(SoarMxResult), **u8))
+    _require_cuda(out.packed, out.scales, out.result)
+    rc = lib().soar_mx_quantize(_ptr(W), rows, cols, W.stride(0), n_dq, n_beta, beta_step_pct, _ptr(out.packed),
+                                _ptr(out.scales), _ptr(out.result), _stream_ptr(stream))
+    _check(rc, "soar_mx_quantize")
     return out
 
 

@@ -1949,6 +1949,153 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
   add_counters(p.ws, unused_zeros, exact_blocks);   // reported as soar_result.wide_candidates
 }
 
+// ------------------------------------------------------------------ MXFP4 (Sec. 4.3, "DSS on MXFP4")
+//
+// The other microscaling format: E2M1 elements in blocks of 32 with one shared power-of-two
+// scale (an E8M0 byte, value 2^(code - 127)) and no tensor-wide scale.  The paper reports results
+// and no procedure; the reading built here (the oracle's) is Sec. 3.3 (i)-(ii) with alpha = 1:
+//   plain rule  shared exponent floor(log2 bmax) - 2, elements rounded to nearest even, saturated;
+//   search      high-precision scale D* = fl(bmax / 6) (Eq. 1); dequantization candidates the n_dq E8M0
+//               values around D* (App. B.3's rule on powers of two; for two candidates the plain
+//               exponent is always one of them); quantization candidates D* * beta_k on App. B.3's
+//               grid; Eq. 8 over all pairs, first minimum in (beta, code) order.
+// Two neighbouring threads share a block of 32, sixteen elements each, and exchange their maxima and
+// block sums by shuffles inside the pair; everything else is the machinery of the NVFP4 kernels.
+// The whole grid is visited, in order: with a power-of-two scale and bf16 inputs an element sits
+// exactly on a rounding midpoint in a fifth of all blocks, so candidates with exactly equal errors
+// are the rule and only the grid order says which one Algorithm 1's strict comparison keeps.
+// One pass over W, no workspace.
+
+__device__ __forceinline__ double pair_sum(unsigned int pair_mask, double v) {
+  return v + __shfl_xor_sync(pair_mask, v, 1);
+}
+
+template <bool kSearch>
+__global__ void __launch_bounds__(kThreads, 2)
+mx_kernel(const __grid_constant__ Batch bt, uint8_t* scales, soar_mx_result* res, double* gsum, int n_dq, int n_beta,
+          int step_pct) {
+  __shared__ Ring ring;
+  __shared__ Slots<2> slots;
+  __shared__ float s_beta[kSearch ? SOAR_MAX_BETA : 1];
+  const Params& p = bt.t[0];
+  if (kSearch)
+    for (int k = threadIdx.x; k < n_beta; k += kThreads)
+      s_beta[k] = static_cast<float>((100.0 + static_cast<double>((k - n_beta / 2) * step_pct)) / 100.0);
+  slots_clear(slots);
+  ring_init(ring);
+  if (is_producer_warp()) {
+    if (threadIdx.x == kTile) ring_produce(ring, bt, 0, 1u);
+    return;
+  }
+  const unsigned int pair_mask = 3u << (threadIdx.x & 30u);
+  const bool first_of_pair = (threadIdx.x & 1u) == 0u;
+  double acc[2] = {0.0, 0.0};   // error minus sum W^2; sum W^2
+  unsigned int zeros = 0, wide = 0, mx = 0;
+  for (unsigned int n = 0;; ++n) {
+    uint4 v0, v1;
+    int ti;
+    unsigned int tile;
+    if (ring_consume(ring, bt, n, v0, v1, ti, tile) != 0) break;
+    const unsigned int b = tile * kTile + threadIdx.x;   // index of this thread's sixteen elements
+    if (b >= p.nblk) continue;                           // pairs leave together: nblk is even
+    const unsigned int u[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) mx = max(mx, max(u[i] & 0x7FFFu, (u[i] >> 16) & 0x7FFFu));
+    {
+      double s0 = 0.0, s1 = 0.0;
+      sumsq_block(u, s0, s1);
+      acc[1] += s0 + s1;
+    }
+    Block blk;
+    unpack_block(v0, v1, blk);
+    const float bmax = fmaxf(blk.bmax, __shfl_xor_sync(pair_mask, blk.bmax, 1));
+    uint2 codes;
+    int code = 0;
+    if (!(bmax >= 0x1p-120f)) {
+      // zero (or vanishing) block: scale code 0, zero codes with the inputs' sign bits
+      round_block(blk, 0.0f, codes.x, codes.y);
+      if (first_of_pair) ++zeros;
+    } else {
+      Fixed fx;
+      make_fixed(blk, fx);
+      double best;
+      float best_r;
+      if (!kSearch) {
+        const int X = static_cast<int>(__float_as_uint(bmax) >> 23) - 129;   // floor(log2 bmax) - 2
+        code = X + 127;
+        best_r = __uint_as_float(static_cast<unsigned int>(127 - X) << 23);   // 2^-X
+        unsigned int c0, c1;
+        double A, B;
+        round_block(blk, best_r, c0, c1);
+        block_sums(blk, fx, best_r, c0, c1, A, B, wide);
+        A = pair_sum(pair_mask, A);
+        B = pair_sum(pair_mask, B);
+        const double sd = __hiloint2double((code + 896) << 20, 0);   // 2^(code - 127)
+        best = sd * fma(sd, B, -2.0 * A);
+      } else {
+        const float center = __fdiv_rn(bmax, 6.0f);
+        const int cf = static_cast<int>(__float_as_uint(center) >> 23);      // biased: value 2^(cf - 127) <= center
+        int d_lo, d_hi;
+        if (n_dq <= 1) {
+          const float mid = __uint_as_float((static_cast<unsigned int>(cf) << 23) | 0x400000u);   // 1.5 * 2^(cf - 127)
+          d_lo = d_hi = center > mid ? cf + 1 : cf;
+        } else {
+          d_lo = cf - (n_dq / 2 - 1);
+          d_hi = cf + n_dq / 2;
+        }
+        best = __longlong_as_double(0x7FF0000000000000ll);
+        best_r = 1.0f;
+        for (int k = 0; k < n_beta; ++k) {
+          const float r = recip_scale(1.0f, __fmul_rn(center, s_beta[k]));
+          unsigned int c0, c1;
+          double A, B;
+          round_block(blk, r, c0, c1);
+          block_sums(blk, fx, r, c0, c1, A, B, wide);
+          A = pair_sum(pair_mask, A);
+          B = pair_sum(pair_mask, B);
+          int prev = -1;
+          for (int d = d_lo; d <= d_hi; ++d) {
+            const int dc = max(0, min(254, d));
+            if (dc == prev) continue;   // clipping at the ends of the E8M0 range repeats a code
+            prev = dc;
+            const double sd = __hiloint2double((dc + 896) << 20, 0);
+            const double g = sd * fma(sd, B, -2.0 * A);
+            if (g < best) { best = g; best_r = r; code = dc; }
+          }
+        }
+      }
+      round_block(blk, best_r, codes.x, codes.y);
+      if (first_of_pair) acc[0] += best;
+    }
+    reinterpret_cast<uint2*>(p.packed)[b] = codes;
+    if (first_of_pair) scales[b >> 1] = static_cast<uint8_t>(code);
+  }
+  mx = __reduce_max_sync(0xFFFFFFFFu, mx);
+  if ((threadIdx.x & 31) == 0 && mx) atomicMax(&res->amax_bits, mx);
+  unsigned int unused = 0;
+  zeros = __reduce_add_sync(0xFFFFFFFFu, zeros);
+  wide = __reduce_add_sync(0xFFFFFFFFu, wide);
+  if ((threadIdx.x & 31) == 0) {
+    if (zeros) atomicAdd(reinterpret_cast<unsigned long long*>(&res->zero_blocks), static_cast<unsigned long long>(zeros));
+    if (wide) atomicAdd(reinterpret_cast<unsigned long long*>(&res->wide_candidates), static_cast<unsigned long long>(wide));
+    if (*static_cast<volatile int*>(&ring.fail)) atomicOr(&res->status, SOAR_STATUS_INTERNAL);
+  }
+  (void)unused;
+  double* const dst[2] = {gsum, &res->sumsq};
+  slots_add(slots, 0, acc, dst);
+}
+
+// Status and error of an MXFP4 call from its sums.
+__global__ void mx_finalize_kernel(soar_mx_result* res, const double* gsum) {
+  const unsigned int amax_bits = res->amax_bits;
+  int st = res->status;
+  if (amax_bits >= 0x7F80u) st |= SOAR_STATUS_NONFINITE;
+  if (amax_bits == 0) st |= SOAR_STATUS_ZERO_TENSOR;
+  res->status = st;
+  res->amax = bits_to_mag(amax_bits);
+  res->sse = fmax(res->sumsq + *gsum, 0.0);
+}
+
 // Counts the binary32 inputs with biased exponent lo_exp..hi_exp (all 2^23 significands each)
 // on which recip_fast differs from rcp.rn.
 __global__ void selftest_reciprocal_kernel(unsigned int lo_exp, unsigned int hi_exp, unsigned long long* mismatches) {
@@ -1968,11 +2115,12 @@ __global__ void selftest_reciprocal_kernel(unsigned int lo_exp, unsigned int hi_
 // is bracketed by two CUDA events on the launching stream.
 enum KernelId {
   K_AMAX = 0, K_INIT, K_ITERATE, K_FINALIZE, K_SWIZZLE, K_DEQUANT_ERROR,
-  K_WEIGHTED_AMAX, K_WEIGHTED_INIT, K_WEIGHTED_ITERATE, K_COUNT
+  K_WEIGHTED_AMAX, K_WEIGHTED_INIT, K_WEIGHTED_ITERATE, K_MX, K_COUNT
 };
 const char* const kKernelNames[K_COUNT] = {"amax_kernel",          "init_kernel",          "iterate_kernel",
                                            "finalize_kernel",      "swizzle_kernel",       "dequant_error_kernel",
-                                           "weighted_amax_kernel", "weighted_init_kernel", "weighted_iterate_kernel"};
+                                           "weighted_amax_kernel", "weighted_init_kernel", "weighted_iterate_kernel",
+                                           "mx_kernel"};
 struct TraceRec {
   int id;
   cudaEvent_t e0, e1;
@@ -2748,6 +2896,49 @@ int soar_selftest_reciprocal(int lo_exp, int hi_exp, unsigned long long* out_mis
   if (cudaMemsetAsync(out_mismatches, 0, sizeof(unsigned long long), st) != cudaSuccess) return SOAR_ERR_CUDA;
   selftest_reciprocal_kernel<<<sm_count() * 8, 256, 0, st>>>(static_cast<unsigned int>(lo_exp),
                                                              static_cast<unsigned int>(hi_exp), out_mismatches);
+  return cudaGetLastError() == cudaSuccess ? SOAR_OK : SOAR_ERR_CUDA;
+}
+
+int soar_mx_quantize(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, int n_dq, int n_beta,
+                     int beta_step_pct, void* out_fp4_packed, void* out_e8m0_scales, soar_mx_result* out_result,
+                     void* stream) {
+  const int rc = check_shape(W_bf16, rows, cols, ld);
+  if (rc != SOAR_OK) return rc;
+  if (cols % 32 != 0) return SOAR_ERR_UNSUPPORTED;
+  if (out_fp4_packed == nullptr || out_e8m0_scales == nullptr || out_result == nullptr) return SOAR_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(out_fp4_packed) % 16 != 0 || reinterpret_cast<uintptr_t>(out_result) % 8 != 0)
+    return SOAR_ERR_UNSUPPORTED;
+  if (n_beta < 0 || n_beta > SOAR_MAX_BETA || n_dq < 1 || n_dq > SOAR_MAX_DQ || beta_step_pct < 0)
+    return SOAR_ERR_INVALID_ARG;
+  if (n_beta > 0 && 100 - (n_beta / 2) * beta_step_pct <= 0) return SOAR_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(out_result, 0, sizeof(soar_mx_result), st) != cudaSuccess) return SOAR_ERR_CUDA;
+  Batch bt;
+  memset(&bt, 0, sizeof(bt));
+  Params& p = bt.t[0];
+  p.W = static_cast<const uint16_t*>(W_bf16);
+  p.packed = static_cast<uint8_t*>(out_fp4_packed);
+  p.ld = ld;
+  p.nbc = static_cast<unsigned int>(cols / 16);
+  p.nblk = static_cast<unsigned int>(rows * (cols / 16));
+  p.ntiles = (p.nblk + kTile - 1) / kTile;
+  p.contiguous = (ld == cols) ? 1 : 0;
+  bt.n = 1;
+  bt.idle_producer = g_idle_producer;
+  bt.total_tiles = p.ntiles;
+  for (int j = 0; j < kMaxBatch; ++j) bt.tile_end[j] = j == 0 ? p.ntiles : 0xFFFFFFFFu;
+  uint8_t* sc = static_cast<uint8_t*>(out_e8m0_scales);
+  double* gsum = &out_result->reserved;   // the running sum of the blocks' errors minus sum W^2
+  {
+    ScopedLaunch sl(K_MX, st);
+    if (n_beta == 0)
+      mx_kernel<false><<<persistent_grid(mx_kernel<false>, p.ntiles, kThreads), kThreads, 0, st>>>(
+          bt, sc, out_result, gsum, n_dq, n_beta, beta_step_pct);
+    else
+      mx_kernel<true><<<persistent_grid(mx_kernel<true>, p.ntiles, kThreads), kThreads, 0, st>>>(
+          bt, sc, out_result, gsum, n_dq, n_beta, beta_step_pct);
+  }
+  mx_finalize_kernel<<<1, 1, 0, st>>>(out_result, gsum);
   return cudaGetLastError() == cudaSuccess ? SOAR_OK : SOAR_ERR_CUDA;
 }
 

@@ -55,7 +55,7 @@ def test_python_mirrors_of_the_public_structs_match_the_header(tmp_path):
     structs = {"soar_cfg": api.SoarCfg, "soar_result": api.SoarResult, "soar_tensor_desc": api.SoarTensorDesc,
                "soar_staging": api.SoarStaging, "soar_trace_entry": api.SoarTraceEntry,
                "soar_workspace_header": api.SoarWorkspaceHeader, "soar_slot": api.SoarSlot,
-               "soar_host_matrix": api.SoarHostMatrix}
+               "soar_host_matrix": api.SoarHostMatrix, "soar_mx_result": api.SoarMxResult}
     lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "soar.h"', "int main(void) {"]
     for cname, py in structs.items():
         lines.append(f'  printf("{cname} %zu\\n", sizeof({cname}));')
