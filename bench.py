@@ -593,9 +593,10 @@ def weighted_kernel_bytes_per_elem(name: str, cfg, t: int = 0) -> float:
 
 
 def run_weighted(args):
-    """The same step under the column-weighted objective: one soar_quantize_weighted call per tensor,
-    W and the column weights resident in HBM."""
+    """The same step under the column-weighted objective: one soar_quantize_weighted_batch call over the
+    workload's tensors, W and the column weights resident in HBM."""
     import torch
+    from ctypes import byref as ctypes_byref
 
     from paper_2605_12245_b200 import api
     from paper_2605_12245_b200 import sharding as SH
@@ -626,9 +627,17 @@ def run_weighted(args):
     elements = wl.elements
     stream = torch.cuda.current_stream()
 
+    batch_ws = torch.empty(int(api.lib().soar_weighted_batch_workspace_bytes(api._descs(dev_w, outs), len(dev_w),
+                                                                             ctypes_byref(cfg))),
+                           dtype=torch.uint8, device="cuda")
+
     def step():
-        for W, h, o in zip(dev_w, dev_h, outs):
-            api.soar_quantize_weighted(W, h, cfg, o, stream)
+        """One batched call over the workload's tensors (one call per tensor with --no-batch)."""
+        if args.no_batch:
+            for W, h, o in zip(dev_w, dev_h, outs):
+                api.soar_quantize_weighted(W, h, cfg, o, stream)
+        else:
+            api.soar_quantize_weighted_batch(dev_w, dev_h, cfg, outs, batch_ws, stream)
 
     def barrier():
         torch.cuda.synchronize()
@@ -749,6 +758,71 @@ def run_weighted(args):
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_mxfp4(args):
+    """The MXFP4 entry point (Sec. 4.3, DSS on MXFP4) on the same workloads: one soar_mx_quantize call per tensor,
+    W resident in HBM; one pass over W per call."""
+    import torch
+
+    from paper_2605_12245_b200 import api
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    api.lib()
+    peaks = load_peaks()
+    wl = pick_workload(args.workload)
+    n_beta = 0 if args.preset == "single_pass" else 101         # single_pass here: the format's plain rule
+    dev_w, outs = [], []
+    for i, spec in enumerate(wl.tensors):
+        dev_w.append(torch.from_numpy(wl.generate(i).view(np.int16)).view(torch.bfloat16).cuda())
+        outs.append(None)
+    elements = wl.elements
+    stream = torch.cuda.current_stream()
+
+    def step():
+        for i, W in enumerate(dev_w):
+            outs[i] = api.soar_mx_quantize(W, 2, n_beta, 1, outs[i], stream)
+
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    sampler.start()
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    res = [o.read_result() for o in outs]
+    byts = elements * (2.0 + 0.5 + 1.0 / 32)                    # read W; write codes and one scale byte per 32
+    gbs = byts / (ms * 1e-3) / 1e9
+    cpu = None
+    if not args.no_cpu:
+        from oracle import soar_ref as R
+        spec = wl.tensors[0]
+        rows = max(1, min(spec.rows, args.cpu_rows) // WL._chunk_rows(spec.cols)) * WL._chunk_rows(spec.cols)
+        w = wl.generate(0, 0, rows)
+        t0 = time.perf_counter()
+        R.mx_quantize(w, n_beta=n_beta)
+        dt = time.perf_counter() - t0
+        cpu = dict(value=2.0 * w.size / dt / 1e9, unit="GB/s", cores=R.num_threads(), kind="oracle",
+                   sample=f"first {rows} rows x {spec.cols} cols of tensor '{spec.name}', {dt:.1f} s")
+    print(json.dumps(dict(
+        metric="soar_quantize_bf16_input_throughput", value=2.0 * elements / (ms * 1e-3) / 1e9, unit="GB/s", n_gpus=1,
+        steps=args.steps, warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
+        dtype="f32", data="synthetic",
+        config=dict(workload=wl.name, format="mxfp4", search=("2 x 101 pairs" if n_beta else "plain rule"),
+                    tensors=len(wl.tensors), elements=elements,
+                    l2="inputs (%.2f GB per step) exceed the 126 MB L2" % (2 * elements / 1e9)),
+        elements_per_s=elements / (ms * 1e-3),
+        roofline=dict(bound="hbm", kernel="mx_kernel", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s",
+                      frac=gbs / peaks["hbm_gbs"], traffic=None, peak_source=peaks["source"]),
+        rel_error=[r.sse / r.sumsq for r in res], cpu_baseline=cpu, e2e=None,
+        gpu_launches=2 * len(wl.tensors) * args.steps, clocks=clocks)), flush=True)
 
 
 def run_row_sharded(args):
@@ -894,6 +968,8 @@ def main():
     ap.add_argument("--sweep", default="", help="comma-separated candidate-pair counts to time, one iteration each")
     ap.add_argument("--objective", default="plain", choices=["plain", "weighted"],
                     help="weighted: the column-weighted objective through soar_quantize_weighted")
+    ap.add_argument("--format", default="nvfp4", choices=["nvfp4", "mxfp4"],
+                    help="mxfp4: the MXFP4 entry point (preset single_pass = the format's plain rule)")
     ap.add_argument("--row-sharded", action="store_true",
                     help="split the workload's largest tensor by rows over the ranks (strong scaling)")
     ap.add_argument("--sweep-dq", default="", help="comma-separated counts of E4M3 codes per block to time with beta = 1")
@@ -912,6 +988,8 @@ def main():
         run_dry(args)
     elif args.impl == "reference":
         run_reference(args)
+    elif args.format == "mxfp4":
+        run_mxfp4(args)
     elif args.row_sharded:
         run_row_sharded(args)
     elif args.objective == "weighted":

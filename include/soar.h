@@ -339,8 +339,15 @@ int soar_dequant_error(const void* W_bf16, int64_t rows, int64_t cols, int64_t l
  *               binary64 and the stored scale code), plus rows*cols/16 bytes when the row-major
  *               scale layout is not requested.
  * Every other argument, the stream semantics, ownership and the error codes are those of
- * soar_quantize.  One matrix per call; the block sums are accumulated in binary64 in element
- * order, so the pass is bound by arithmetic, not by HBM, even with one candidate.
+ * soar_quantize.  The block sums are accumulated in binary64 in element order, so the pass is
+ * bound by arithmetic, not by HBM, even with one candidate.
+ *
+ * soar_quantize_weighted_batch is the same on n independent matrices with shared settings, walked
+ * by the same kernels (up to 16 matrices per launch) like soar_quantize_batch: `tensors` and
+ * `col_weights` are host arrays of n entries (col_weights[i]: the device vector of matrix i's
+ * `cols` weights), `workspace` is device scratch of soar_weighted_batch_workspace_bytes() (the sum
+ * of soar_weighted_workspace_bytes over the matrices), 256-byte aligned.  Every matrix gets exactly
+ * what soar_quantize_weighted gives it.
  */
 size_t soar_weighted_workspace_bytes(int64_t rows, int64_t cols, const soar_cfg* cfg);
 int soar_quantize_weighted(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld,
@@ -348,6 +355,10 @@ int soar_quantize_weighted(const void* W_bf16, int64_t rows, int64_t cols, int64
                            void* out_e4m3_scales, void* out_e4m3_scales_sw, float* out_global_fp32,
                            void* workspace, size_t workspace_bytes, soar_result* out_result,
                            void* stream);
+size_t soar_weighted_batch_workspace_bytes(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg);
+int soar_quantize_weighted_batch(const soar_tensor_desc* tensors, const float* const* col_weights, int n,
+                                 const soar_cfg* cfg, void* workspace, size_t workspace_bytes,
+                                 void* stream);
 
 /*
  * soar_dequant_error under the same column weights: *out_sse = sum h_j (W - code value *

@@ -32,6 +32,7 @@ EXPORTS = (
     "soar_weighted_workspace_bytes", "soar_quantize_weighted", "soar_dequant_error_weighted",
     "soar_quantize_stage", "soar_pipeline_create", "soar_pipeline_run", "soar_pipeline_synchronize",
     "soar_pipeline_destroy", "soar_debug_fail_waits", "soar_mx_quantize",
+    "soar_weighted_batch_workspace_bytes", "soar_quantize_weighted_batch",
 )
 
 
@@ -134,6 +135,11 @@ def lib() -> C.CDLL:
         L.soar_quantize_weighted.restype = C.c_int
         L.soar_quantize_weighted.argtypes = [vp, i64, i64, i64, vp, C.POINTER(SoarCfg), vp, vp, vp, vp, vp,
                                              C.c_size_t, vp, vp]
+        L.soar_weighted_batch_workspace_bytes.restype = C.c_size_t
+        L.soar_weighted_batch_workspace_bytes.argtypes = [C.POINTER(SoarTensorDesc), C.c_int, C.POINTER(SoarCfg)]
+        L.soar_quantize_weighted_batch.restype = C.c_int
+        L.soar_quantize_weighted_batch.argtypes = [C.POINTER(SoarTensorDesc), C.POINTER(C.c_void_p), C.c_int,
+                                                   C.POINTER(SoarCfg), vp, C.c_size_t, vp]
         L.soar_dequant_error_weighted.restype = C.c_int
         L.soar_dequant_error_weighted.argtypes = [vp, i64, i64, i64, vp, vp, vp, C.c_int, vp, vp, vp, vp]
         L.soar_quantize_stage.restype = C.c_int
@@ -324,6 +330,30 @@ def soar_quantize_batch(Ws, cfg: SoarCfg, outs, workspace: torch.Tensor | None =
     _require_cuda(workspace)
     rc = lib().soar_quantize_batch(d, len(Ws), C.byref(cfg), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
     _check(rc, "soar_quantize_batch")
+    return workspace
+
+
+def soar_quantize_weighted_batch(Ws, col_weights, cfg: SoarCfg, outs, workspace: torch.Tensor | None = None,
+                                 stream=None):
+    """Enqueue ``soar_quantize_weighted_batch``: a list of bf16 CUDA matrices, one float32 CUDA weight vector per
+    matrix, their ``QuantBuffers`` (own ``workspace`` fields unused) and one uint8 CUDA ``workspace`` of
+    ``soar_weighted_batch_workspace_bytes`` (allocated here when omitted).  Returns the workspace."""
+    d = _descs(Ws, outs)
+    n = len(Ws)
+    for W, h in zip(Ws, col_weights):
+        _require_cuda(h)
+        if h.dtype != torch.float32 or h.shape != (W.shape[1],) or not h.is_contiguous():
+            raise SoarError("each col_weight must be a contiguous float32 vector with one entry per column")
+    if workspace is None:
+        need = int(lib().soar_weighted_batch_workspace_bytes(d, n, C.byref(cfg)))
+        if need == 0:
+            raise SoarError("soar_weighted_batch_workspace_bytes rejected the shapes or cfg")
+        workspace = torch.empty(need, dtype=torch.uint8, device=Ws[0].device)
+    _require_cuda(workspace)
+    hp = (C.c_void_p * n)(*[h.data_ptr() for h in col_weights])
+    rc = lib().soar_quantize_weighted_batch(d, hp, n, C.byref(cfg), _ptr(workspace), workspace.numel(),
+                                            _stream_ptr(stream))
+    _check(rc, "soar_quantize_weighted_batch")
     return workspace
 
 

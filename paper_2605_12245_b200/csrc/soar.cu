@@ -34,7 +34,7 @@
 // taken.  Tensor sums and candidate comparisons are binary64.
 //
 // Column-weighted objective (Sec. 5 in diagonal form; soar_quantize_weighted): the same passes as
-// weighted_amax_kernel, weighted_init_kernel and weighted_iterate_kernel, one matrix per launch.
+// weighted_amax_kernel, weighted_init_kernel and weighted_iterate_kernel (batched like the others).
 // Block sums carry a binary32 weight per column, so they are binary64 sums in element order
 // (17 bytes of state per block); the candidate loop ranks on exact integer sums over
 // fixed-point images of the weighted magnitudes and falls back to binary64 sums only for
@@ -943,25 +943,30 @@ __device__ __forceinline__ float grid_divisor(float alpha, float center, float b
 // For a fixed dequantization scale sd = alpha * value(code) the error of element j,
 // (a_j - m sd)^2, is convex in its code value m with its minimum at a_j / sd.  The codes
 // m_j(k) = E2M1(fl(a_j * fl(1 / s_k))), s_k = grid_divisor(beta_k), never rise with k, because every
-// step of that binary32 chain is monotone.  While s_k <= sd (1 - 2^-23) every fl(a_j * fl(1 / s_k)) is at
-// least a_j / sd (two roundings of 2^-24 each), so every code is at or above the nearest one
-// to a_j / sd and each element's error can only fall as k grows; once s_k >= sd (1 + 2^-22) every code
-// is at or below it and the error can only rise.  The block error of Eq. 8 is therefore smallest at
-// the last multiplier of the first kind, at the first of the second kind, or at one in between
-// (the band is 2^-21 wide against a grid step of a hundredth: almost always empty): two
-// multipliers in the typical case, where the grid has 101.
+// step of that binary32 chain is monotone.  While s_k <= sd (1 - 2^-21) every fl(a_j * fl(1 / s_k)) lies
+// above a_j / sd (by at least 2^-22 of it: the chain's two roundings cost 2^-24 each), so every code
+// is at or above the nearest one to a_j / sd and each element's error can only fall as k grows; once
+// s_k >= sd (1 + 2^-21) every scaled value lies below a_j / sd, every code is at or below the nearest
+// one and the error can only rise.  The block error of Eq. 8 is therefore smallest at the last
+// multiplier of the first kind, at the first of the second kind, or at one in between (the band is
+// 2^-20 wide against a grid step of a hundredth: almost always empty): two multipliers in the typical
+// case, where the grid has 101.
 //
-// Equal errors.  Different codes of an element cost the same only when a_j / sd is exactly a
-// rounding midpoint, which needs sd, and with it alpha, to have at most eight significant bits;
-// callers send such tensors through the whole grid, so that the first minimum in grid order is
-// kept as Algorithm 1's strict comparison keeps it.
+// Equal errors.  Two multipliers with the same codes are one outcome (the quantization scale is
+// never stored).  Different codes of an element cost the same only when a_j / sd is exactly a
+// rounding midpoint; because the band keeps the scaled value of such an element strictly above the
+// midpoint before it and strictly below after it, the element holds its upper code for every
+// multiplier before the band and its lower code for every one after, whatever the tie rule of
+// the rounding: all of its free code changes happen among the multipliers of [ka, kb].  Those are
+// scored in grid order with Algorithm 1's strict comparison, and outside [ka, kb] the error changes
+// strictly with every code change, so the first minimum of the whole grid has the codes of the
+// first minimum found here.
 
-// Binary32 bounds of the band around sd = alpha * dv (the exact product): lo <= sd (1 - 2^-23) and
-// hi >= sd (1 + 2^-22), from the directed roundings of the product moved two and four units in the
-// last place (one unit is more than 2^-24 of the value).
+// Binary32 bounds of the band around sd = alpha * dv (the exact product): lo <= sd (1 - 2^-21) and
+// hi >= sd (1 + 2^-21), by directed roundings.
 __device__ __forceinline__ void divisor_band(float alpha, float dv, float& lo, float& hi) {
-  lo = __uint_as_float(__float_as_uint(__fmul_rd(alpha, dv)) - 2u);
-  hi = __uint_as_float(__float_as_uint(__fmul_ru(alpha, dv)) + 4u);
+  lo = __fmul_rd(__fmul_rd(alpha, dv), 1.0f - 0x1p-21f);
+  hi = __fmul_ru(__fmul_ru(alpha, dv), 1.0f + 0x1p-21f);
 }
 
 // The range [ka, kb] of multipliers that can win for a code whose band is [lo, hi], for any start
@@ -977,53 +982,12 @@ __device__ __forceinline__ void winning_range(const float* s_beta, int n_beta, f
   kb = min(kb, n_beta - 1);
 }
 
-// True when different codes of an element can cost exactly the same under this alpha (see
-// above): alpha has at most eight significant bits.
-__device__ __forceinline__ bool alpha_allows_exact_ties(float alpha) {
-  return (__float_as_uint(alpha) & 0xFFFFu) == 0u;
-}
-
 // A block's winner of Eq. 8: error minus sum W^2, its sums, codes (signs included) and E4M3 code.
 struct Winner {
   double g, A, B;
   unsigned int c0, c1;
   int d;
 };
-
-// Eq. 8 over the whole grid for the block at `w16` (sixteen bf16 values in global memory), beta
-// ascending, then scale code ascending; strict '<' keeps the first minimum.  Out of line, and
-// fed from memory rather than from the caller's registers: it serves only tensors that can
-// have exactly equal candidates.
-__device__ __forceinline__ void whole_grid_search(const uint16_t* w16, float alpha, float center, const float* s_beta,
-                                               int n_beta, int d_lo, int nd, Winner* out, unsigned int* wide_out) {
-  const uint4* src = reinterpret_cast<const uint4*>(w16);
-  Block blk;
-  unpack_block(__ldg(src), __ldg(src + 1), blk);
-  Fixed fx;
-  make_fixed(blk, fx);
-  const double alpha_d = static_cast<double>(alpha);
-  Winner w;
-  w.g = __longlong_as_double(0x7FF0000000000000ll);
-  w.d = clip_code(d_lo);
-  w.A = w.B = 0.0;
-  w.c0 = w.c1 = 0u;
-  unsigned int wide = 0;
-  for (int k = 0; k < n_beta; ++k) {
-    const float r = recip_scale(alpha, __fmul_rn(center, s_beta[k]));
-    unsigned int c0, c1;
-    double A, B;
-    round_block(blk, r, c0, c1);
-    block_sums(blk, fx, r, c0, c1, A, B, wide);
-    for (int d = 0; d < nd; ++d) {
-      const int dc = clip_code(d_lo + d);
-      const double sd = alpha_d * static_cast<double>(e4m3_value(dc));
-      const double g = sd * fma(sd, B, -2.0 * A);
-      if (g < w.g) { w.g = g; w.A = A; w.B = B; w.c0 = c0; w.c1 = c1; w.d = dc; }
-    }
-  }
-  *out = w;
-  *wide_out += wide;
-}
 
 // One candidate of the search scored on the exact integer sums: codes (signs included), afix, 4B and
 // e = rho * 4B - afix, which orders candidates of one E4M3 code like their errors.
@@ -1087,7 +1051,6 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
   }
   float alpha = 1.0f;
   double alpha_d = 1.0;
-  bool whole_grid = false;           // mode 4: the current tensor's alpha allows exactly equal candidates
   // mode 4: multiplier index of a scale ratio, k = (ratio - 1) * 100 / step + n_beta / 2
   const float k_scale = 100.0f / static_cast<float>(max(bt.t[0].beta_step_pct, 1));
   const float k_off = static_cast<float>(n_beta / 2) - k_scale;   // k = (dv / center) * k_scale + k_off
@@ -1118,7 +1081,6 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
       cur = ti;
       alpha = s_alpha[ti];
       alpha_d = static_cast<double>(alpha);
-      whole_grid = alpha_allows_exact_ties(alpha);
       if (kMode != 0) p = tensor_view(bt.t[ti]);
     }
     // the long candidate loop does better re-reading these from the parameter block per tile than
@@ -1175,19 +1137,7 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
       }
     } else if (kMode == 4) {
       const int nd = d_hi - d_lo + 1;
-      if (whole_grid) {   // the same for every block of the tensor
-        const Params& q = bt.t[ti];
-        const unsigned int row = b / q.nbc, cb = b - row * q.nbc;
-        Winner w;
-        whole_grid_search(q.W + static_cast<long long>(row) * q.ld + static_cast<long long>(cb) * 16, alpha, center,
-                          s_beta, n_beta, d_lo, nd, &w, &wide);
-        best = w.g;
-        bestA = w.A;
-        bestB = w.B;
-        best0 = w.c0;
-        best1 = w.c1;
-        best_d = w.d;
-      } else {
+      {
         // Typical block: two E4M3 codes at most, each with exactly two multipliers that can win (the one
         // just below value(code) / center and its successor), the exact integer sums valid and the
         // fast reciprocal in range for the whole grid.  Those four candidates are scored in straight
@@ -1557,12 +1507,16 @@ __global__ void __launch_bounds__(kThreads) dequant_error_kernel(const __grid_co
 // in Eq. 5, Eq. 6 and the error of Eq. 8.  The weights are arbitrary binary32 numbers, so the
 // integer dot products of the unweighted kernels do not apply: the sums are binary64, taken in
 // element order (each product is exact: 24 + 8 + 2 and 24 + 4 significant bits), and the state
-// kept between iterations is {A, B} in binary64 plus the scale code.  One tensor per launch.
+// kept between iterations is {A, B} in binary64 plus the scale code.
 
 struct Weighted {
   const float* h;    // cols weights
   double2* sums;     // per block {A, B} of the current codes; null when T == 0
   uint8_t* code;     // per block stored scale code (0: all-zero block); null when T == 0
+};
+// One launch works on up to kMaxBatch matrices (see Batch): entry i belongs to bt.t[i].
+struct WeightedBatch {
+  Weighted t[kMaxBatch];
 };
 
 // A and B of a code vector (sign bits ignored) for hw[j] = h_j |w_j| and hd[j] = h_j.
@@ -1634,29 +1588,50 @@ __device__ __forceinline__ bool weight_ok(float h) {
 }
 
 // Eq. 1's tensor maximum, sum h_j W^2 for the error report, and the check of the weights.
-__global__ void __launch_bounds__(kThreads, 2) weighted_amax_kernel(const __grid_constant__ Batch bt, const float* h) {
+__global__ void __launch_bounds__(kThreads, 2)
+weighted_amax_kernel(const __grid_constant__ Batch bt, const __grid_constant__ WeightedBatch wb) {
   __shared__ Ring ring;
   __shared__ Slots<1> slots;
   slots_clear(slots);
   ring_init(ring);
   if (is_producer_warp()) {
-    if (threadIdx.x == kTile) ring_produce(ring, bt, 0, 1u);
+    if (threadIdx.x == kTile) ring_produce(ring, bt, 0, 0xFFFFFFFFu);
     return;
   }
-  const Params& p = bt.t[0];
-  unsigned int mx = 0;
+  unsigned int mx = 0, nblk = 0, nbc = 1;
+  const float* h = nullptr;
   bool bad = false;
   double sq[1] = {0.0};
+  int cur = -1;
   for (unsigned int n = 0;; ++n) {
     uint4 v0, v1;
-    int ti;
-    unsigned int tile;
-    if (ring_consume(ring, bt, n, v0, v1, ti, tile) != 0) break;
+    int ti = -1;
+    unsigned int tile = 0;
+    const int rc = ring_consume(ring, bt, n, v0, v1, ti, tile);
+    if (rc != 0 || ti != cur) {
+      if (cur >= 0) {   // leaving tensor `cur`: hand over its maximum, its sum and the verdict on its weights
+        mx = __reduce_max_sync(0xFFFFFFFFu, mx);
+        const bool any_bad = __any_sync(0xFFFFFFFFu, bad);
+        if ((threadIdx.x & 31) == 0) {
+          if (mx) atomicMax(&bt.t[cur].ws->amax_bits, mx);
+          if (any_bad) atomicOr(&bt.t[cur].ws->error, kErrWeight);
+        }
+        double* const dst[1] = {&bt.t[cur].ws->sumsq};
+        slots_add(slots, cur, sq, dst);
+        mx = 0;
+        bad = false;
+      }
+      if (rc != 0) break;
+      cur = ti;
+      nblk = bt.t[ti].nblk;
+      nbc = bt.t[ti].nbc;
+      h = wb.t[ti].h;
+    }
     const unsigned int b = tile * kTile + threadIdx.x;
-    if (b >= p.nblk) continue;
+    if (b >= nblk) continue;
     const unsigned int u[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
     double hd[16];
-    load_weights(h, b % p.nbc, hd);
+    load_weights(h, b % nbc, hd);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       // magnitude bit patterns order like the magnitudes; NaN patterns lie above infinity's
@@ -1668,44 +1643,58 @@ __global__ void __launch_bounds__(kThreads, 2) weighted_amax_kernel(const __grid
       bad = bad || !weight_ok(static_cast<float>(hd[2 * i])) || !weight_ok(static_cast<float>(hd[2 * i + 1]));
     }
   }
-  mx = __reduce_max_sync(0xFFFFFFFFu, mx);
-  const bool any_bad = __any_sync(0xFFFFFFFFu, bad);
-  if ((threadIdx.x & 31) == 0) {
-    if (mx) atomicMax(&p.ws->amax_bits, mx);
-    if (any_bad) atomicOr(&p.ws->error, kErrWeight);
-  }
-  double* const dst[1] = {&p.ws->sumsq};
-  slots_add(slots, 0, sq, dst);
 }
 
 // Algorithm 1 "Initialization" (Eq. 1; the weights play no part in it), the first codes, and
 // the weighted stage-0 sums of Eq. 5 and of the starting error.
 __global__ void __launch_bounds__(kThreads, 2)
-weighted_init_kernel(const __grid_constant__ Batch bt, const Weighted wq, int reverse, int final) {
+weighted_init_kernel(const __grid_constant__ Batch bt, const __grid_constant__ WeightedBatch wb, int reverse,
+                     int final) {
   __shared__ Ring ring;
   __shared__ Slots<3> slots;
   slots_clear(slots);
   ring_init(ring);
-  const Params& p = bt.t[0];
   if (is_producer_warp()) {
     if (threadIdx.x == kTile) {
-      const bool run = !(status_from_amax(p.ws->amax_bits) & (SOAR_STATUS_NONFINITE | SOAR_STATUS_RANGE)) &&
-                       p.ws->error == 0;
-      ring_produce(ring, bt, reverse, run ? 1u : 0u);
+      unsigned int run = 0;
+      for (int i = 0; i < bt.n; ++i)
+        if (!(status_from_amax(bt.t[i].ws->amax_bits) & (SOAR_STATUS_NONFINITE | SOAR_STATUS_RANGE)) &&
+            bt.t[i].ws->error == 0)
+          run |= 1u << i;
+      ring_produce(ring, bt, reverse, run);
     }
     return;
   }
-  const unsigned int amax_bits = p.ws->amax_bits;
-  const float alpha = amax_bits == 0 ? 1.0f : __fdiv_rn(bits_to_mag(amax_bits), 2688.0f);
-  const float six_alpha = __fmul_rn(alpha, 6.0f);
-  const double alpha_d = static_cast<double>(alpha);
+  float alpha = 1.0f, six_alpha = 6.0f;
+  double alpha_d = 1.0;
   double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum
   unsigned int zeros = 0, unused_wide = 0;
+  int cur = -1;
+  Tensor p = {};
+  Weighted wq = {};
+  unsigned int nbc = 1;
   for (unsigned int n = 0;; ++n) {
     uint4 v0, v1;
-    int ti;
-    unsigned int tile;
-    if (ring_consume(ring, bt, n, v0, v1, ti, tile) != 0) break;
+    int ti = -1;
+    unsigned int tile = 0;
+    const int rc = ring_consume(ring, bt, n, v0, v1, ti, tile);
+    if (rc != 0 || ti != cur) {
+      if (cur >= 0) {
+        Ws* ws = bt.t[cur].ws;
+        double* const dst[3] = {&ws->num[0], &ws->den[0], &ws->gsum[0]};
+        slots_add(slots, cur, acc, dst);
+        add_counters(ws, zeros, unused_wide);
+      }
+      if (rc != 0) break;
+      cur = ti;
+      const unsigned int amax_bits = bt.t[ti].ws->amax_bits;
+      alpha = amax_bits == 0 ? 1.0f : __fdiv_rn(bits_to_mag(amax_bits), 2688.0f);
+      six_alpha = __fmul_rn(alpha, 6.0f);
+      alpha_d = static_cast<double>(alpha);
+      p = tensor_view(bt.t[ti]);
+      nbc = bt.t[ti].nbc;
+      wq = wb.t[ti];
+    }
     const unsigned int b = tile * kTile + threadIdx.x;
     if (b >= p.nblk) continue;
     Block blk;
@@ -1724,7 +1713,7 @@ weighted_init_kernel(const __grid_constant__ Batch bt, const Weighted wq, int re
     const float v = e4m3_value(c);
     round_block(blk, recip_scale(alpha, v), codes.x, codes.y);
     double hd[16], hw[16];
-    load_weights(wq.h, b % p.nbc, hd);
+    load_weights(wq.h, b % nbc, hd);
 #pragma unroll
     for (int j = 0; j < 16; ++j) hw[j] = hd[j] * static_cast<double>(fabsf(blk.w[j]));
     double A, B;
@@ -1743,9 +1732,6 @@ weighted_init_kernel(const __grid_constant__ Batch bt, const Weighted wq, int re
     acc[1] = fma(B * vd, vd, acc[1]);
     acc[2] += sd * fma(sd, B, -2.0 * A);
   }
-  double* const dst[3] = {&p.ws->num[0], &p.ws->den[0], &p.ws->gsum[0]};
-  slots_add(slots, 0, acc, dst);
-  add_counters(p.ws, zeros, unused_wide);
 }
 
 // Eq. 8 for one block over the whole grid with binary64 sums for every candidate, first minimum in
@@ -1810,49 +1796,69 @@ __device__ __noinline__ void weighted_whole_grid_search(const float* h, unsigned
 // One iteration t of Algorithm 1 under the weighted objective: Eq. 5 from the stage-t sums,
 // Eq. 6 per block from its stored {A, B}, App. B.3's candidates, Eq. 8 with the weighted
 // error written as  sum h w^2 + sd^2 B - 2 sd A  (sd = alpha * candidate scale value), first
-// minimum in (beta, code) order.  All of cfg's shapes and arms run through this one loop.
+// minimum in (beta, code) order.  All of cfg's shapes and arms run through this one kernel, on up
+// to kMaxBatch matrices per launch like the unweighted kernels.
 __global__ void __launch_bounds__(kThreads, 2)
-weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int t, int reverse, int emit,
-                        int keep) {
+weighted_iterate_kernel(const __grid_constant__ Batch bt, const __grid_constant__ WeightedBatch wb, int t,
+                        int reverse, int emit, int keep) {
   __shared__ Ring ring;
   __shared__ Slots<3> slots;
   __shared__ float s_beta[SOAR_MAX_BETA];
-  __shared__ float s_alpha;
-  __shared__ int s_run;
-  const Params& p = bt.t[0];
-  if (threadIdx.x == 0) {
+  __shared__ float s_alpha[kMaxBatch];
+  __shared__ unsigned int s_run;
+  if (threadIdx.x == 0) s_run = 0;
+  __syncthreads();
+  if (threadIdx.x < bt.n) {   // per tensor: still running?  its alpha for this iteration
     float a;
     int run;
-    iteration_head(p, t, a, run);
-    s_alpha = a;
-    s_run = run;
+    iteration_head(bt.t[threadIdx.x], t, a, run);
+    s_alpha[threadIdx.x] = a;
+    if (run) atomicOr(&s_run, 1u << threadIdx.x);
   }
-  const int n_dq = p.n_dq, n_beta = p.n_beta;
+  const Params& p0 = bt.t[0];
+  const int n_dq = p0.n_dq, n_beta = p0.n_beta;
   for (int k = threadIdx.x; k < n_beta; k += kThreads)
-    s_beta[k] = static_cast<float>((100.0 + static_cast<double>((k - n_beta / 2) * p.beta_step_pct)) / 100.0);
+    s_beta[k] = static_cast<float>((100.0 + static_cast<double>((k - n_beta / 2) * p0.beta_step_pct)) / 100.0);
   slots_clear(slots);
   __syncthreads();
-  if (s_run == 0) return;   // stopped earlier (Sec. 4.1), or the input was rejected
+  if (s_run == 0) return;   // every tensor of the batch has stopped (Sec. 4.1), or was rejected
   ring_init(ring);
   if (is_producer_warp()) {
-    if (threadIdx.x == kTile) ring_produce(ring, bt, reverse, 1u);
+    if (threadIdx.x == kTile) ring_produce(ring, bt, reverse, s_run);
     return;
   }
-  const float alpha = s_alpha;
-  const double alpha_d = static_cast<double>(alpha);
-  const bool coupled = (p.flags & SOAR_FLAG_COUPLED_SCALE) != 0;
-  const bool keep_scale = (p.flags & SOAR_FLAG_KEEP_BLOCK_SCALE) != 0;
+  float alpha = 1.0f;
+  double alpha_d = 1.0;
+  const bool coupled = (p0.flags & SOAR_FLAG_COUPLED_SCALE) != 0;
+  const bool keep_scale = (p0.flags & SOAR_FLAG_KEEP_BLOCK_SCALE) != 0;
   // multiplier index of a scale ratio: k = (ratio - 1) * 100 / step + n_beta / 2
-  const bool bracketed = p.beta_step_pct >= 1 && n_beta >= 2;
-  const float k_scale = 100.0f / static_cast<float>(max(p.beta_step_pct, 1));
+  const bool bracketed = p0.beta_step_pct >= 1 && n_beta >= 2;
+  const float k_scale = 100.0f / static_cast<float>(max(p0.beta_step_pct, 1));
   const float k_off = static_cast<float>(n_beta / 2) - k_scale;
   double acc[3] = {0.0, 0.0, 0.0};   // num, den, gsum of stage t+1
   unsigned int exact_blocks = 0, unused_zeros = 0;
+  int cur = -1;
   for (unsigned int n = 0;; ++n) {
     uint4 v0, v1;
-    int ti;
-    unsigned int tile;
-    if (ring_consume(ring, bt, n, v0, v1, ti, tile) != 0) break;
+    int ti = -1;
+    unsigned int tile = 0;
+    const int rc = ring_consume(ring, bt, n, v0, v1, ti, tile);
+    if (rc != 0 || ti != cur) {
+      if (cur >= 0) {
+        Ws* ws = bt.t[cur].ws;
+        double* const dst[3] = {&ws->num[t + 1], &ws->den[t + 1], &ws->gsum[t + 1]};
+        slots_add(slots, cur, acc, dst);
+        add_counters(ws, unused_zeros, exact_blocks);   // reported as soar_result.wide_candidates
+      }
+      if (rc != 0) break;
+      cur = ti;
+      alpha = s_alpha[ti];
+      alpha_d = static_cast<double>(alpha);
+    }
+    // pointers and sizes of the current tensor are re-read from the parameter block per tile rather than
+    // carried in registers across the scoring of the block
+    const Params& p = bt.t[ti];
+    const Weighted& wq = wb.t[ti];
     const unsigned int b = tile * kTile + threadIdx.x;
     if (b >= p.nblk) continue;
     const int d_cur = wq.code[b];
@@ -1881,16 +1887,16 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
       }
     }
     // The weighted error of element j, h_j (a_j - m sd)^2, is convex in m like the unweighted one, so per
-    // E4M3 code only the multipliers of winning_range can win (see there).  Candidates can cost exactly the
-    // same when alpha has few significant bits or when a column's weight is zero (its code then costs
-    // nothing, whatever it is): such blocks, and the coupled arm, walk the whole grid.
+    // E4M3 code only the multipliers of winning_range can win (see there).  When a column's weight is zero,
+    // its code costs nothing whatever it is, and equal errors of different codes occur all along the grid:
+    // such blocks, and the coupled arm, walk the whole grid.
     bool zero_weight = false;
 #pragma unroll
     for (int j = 0; j < 16; ++j) zero_weight = zero_weight || hf[j] == 0.0f;
     unsigned int best0 = 0, best1 = 0;
     double bestA = 0.0, bestB = 0.0;
     int best_d = clip_code(d_lo);
-    if (!coupled && bracketed && !zero_weight && !alpha_allows_exact_ties(alpha)) {
+    if (!coupled && bracketed && !zero_weight) {
       double best = __longlong_as_double(0x7FF0000000000000ll);
       int best_k = 0, prev = -1;
       const float per_center = __fdividef(k_scale, center);
@@ -1944,9 +1950,6 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
     acc[1] = fma(bestB * vd, vd, acc[1]);
     acc[2] += sd * fma(sd, bestB, -2.0 * bestA);
   }
-  double* const dst[3] = {&p.ws->num[t + 1], &p.ws->den[t + 1], &p.ws->gsum[t + 1]};
-  slots_add(slots, 0, acc, dst);
-  add_counters(p.ws, unused_zeros, exact_blocks);   // reported as soar_result.wide_candidates
 }
 
 // ------------------------------------------------------------------ MXFP4 (Sec. 4.3, "DSS on MXFP4")
@@ -1961,10 +1964,9 @@ weighted_iterate_kernel(const __grid_constant__ Batch bt, const Weighted wq, int
 //               grid; Eq. 8 over all pairs, first minimum in (beta, code) order.
 // Two neighbouring threads share a block of 32, sixteen elements each, and exchange their maxima and
 // block sums by shuffles inside the pair; everything else is the machinery of the NVFP4 kernels.
-// The whole grid is visited, in order: with a power-of-two scale and bf16 inputs an element sits
-// exactly on a rounding midpoint in a fifth of all blocks, so candidates with exactly equal errors
-// are the rule and only the grid order says which one Algorithm 1's strict comparison keeps.
-// One pass over W, no workspace.
+// Candidates with exactly equal errors are the rule here (a power-of-two scale and bf16 inputs put an
+// element exactly on a rounding midpoint in a fifth of all blocks), so the search keeps the grid's
+// order where it matters: see the comment in the kernel.  One pass over W, no workspace.
 
 __device__ __forceinline__ double pair_sum(unsigned int pair_mask, double v) {
   return v + __shfl_xor_sync(pair_mask, v, 1);
@@ -1989,6 +1991,10 @@ mx_kernel(const __grid_constant__ Batch bt, uint8_t* scales, soar_mx_result* res
   }
   const unsigned int pair_mask = 3u << (threadIdx.x & 30u);
   const bool first_of_pair = (threadIdx.x & 1u) == 0u;
+  // multiplier index of a scale ratio: k = (ratio - 1) * 100 / step + n_beta / 2
+  const bool bracketed = kSearch && n_beta >= kBracketMinBeta && step_pct >= 1;
+  const float k_scale = 100.0f / static_cast<float>(max(step_pct, 1));
+  const float k_off = static_cast<float>(n_beta / 2) - k_scale;
   double acc[2] = {0.0, 0.0};   // error minus sum W^2; sum W^2
   unsigned int zeros = 0, wide = 0, mx = 0;
   for (unsigned int n = 0;; ++n) {
@@ -2045,22 +2051,59 @@ mx_kernel(const __grid_constant__ Batch bt, uint8_t* scales, soar_mx_result* res
         }
         best = __longlong_as_double(0x7FF0000000000000ll);
         best_r = 1.0f;
-        for (int k = 0; k < n_beta; ++k) {
-          const float r = recip_scale(1.0f, __fmul_rn(center, s_beta[k]));
-          unsigned int c0, c1;
-          double A, B;
-          round_block(blk, r, c0, c1);
-          block_sums(blk, fx, r, c0, c1, A, B, wide);
-          A = pair_sum(pair_mask, A);
-          B = pair_sum(pair_mask, B);
-          int prev = -1;
+        if (!bracketed) {
+          // every multiplier in turn (grids of a few multipliers)
+          for (int k = 0; k < n_beta; ++k) {
+            const float r = recip_scale(1.0f, __fmul_rn(center, s_beta[k]));
+            unsigned int c0, c1;
+            double A, B;
+            round_block(blk, r, c0, c1);
+            block_sums(blk, fx, r, c0, c1, A, B, wide);
+            A = pair_sum(pair_mask, A);
+            B = pair_sum(pair_mask, B);
+            int prev = -1;
+            for (int d = d_lo; d <= d_hi; ++d) {
+              const int dc = max(0, min(254, d));
+              if (dc == prev) continue;   // clipping at the ends of the E8M0 range repeats a code
+              prev = dc;
+              const double sd = __hiloint2double((dc + 896) << 20, 0);
+              const double g = sd * fma(sd, B, -2.0 * A);
+              if (g < best) { best = g; best_r = r; code = dc; }
+            }
+          }
+        } else {
+          // Per E8M0 code only the multipliers around divisor = 2^(code - 127) can win (see winning_range's
+          // comment above iterate_kernel).  With a power-of-two scale and bf16 inputs, elements sit exactly on
+          // rounding midpoints in a fifth of all blocks, so equal errors of different codes are the rule here.
+          // The band is therefore 2^-21 wide on each side: before it the scaled value of such an element lies
+          // strictly above its midpoint for every multiplier (it keeps the upper code, whatever the tie rule),
+          // after it strictly below, so all of those free code changes happen inside [ka, kb], where the
+          // candidates are scored in grid order with the strict comparison of Algorithm 1; outside it the
+          // error changes strictly whenever a code changes.  The first minimum in (multiplier, code) order
+          // then has the codes of the first minimum found here.
+          int best_k = 0, prev = -1;
+          const float per_center = __fdividef(k_scale, center);
           for (int d = d_lo; d <= d_hi; ++d) {
             const int dc = max(0, min(254, d));
-            if (dc == prev) continue;   // clipping at the ends of the E8M0 range repeats a code
+            if (dc == prev) continue;
             prev = dc;
             const double sd = __hiloint2double((dc + 896) << 20, 0);
-            const double g = sd * fma(sd, B, -2.0 * A);
-            if (g < best) { best = g; best_r = r; code = dc; }
+            const float sdf = static_cast<float>(sd);                       // exact (2^-127 is a binary32 subnormal)
+            const float lo = __fmul_rn(sdf, 1.0f - 0x1p-21f), hi = __fmul_rn(sdf, 1.0f + 0x1p-21f);
+            int ka, kb;
+            winning_range(s_beta, n_beta, 1.0f, center, lo, hi, __float2int_rd(__fmaf_rn(sdf, per_center, k_off)), ka, kb);
+            for (int k = ka; k <= kb; ++k) {
+              const float r = recip_scale(1.0f, __fmul_rn(center, s_beta[k]));
+              unsigned int c0, c1;
+              double A, B;
+              round_block(blk, r, c0, c1);
+              block_sums(blk, fx, r, c0, c1, A, B, wide);
+              A = pair_sum(pair_mask, A);
+              B = pair_sum(pair_mask, B);
+              const double g = sd * fma(sd, B, -2.0 * A);
+              // equal errors: the earlier multiplier, then the smaller code, as in grid order
+              if (g < best || (g == best && k < best_k)) { best = g; best_r = r; code = dc; best_k = k; }
+            }
           }
         }
       }
@@ -2604,100 +2647,148 @@ size_t soar_weighted_workspace_bytes(int64_t rows, int64_t cols, const soar_cfg*
   return n;
 }
 
-int soar_quantize_weighted(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, const float* col_weight,
-                           const soar_cfg* cfg, void* out_fp4_packed, void* out_e4m3_scales,
-                           void* out_e4m3_scales_sw, float* out_global_fp32, void* workspace,
-                           size_t workspace_bytes, soar_result* out_result, void* stream) {
+size_t soar_weighted_batch_workspace_bytes(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg) {
+  if (tensors == nullptr || n <= 0) return 0;
+  size_t total = 0;
+  for (int i = 0; i < n; ++i) {
+    const size_t b = soar_weighted_workspace_bytes(tensors[i].rows, tensors[i].cols, cfg);
+    if (b == 0) return 0;
+    total += b;
+  }
+  return total;
+}
+
+int soar_quantize_weighted_batch(const soar_tensor_desc* tensors, const float* const* col_weights, int n,
+                                 const soar_cfg* cfg, void* workspace, size_t workspace_bytes, void* stream) {
   int rc = check_cfg(cfg);
   if (rc != SOAR_OK) return rc;
   if (cfg->flags & SOAR_FLAG_DETERMINISTIC) return SOAR_ERR_UNSUPPORTED;   // the weighted passes add with atomics only
-  rc = check_shape(W_bf16, rows, cols, ld);
-  if (rc != SOAR_OK) return rc;
+  if (tensors == nullptr || col_weights == nullptr || n <= 0) return SOAR_ERR_INVALID_ARG;
   const bool want_lin = (cfg->scale_layout & SOAR_SCALES_LINEAR) != 0;
   const bool want_sw = (cfg->scale_layout & SOAR_SCALES_SWIZZLED) != 0;
-  if (col_weight == nullptr || out_fp4_packed == nullptr || out_global_fp32 == nullptr) return SOAR_ERR_INVALID_ARG;
-  if (reinterpret_cast<uintptr_t>(col_weight) % 16 != 0 || reinterpret_cast<uintptr_t>(out_fp4_packed) % 16 != 0)
-    return SOAR_ERR_UNSUPPORTED;
-  if (want_lin && out_e4m3_scales == nullptr) return SOAR_ERR_INVALID_ARG;
-  if (want_sw && out_e4m3_scales_sw == nullptr) return SOAR_ERR_INVALID_ARG;
-  const size_t need = soar_weighted_workspace_bytes(rows, cols, cfg);
+  for (int i = 0; i < n; ++i) {   // every argument is checked before anything is enqueued
+    const soar_tensor_desc& d = tensors[i];
+    rc = check_shape(d.W_bf16, d.rows, d.cols, d.ld);
+    if (rc != SOAR_OK) return rc;
+    if (col_weights[i] == nullptr || d.out_fp4_packed == nullptr || d.out_global_fp32 == nullptr)
+      return SOAR_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(col_weights[i]) % 16 != 0 || reinterpret_cast<uintptr_t>(d.out_fp4_packed) % 16 != 0)
+      return SOAR_ERR_UNSUPPORTED;
+    if (want_lin && d.out_e4m3_scales == nullptr) return SOAR_ERR_INVALID_ARG;
+    if (want_sw && d.out_e4m3_scales_sw == nullptr) return SOAR_ERR_INVALID_ARG;
+  }
+  const size_t need = soar_weighted_batch_workspace_bytes(tensors, n, cfg);
   if (workspace == nullptr || need == 0 || workspace_bytes < need) return SOAR_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return SOAR_ERR_UNSUPPORTED;
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  uint8_t* next = static_cast<uint8_t*>(workspace);
-  if (cudaMemsetAsync(next, 0, kWsFixedBytes, st) != cudaSuccess) return SOAR_ERR_CUDA;
-  Batch bt;
-  Reports rp;
-  memset(&bt, 0, sizeof(bt));
-  memset(&rp, 0, sizeof(rp));
-  Params& p = bt.t[0];
-  p.W = static_cast<const uint16_t*>(W_bf16);
-  p.packed = static_cast<uint8_t*>(out_fp4_packed);
-  p.ws = reinterpret_cast<Ws*>(next);
-  next += kWsFixedBytes;
-  p.ld = ld;
-  p.nbc = static_cast<unsigned int>(cols / 16);
-  p.nblk = static_cast<unsigned int>(rows * (cols / 16));
-  p.ntiles = (p.nblk + kTile - 1) / kTile;
-  p.contiguous = (ld == cols) ? 1 : 0;
-  Weighted wq;
-  wq.h = col_weight;
-  wq.sums = nullptr;
-  wq.code = nullptr;
-  if (cfg->max_iters > 0) {
-    wq.sums = reinterpret_cast<double2*>(next);
-    next += round256(static_cast<size_t>(p.nblk) * sizeof(double2));
-    wq.code = next;
-    next += round256(p.nblk);
-  }
-  p.scales = want_lin ? static_cast<uint8_t*>(out_e4m3_scales) : next;
-  p.max_iters = cfg->max_iters;
-  p.early_stop_rel = cfg->early_stop_rel;
-  p.n_dq = cfg->n_dq;
-  p.n_beta = cfg->n_beta;
-  p.beta_step_pct = cfg->beta_step_pct;
-  p.flags = cfg->flags;
-  bt.n = 1;
-  bt.idle_producer = g_idle_producer;
-  bt.total_tiles = p.ntiles;
-  for (int j = 0; j < kMaxBatch; ++j) bt.tile_end[j] = j == 0 ? p.ntiles : 0xFFFFFFFFu;
-  rp.alpha[0] = out_global_fp32;
-  rp.result[0] = out_result;
-
-  const unsigned int tiles = p.ntiles;
-  int reverse = 1;   // the first pass runs forward; each later one starts where the last ended
-  {
-    ScopedLaunch sl(K_WEIGHTED_AMAX, st);
-    weighted_amax_kernel<<<persistent_grid(weighted_amax_kernel, tiles, kThreads), kThreads, 0, st>>>(bt, col_weight);
-  }
-  {
-    ScopedLaunch sl(K_WEIGHTED_INIT, st);
-    weighted_init_kernel<<<persistent_grid(weighted_init_kernel, tiles, kThreads), kThreads, 0, st>>>(
-        bt, wq, reverse, cfg->max_iters == 0 ? 1 : 0);
-  }
+  // workspace: the n headers first (one memset clears them all), then each tensor's arrays
+  uint8_t* const headers = static_cast<uint8_t*>(workspace);
+  uint8_t* next = headers + static_cast<size_t>(n) * kWsFixedBytes;
+  if (cudaMemsetAsync(headers, 0, static_cast<size_t>(n) * kWsFixedBytes, st) != cudaSuccess) return SOAR_ERR_CUDA;
   const bool may_stop = cfg->early_stop_rel > 0.0f;
-  const unsigned int g_it = persistent_grid(weighted_iterate_kernel, tiles, kThreads);
-  for (int t = 0; t < cfg->max_iters; ++t) {
-    reverse ^= 1;
-    const int last = (t == cfg->max_iters - 1) ? 1 : 0;
-    ScopedLaunch sl(K_WEIGHTED_ITERATE, st);
-    weighted_iterate_kernel<<<g_it, kThreads, 0, st>>>(bt, wq, t, reverse, (may_stop || last) ? 1 : 0, !last);
-  }
-  {
-    ScopedLaunch sl(K_FINALIZE, st);
-    finalize_kernel<<<1, 128, 0, st>>>(bt, rp, 0);
-  }
-  if (want_sw) {
-    const unsigned int rt = static_cast<unsigned int>((rows + 127) / 128);
-    const unsigned int ct = (p.nbc + 3) / 4;
-    const size_t blocks = (static_cast<size_t>(rt) * ct * 512 + 255) / 256;
-    const unsigned int grid = static_cast<unsigned int>(blocks < 65535u * 16u ? blocks : 65535u * 16u);
-    ScopedLaunch sl(K_SWIZZLE, st);
-    swizzle_kernel<<<grid, 256, 0, st>>>(p.scales, static_cast<uint8_t*>(out_e4m3_scales_sw),
-                                         static_cast<unsigned int>(rows), p.nbc, rt, ct);
+  for (int first = 0; first < n; first += kMaxBatch) {
+    Batch bt;
+    WeightedBatch wb;
+    Reports rp;
+    memset(&bt, 0, sizeof(bt));
+    memset(&wb, 0, sizeof(wb));
+    memset(&rp, 0, sizeof(rp));
+    bt.n = (n - first < kMaxBatch) ? n - first : kMaxBatch;
+    bt.idle_producer = g_idle_producer;
+    unsigned int tiles = 0;
+    for (int j = 0; j < bt.n; ++j) {
+      const soar_tensor_desc& d = tensors[first + j];
+      Params& p = bt.t[j];
+      Weighted& wq = wb.t[j];
+      p.W = static_cast<const uint16_t*>(d.W_bf16);
+      p.packed = static_cast<uint8_t*>(d.out_fp4_packed);
+      p.ws = reinterpret_cast<Ws*>(headers + static_cast<size_t>(first + j) * kWsFixedBytes);
+      p.ld = d.ld;
+      p.nbc = static_cast<unsigned int>(d.cols / 16);
+      p.nblk = static_cast<unsigned int>(d.rows * (d.cols / 16));
+      p.ntiles = (p.nblk + kTile - 1) / kTile;
+      p.contiguous = (d.ld == d.cols) ? 1 : 0;
+      wq.h = col_weights[first + j];
+      if (cfg->max_iters > 0) {
+        wq.sums = reinterpret_cast<double2*>(next);
+        next += round256(static_cast<size_t>(p.nblk) * sizeof(double2));
+        wq.code = next;
+        next += round256(p.nblk);
+      }
+      if (want_lin) {
+        p.scales = static_cast<uint8_t*>(d.out_e4m3_scales);
+      } else {
+        p.scales = next;
+        next += round256(p.nblk);
+      }
+      p.max_iters = cfg->max_iters;
+      p.early_stop_rel = cfg->early_stop_rel;
+      p.n_dq = cfg->n_dq;
+      p.n_beta = cfg->n_beta;
+      p.beta_step_pct = cfg->beta_step_pct;
+      p.flags = cfg->flags;
+      tiles += p.ntiles;
+      bt.tile_end[j] = tiles;
+      rp.alpha[j] = d.out_global_fp32;
+      rp.result[j] = d.out_result;
+    }
+    for (int j = bt.n; j < kMaxBatch; ++j) bt.tile_end[j] = 0xFFFFFFFFu;   // never reached by a tile index
+    bt.total_tiles = tiles;
+
+    int reverse = 1;   // the first pass runs forward; each later one starts where the last ended
+    {
+      ScopedLaunch sl(K_WEIGHTED_AMAX, st);
+      weighted_amax_kernel<<<persistent_grid(weighted_amax_kernel, tiles, kThreads), kThreads, 0, st>>>(bt, wb);
+    }
+    {
+      ScopedLaunch sl(K_WEIGHTED_INIT, st);
+      weighted_init_kernel<<<persistent_grid(weighted_init_kernel, tiles, kThreads), kThreads, 0, st>>>(
+          bt, wb, reverse, cfg->max_iters == 0 ? 1 : 0);
+    }
+    const unsigned int g_it = persistent_grid(weighted_iterate_kernel, tiles, kThreads);
+    for (int t = 0; t < cfg->max_iters; ++t) {
+      reverse ^= 1;
+      const int last = (t == cfg->max_iters - 1) ? 1 : 0;
+      ScopedLaunch sl(K_WEIGHTED_ITERATE, st);
+      weighted_iterate_kernel<<<g_it, kThreads, 0, st>>>(bt, wb, t, reverse, (may_stop || last) ? 1 : 0, !last);
+    }
+    {
+      ScopedLaunch sl(K_FINALIZE, st);
+      finalize_kernel<<<bt.n, 128, 0, st>>>(bt, rp, 0);
+    }
+    if (want_sw) {
+      for (int j = 0; j < bt.n; ++j) {
+        const soar_tensor_desc& d = tensors[first + j];
+        const Params& p = bt.t[j];
+        const unsigned int rt = static_cast<unsigned int>((d.rows + 127) / 128);
+        const unsigned int ct = (p.nbc + 3) / 4;
+        const size_t blocks = (static_cast<size_t>(rt) * ct * 512 + 255) / 256;
+        const unsigned int grid = static_cast<unsigned int>(blocks < 65535u * 16u ? blocks : 65535u * 16u);
+        ScopedLaunch sl(K_SWIZZLE, st);
+        swizzle_kernel<<<grid, 256, 0, st>>>(p.scales, static_cast<uint8_t*>(d.out_e4m3_scales_sw),
+                                             static_cast<unsigned int>(d.rows), p.nbc, rt, ct);
+      }
+    }
   }
   return cudaGetLastError() == cudaSuccess ? SOAR_OK : SOAR_ERR_CUDA;
+}
+
+int soar_quantize_weighted(const void* W_bf16, int64_t rows, int64_t cols, int64_t ld, const float* col_weight,
+                           const soar_cfg* cfg, void* out_fp4_packed, void* out_e4m3_scales,
+                           void* out_e4m3_scales_sw, float* out_global_fp32, void* workspace,
+                           size_t workspace_bytes, soar_result* out_result, void* stream) {
+  soar_tensor_desc d;
+  d.W_bf16 = W_bf16;
+  d.rows = rows;
+  d.cols = cols;
+  d.ld = ld;
+  d.out_fp4_packed = out_fp4_packed;
+  d.out_e4m3_scales = out_e4m3_scales;
+  d.out_e4m3_scales_sw = out_e4m3_scales_sw;
+  d.out_global_fp32 = out_global_fp32;
+  d.out_result = out_result;
+  return soar_quantize_weighted_batch(&d, &col_weight, 1, cfg, workspace, workspace_bytes, stream);
 }
 
 int soar_quantize_host(const void* W_host, int64_t rows, int64_t cols, int64_t ld, const soar_cfg* cfg,

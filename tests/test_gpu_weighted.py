@@ -218,3 +218,35 @@ def test_the_weighted_call_and_the_staged_calls_replay_from_a_cuda_graph():
     gpu2 = P.GpuOut(out2.packed.cpu().numpy(), out2.scales.cpu().numpy(), float(out2.alpha.cpu()[0]),
                     out2.read_result(), out2)
     P.assert_parity(gpu2, R.quantize(w, ref_cfg))
+
+
+def test_weighted_batch_gives_each_matrix_what_a_single_call_gives():
+    """Nineteen matrices with their own weight vectors through soar_quantize_weighted_batch (two launch groups,
+    one block to hundreds of tiles, a matrix with zero weights, one all zero, one with a bad weight): the same
+    bytes as separate soar_quantize_weighted calls, and the oracle's."""
+    shapes = [(1, 16), (3, 48), (37, 1040), (300, 4096), (64, 4096), (5, 16), (257, 512), (8, 8192), (600, 2064)] * 2 + \
+             [(96, 1024)]
+    ws = [WL.small_case(r, c, 500 + i, dist=("laplace" if i % 3 == 0 else "student_t4"),
+                        outlier_entry_frac=0.004 * (i % 2), outlier_scale=40.0) for i, (r, c) in enumerate(shapes)]
+    hs = [WL.column_weights(c, 600 + i, zero_frac=(0.1 if i == 4 else 0.0)) for i, (r, c) in enumerate(shapes)]
+    ws[5][:] = 0
+    hs[7] = hs[7].copy(); hs[7][3] = -1.0                     # a bad weight: that matrix alone is rejected
+    cfg, ref_cfg = P.cfg_pair()
+    dev = [P.to_device(w) for w in ws]
+    dh = [torch.from_numpy(h).cuda() for h in hs]
+    outs = [api.alloc_buffers(w.shape[0], w.shape[1], cfg) for w in ws]
+    api.soar_quantize_weighted_batch(dev, dh, cfg, outs)
+    torch.cuda.synchronize()
+    for i, (w, h, W, H, o) in enumerate(zip(ws, hs, dev, dh, outs)):
+        one = api.soar_quantize_weighted(W, H, cfg)
+        torch.cuda.synchronize()
+        r1, rb = one.read_result(), o.read_result()
+        assert rb.status == r1.status and rb.iters_run == r1.iters_run, i
+        if rb.status & api.STATUS_BAD_WEIGHT:
+            assert i == 7
+            continue
+        assert torch.equal(o.packed, one.packed) and torch.equal(o.scales, one.scales) and torch.equal(o.alpha, one.alpha), i
+        assert rb.sse == pytest.approx(r1.sse, rel=1e-12), i
+        if rb.status == 0 and i % 3 == 0:
+            g = P.GpuOut(o.packed.cpu().numpy(), o.scales.cpu().numpy(), float(o.alpha.cpu()[0]), rb, o)
+            P.assert_parity(g, R.quantize(w, ref_cfg, h=h), mismatch_cap=(0 if w.size < 16 * 20000 else None))
