@@ -84,7 +84,10 @@ def preset_cfg(api, preset: str, args=None, **over):
         over.update(n_dq=n_dq, n_beta=max(1, args.pairs // n_dq))
     if args is not None and args.iters is not None:
         over.update(max_iters=args.iters, early_stop_rel=0.0)
-    return api.soar_default_cfg(base, **over)
+    cfg = api.soar_default_cfg(base, **over)
+    if args is not None and getattr(args, "deterministic", False):
+        cfg.flags |= api.FLAG_DETERMINISTIC
+    return cfg
 
 
 def ref_cfg_of(R, cfg):
@@ -328,7 +331,7 @@ def run_ours(args):
             for W, o in zip(dev_w, outs):
                 api.soar_quantize(W, c, o, st)
             return
-        key = (c.max_iters, c.scale_layout)
+        key = (c.max_iters, c.scale_layout, c.flags)
         if key not in batch_ws:
             batch_ws[key] = torch.empty(api.soar_batch_workspace_bytes(dev_w, outs, c), dtype=torch.uint8, device="cuda")
         api.soar_quantize_batch(dev_w, c, outs, batch_ws[key], st)
@@ -975,6 +978,7 @@ def main():
     ap.add_argument("--sweep-dq", default="", help="comma-separated counts of E4M3 codes per block to time with beta = 1")
     ap.add_argument("--no-batch", action="store_true", help="one soar_quantize call per tensor instead of soar_quantize_batch")
     ap.add_argument("--graph", action="store_true", help="replay each step from a CUDA graph (no per-kernel trace)")
+    ap.add_argument("--deterministic", action="store_true", help="SOAR_FLAG_DETERMINISTIC: sums added in a fixed order")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-single-pass", action="store_true")

@@ -468,7 +468,7 @@ int soar_selftest_reciprocal(int lo_exp, int hi_exp, unsigned long long* out_mis
  * kernel (a consumer warp waiting for the tile its producer fetches) counts its polls and gives
  * up at a limit; the call then reports SOAR_STATUS_INTERNAL instead of hanging.  While the hook
  * is on, kernels launched afterwards fetch no tiles at all, so their consumers' waits run to
- * the limit (about four million polls, well under a second per kernel) with no copy in flight:
+ * the limit (a quarter of a million polls, about a second per kernel) with no copy in flight:
  * the pass kernels then return, the remaining kernels of the call return at once,
  * soar_result.status carries SOAR_STATUS_INTERNAL and the outputs are unspecified.  on = 0
  * restores normal operation.  Process-wide; not for production use.

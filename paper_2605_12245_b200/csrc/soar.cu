@@ -57,7 +57,7 @@ constexpr int kThreads = kTile + 32;           // plus one producer warp that is
 constexpr int kStages = 4;                     // depth of the shared-memory ring
 constexpr int kTileBytes = kTile * 32;         // 16 bf16 per block
 constexpr size_t kWsFixedBytes = 2048;
-constexpr unsigned int kWaitLimit = 1u << 22;  // mbarrier polls before a wait gives up
+constexpr unsigned int kWaitLimit = 1u << 18;  // mbarrier polls before a wait gives up (a poll takes microseconds: about a second)
 constexpr unsigned int kProducerSleepNs = 32;  // the producer's pause between polls for a free stage
 constexpr int kBracketMinBeta = 6;             // grids below this many multipliers are cheaper visited in full
 
