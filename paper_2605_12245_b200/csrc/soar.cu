@@ -59,7 +59,7 @@ constexpr int kTileBytes = kTile * 32;         // 16 bf16 per block
 constexpr size_t kWsFixedBytes = 2048;
 constexpr unsigned int kWaitLimit = 1u << 18;  // mbarrier polls before a wait gives up (a poll takes microseconds: about a second)
 constexpr unsigned int kProducerSleepNs = 32;  // the producer's pause between polls for a free stage
-constexpr int kBracketMinBeta = 6;             // grids below this many multipliers are cheaper visited in full
+constexpr int kBracketMinBeta = 2;             // the bracket needs two multipliers; a single one is modes 1-3
 
 struct Ws {
   unsigned int amax_bits;            // max over the tensor of the bf16 magnitude bit pattern
@@ -1011,7 +1011,8 @@ __device__ __forceinline__ void score_candidate(const Block& blk, const Fixed& f
 // are rounded and scored, which gives the winner of the whole grid.
 template <int kMode, bool kDet>   // 0: candidate grid, every multiplier visited; 1: one candidate scale (beta = 1), at most two
                        // codes; 2: the same with the coupled scale; 3: one candidate scale, any number of codes;
-                       // 4: candidate grid, only the multipliers that can win
+                       // 4: candidate grid, only the multipliers that can win; 5: the same for grids so short that
+                       // a block's bracket often reaches past their first or last multiplier
 __global__ void __launch_bounds__(kThreads, (kMode == 1 || kMode == 3) ? 3 : 2)
 iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, int keep, int prev_grid) {
   constexpr bool kSingle = kMode == 1 || kMode == 2 || kMode == 3;
@@ -1135,7 +1136,7 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
           if (g < best) { best = g; best_d = dc; }
         }
       }
-    } else if (kMode == 4) {
+    } else if (kMode == 4 || kMode == 5) {
       const int nd = d_hi - d_lo + 1;
       {
         // Typical block: two E4M3 codes at most, each with exactly two multipliers that can win (the one
@@ -1156,24 +1157,31 @@ iterate_kernel(const __grid_constant__ Batch bt, int t, int reverse, int emit, i
         // of the fast reciprocal, and the smallest one decides whether the exact integer sums hold
         const float s_hi = second ? s11 : s01;
         bool direct = nd <= 2 && fx.ok && recip_fast_ok(s00) && recip_fast_ok(s_hi) &&
-                      __fmul_rn(blk.bmax, recip_fast(s00)) <= 32.0f && s00 <= lo0 && s01 >= hi0;
-        if (second) direct = direct && s10 <= lo1 && s11 >= hi1;
+                      __fmul_rn(blk.bmax, recip_fast(s00)) <= 32.0f;
+        // Where the grid ends before the band does, one multiplier is all that can win: the first one when
+        // even its divisor lies beyond the band, the last one when even its divisor lies before it.  The
+        // pair then holds that multiplier twice.
+        // (Mode 5 only: a grid that spans 0.85 .. 1.15 holds the whole bracket of every regular block.)
+        const bool low0 = kMode == 5 && k0 == 0 && s00 >= hi0, high0 = kMode == 5 && k0 == n_beta - 2 && s01 <= lo0;
+        const bool low1 = kMode == 5 && k1 == 0 && s10 >= hi1, high1 = kMode == 5 && k1 == n_beta - 2 && s11 <= lo1;
+        direct = direct && ((s00 <= lo0 && s01 >= hi0) || low0 || high0);
+        if (second) direct = direct && ((s10 <= lo1 && s11 >= hi1) || low1 || high1);
         if (direct) {
           // error minus sum W^2 = 2 sd unit (rho * 4B - afix) with rho = sd / (8 unit): per code the two
           // candidates are ranked on the exact integer sums, the codes' winners compared once
           Scored a, c;
-          score_candidate(blk, fx, s00, sd0 * fx.inv8, a);
+          score_candidate(blk, fx, high0 ? s01 : s00, sd0 * fx.inv8, a);
           {
             Scored b2;
-            score_candidate(blk, fx, s01, sd0 * fx.inv8, b2);
+            score_candidate(blk, fx, low0 ? s00 : s01, sd0 * fx.inv8, b2);
             if (b2.e < a.e) a = b2;
           }
           double ga = 2.0 * sd0 * fx.unit * a.e;
           best_d = dc0;
           if (second) {
-            score_candidate(blk, fx, s10, sd1 * fx.inv8, c);
+            score_candidate(blk, fx, high1 ? s11 : s10, sd1 * fx.inv8, c);
             Scored b2;
-            score_candidate(blk, fx, s11, sd1 * fx.inv8, b2);
+            score_candidate(blk, fx, low1 ? s10 : s11, sd1 * fx.inv8, b2);
             const bool later = b2.e < c.e;
             if (later) c = b2;
             const double gc = 2.0 * sd1 * fx.unit * c.e;
@@ -1609,7 +1617,7 @@ weighted_amax_kernel(const __grid_constant__ Batch bt, const __grid_constant__ W
     unsigned int tile = 0;
     const int rc = ring_consume(ring, bt, n, v0, v1, ti, tile);
     if (rc != 0 || ti != cur) {
-      if (cur >= 0) {   // leaving tensor `cur`: hand over its maximum, its sum and the verdict on its weights
+      if (cur >= 0) {   // leaving tensor `cur`: hand over its maximum, its sum and the outcome of the weight check
         mx = __reduce_max_sync(0xFFFFFFFFu, mx);
         const bool any_bad = __any_sync(0xFFFFFFFFu, bad);
         if ((threadIdx.x & 31) == 0) {
@@ -2440,7 +2448,13 @@ int run_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void*
       // are visited (mode 4); the coupled arm and grids of a few multipliers visit them all (mode 0)
       const bool bracketed = !(cfg->flags & SOAR_FLAG_COUPLED_SCALE) && cfg->n_beta >= kBracketMinBeta &&
                              cfg->beta_step_pct >= 1;
-      const int mode = !single ? (bracketed ? 4 : 0)
+      // the brackets of two E4M3 codes around the Eq. 6 solution lie at multipliers 0.89 .. 1.13 (E4M3 values are
+      // at most an eighth apart): a grid from 0.85 to 1.15 or wider holds them whole (mode 4), a shorter one
+      // needs the straight-line path to know the grid's ends (mode 5)
+      const int half = cfg->n_beta / 2;
+      const bool spans = 100 - half * cfg->beta_step_pct <= 85 &&
+                         100 + (cfg->n_beta - 1 - half) * cfg->beta_step_pct >= 115;
+      const int mode = !single ? (bracketed ? (spans ? 4 : 5) : 0)
                                : ((cfg->flags & SOAR_FLAG_COUPLED_SCALE) ? 2 : (cfg->n_dq <= 2 ? 1 : 3));
       unsigned int g_it = 0;
       for (int t = t_lo; t < t_hi; ++t) {
@@ -2460,13 +2474,15 @@ int run_batch(const soar_tensor_desc* tensors, int n, const soar_cfg* cfg, void*
           else if (mode == 1) SOAR_LAUNCH_ITERATE(1, true);
           else if (mode == 2) SOAR_LAUNCH_ITERATE(2, true);
           else if (mode == 3) SOAR_LAUNCH_ITERATE(3, true);
-          else SOAR_LAUNCH_ITERATE(4, true);
+          else if (mode == 4) SOAR_LAUNCH_ITERATE(4, true);
+          else SOAR_LAUNCH_ITERATE(5, true);
         } else {
           if (mode == 0) SOAR_LAUNCH_ITERATE(0, false);
           else if (mode == 1) SOAR_LAUNCH_ITERATE(1, false);
           else if (mode == 2) SOAR_LAUNCH_ITERATE(2, false);
           else if (mode == 3) SOAR_LAUNCH_ITERATE(3, false);
-          else SOAR_LAUNCH_ITERATE(4, false);
+          else if (mode == 4) SOAR_LAUNCH_ITERATE(4, false);
+          else SOAR_LAUNCH_ITERATE(5, false);
         }
 #undef SOAR_LAUNCH_ITERATE
         g_last = g_it;
