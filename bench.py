@@ -137,11 +137,11 @@ def kernel_bytes_per_elem(name: str, cfg, t: int = 0) -> float:
 # belong to one version of the kernels: they are dropped when the device part of the source (everything above
 # the host-side section of soar.cu) no longer matches.
 NCU_TRAFFIC = {
-    "kernel_source_sha256_16": "7b27270025a5ae1d",
-    "bytes_per_elem": {"amax_kernel": 2.02, "init_kernel": 2.43, "iterate_kernel/single": 3.00,
-                       "iterate_kernel/grid": 3.45, "weighted_iterate_kernel": 4.58},
+    "kernel_source_sha256_16": "01bec268fb069bbc",
+    "bytes_per_elem": {"amax_kernel": 2.02, "init_kernel": 2.44, "iterate_kernel/single": 3.01,
+                       "iterate_kernel/grid": 3.47, "weighted_iterate_kernel": 4.57},
     "inst_per_block": {"amax_kernel": 125, "init_kernel": 218, "iterate_kernel/single": 258,
-                       "iterate_kernel/grid": 6117, "weighted_iterate_kernel": 14400},
+                       "iterate_kernel/grid": 490, "weighted_iterate_kernel": 1204},
 }
 
 
