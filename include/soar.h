@@ -112,7 +112,8 @@ typedef struct soar_result {
   int64_t wide_candidates;                  /* candidate evaluations that took the binary64
                                                accumulation path (scale far below block max);
                                                soar_quantize_weighted: blocks (summed over the
-                                               iterations) ranked by the exact loop            */
+                                               iterations) that visited every multiplier: the
+                                               coupled arm and blocks with a zero column weight */
   double trace_alpha[SOAR_MAX_ITERS + 1];   /* alpha^(0), then alpha of each executed iteration */
   double trace_sse[SOAR_MAX_ITERS + 1];     /* error of the start, then after each iteration */
 } soar_result;
