@@ -334,6 +334,37 @@ def test_host_pipeline_returns_what_direct_calls_return():
         assert hb.read_result().iters_run == want.result.iters_run
 
 
+def test_host_pipeline_weighted_objective_and_slot_capacity():
+    """The pipeline with column weights equals direct soar_quantize_weighted calls; a matrix that does not fit
+    the slots is refused before anything is enqueued."""
+    shapes = [(64, 1024), (130, 2064), (16, 256)]
+    ws = [WL.small_case(r, c, 230 + i, outlier_entry_frac=0.004, outlier_scale=30.0) for i, (r, c) in enumerate(shapes)]
+    hs = [torch.from_numpy(WL.column_weights(c, 240 + i)).cuda() for i, (r, c) in enumerate(shapes)]
+    cfg, _ = P.cfg_pair(max_iters=3)
+    hosts = []
+    for w in ws:
+        hb = api.alloc_host_buffers(w.shape[0], w.shape[1], cfg)
+        hb.W.copy_(torch.from_numpy(w.view(np.int16)).view(torch.bfloat16))
+        hosts.append(hb)
+    pipe = api.HostPipeline(shapes, cfg, depth=2, weighted=True)
+    pipe.run(hosts, hs)
+    pipe.synchronize()
+    for w, h, hb in zip(ws, hs, hosts):
+        want = api.soar_quantize_weighted(P.to_device(w), h, cfg)
+        torch.cuda.synchronize()
+        assert np.array_equal(hb.packed.numpy(), want.packed.cpu().numpy())
+        assert np.array_equal(hb.scales.numpy(), want.scales.cpu().numpy())
+        assert float(hb.alpha[0]) == float(want.alpha.cpu()[0])
+    big = api.alloc_host_buffers(512, 4096, cfg)             # larger than the slots
+    big.W.zero_()
+    marker = hosts[0].packed.clone()
+    with pytest.raises(api.SoarError, match="pipeline slot"):
+        pipe.run([hosts[0], big])
+    pipe.synchronize()
+    assert torch.equal(hosts[0].packed, marker)
+    pipe.close()
+
+
 def test_argument_errors_are_reported_on_the_host():
     w = P.to_device(WL.small_case(4, 64, 0))
     cfg = api.soar_default_cfg()
